@@ -1,0 +1,197 @@
+/*
+ * essa.h -- C ABI of the B200 (sm_100a) ESSA population-projection library.
+ *
+ * The library computes, for a whole CMA-ES population at once, the forward of the
+ * SVD-reparameterised LoRA attention projections of ESSA (arXiv 2507.04453):
+ *
+ *   Section 3, "LoRA + SVD parameterization":  W0 in R^{m x n} frozen, update B A with
+ *       A = U_A Sigma_A V_A^T (r x n),  B = U_B Sigma_B V_B^T (m x r), bases frozen;
+ *   Algorithm 1, line 7:  candidate k uses  W'_k = W0 + U_B diag(sB_k) V_B^T U_A diag(sA_k) V_A^T;
+ *   Section 3, "Evolutionary optimization" / Algorithm 1, line 5:  candidates are drawn from
+ *       N(m, step^2 C) out of one shared random stream and are regenerable from a seed.
+ *
+ * The GPU path never materialises A'_k, B'_k or W'_k: with M = V_B^T U_A (r x r, computed once
+ * per adapter) it evaluates   y_t = W0 x_t + U_B (sB_k .* (M (sA_k .* (V_A^T x_t)))),  k = cand(t).
+ *
+ * Conventions
+ *   - C linkage, plain pointers and sizes.  "dev" = device pointer on the context's GPU,
+ *     "host" = host pointer.  All matrices are row-major and dense unless a leading dimension
+ *     is given.  bf16 = upper 16 bits of an IEEE fp32; fp16 = IEEE binary16.
+ *   - Every call returns an int32 status: ESSA_OK (0) or a negative ESSA_ERR_* code; the text of
+ *     the most recent error on a context is available from essa_last_error().
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  Calls do not synchronise unless stated.
+ *   - Ownership: the caller owns every pointer it passes.  essa_load_adapter copies what it
+ *     needs into library-owned device memory (released by essa_free_adapter).  Device buffers
+ *     passed to asynchronous calls must stay valid until the stream has executed the call.
+ *   - Host-side validation happens before anything is launched.  Conditions only visible on
+ *     the device (a bounded wait that expired) are recorded in a device status word that
+ *     essa_get_status() reads; kernels never trap.
+ *   - There is no CPU fallback: without a usable sm_100 device essa_create fails with
+ *     ESSA_ERR_NO_DEVICE and nothing else can be called.
+ */
+#ifndef ESSA_H_
+#define ESSA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ESSA_OK 0
+#define ESSA_ERR_INVALID_ARG (-1)       /* null pointer, negative size, bad offsets, bad columns   */
+#define ESSA_ERR_UNSUPPORTED_SHAPE (-2) /* a size outside what the kernels are built for           */
+#define ESSA_ERR_ALLOC (-3)             /* device or host allocation failed                        */
+#define ESSA_ERR_CUDA (-4)              /* a CUDA runtime/driver call returned an error            */
+#define ESSA_ERR_DEVICE_TIMEOUT (-5)    /* a bounded device-side wait expired (see essa_get_status) */
+#define ESSA_ERR_NO_DEVICE (-6)         /* no CUDA device, or not compute capability 10.x          */
+
+#define ESSA_W0_BF16 0            /* W0 stored as bf16                                               */
+#define ESSA_W0_INT8_PERCHANNEL 1 /* W0[o][i] = q[o][i] * scale[o], q int8, scale fp16 per out-channel */
+
+#define ESSA_MAX_RANK 64
+
+typedef struct essa_ctx essa_ctx;         /* one per (process, device); not thread-safe */
+typedef struct essa_adapter essa_adapter; /* one per adapted projection matrix          */
+
+/* Library version (major*10000 + minor*100 + patch). Needs no device. */
+int32_t essa_version(void);
+/* Static description of a status code. Needs no device. */
+const char* essa_status_string(int32_t status);
+
+/* Create a context on CUDA device `device` (makes it current for the calling thread).
+ * Fails with ESSA_ERR_NO_DEVICE if there is no such device or it is not sm_100-class. */
+int32_t essa_create(essa_ctx** out, int32_t device);
+/* Release the context's scratch memory. Adapters must have been freed before. Synchronises the device. */
+int32_t essa_destroy(essa_ctx* ctx);
+/* Text of the last error recorded on ctx (never NULL; "" if none). Valid until the next call on ctx. */
+const char* essa_last_error(essa_ctx* ctx);
+/* Synchronise the device, then read (and clear) the device status word: 0, or the ESSA_ERR_* code a
+ * kernel recorded (ESSA_ERR_DEVICE_TIMEOUT if a bounded wait ran out; the affected output is undefined). */
+int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
+/* Pre-size the context's scratch memory (rank-path buffer, split-K workspace, host-call staging) for
+ * up to max_tokens tokens and max_d_out output channels so that later calls do not allocate. */
+int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out);
+
+/* Frozen data of one adapted projection (Section 3, "LoRA + SVD parameterization"). */
+typedef struct essa_adapter_desc {
+  int32_t d_in;     /* n: input features.  Must be a multiple of 64.                           */
+  int32_t d_out;    /* m: output features. Must be a multiple of 8.                            */
+  int32_t rank;     /* r: LoRA rank, 1..ESSA_MAX_RANK                                          */
+  int32_t w0_dtype; /* ESSA_W0_BF16 or ESSA_W0_INT8_PERCHANNEL                                 */
+  const void* W0;       /* [d_out][d_in], bf16 or int8                                         */
+  const void* w0_scale; /* [d_out] fp16 (INT8 only; NULL for bf16)                             */
+  const void* U_A;      /* [r][r]      bf16: left singular vectors of A                        */
+  const void* V_A;      /* [d_in][r]   bf16: right singular vectors of A                       */
+  const void* U_B;      /* [d_out][r]  bf16: left singular vectors of B                        */
+  const void* V_B;      /* [r][r]      bf16: right singular vectors of B                       */
+  int32_t on_device;    /* 0: the six pointers are host pointers; 1: device pointers           */
+} essa_adapter_desc;
+
+/* Copy and re-lay-out an adapter into library-owned device memory and precompute M = V_B^T U_A.
+ * The bases are used as given (orthonormality is not assumed).  Asynchronous on `stream` when the
+ * sources are device pointers; with host pointers the call returns after the copies have completed. */
+int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* desc, essa_adapter** out, void* stream);
+/* Free an adapter. Synchronises the device first. */
+int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* adapter);
+
+/* Draw a population (Section 3: x^(k) ~ N(m_t, sigma_t^2 C_t); Algorithm 1 line 5).
+ *   sigma_out[k][i] = mean[i] + step * sum_j Bfactor[i][j] * Dvec[j] * z_k[j],   k = 0..P-1,
+ * a sample of N(mean, step^2 * Bfactor diag(Dvec)^2 Bfactor^T).  z_k is a standard-normal vector
+ * taken from the shared stream: Philox4x32-10 with key = (seed low word, seed high word) and counter
+ * (j, k, 0, 0) yields four 32-bit words per block j; word w maps to u = (2*(w>>9)+1)*2^-24 and the
+ * word pairs (0,1) and (2,3) give coordinates 4j..4j+3 by Box-Muller
+ * (sqrt(-2 ln u0) * {cos, sin}(2 pi u1)).  A candidate therefore depends on <seed, k> only.
+ *   mean    [d] fp32 dev;  Bfactor [d][d] fp32 dev, row-major, or NULL for identity;
+ *   Dvec    [d] fp32 dev or NULL for ones;  sigma_out [P][d] fp32 dev (written).
+ * d >= 1; with a non-NULL Bfactor d <= 8192.  P = 0 is a legal no-op. */
+int32_t essa_sample_population(essa_ctx* ctx, const float* mean, float step, const float* Bfactor,
+                               const float* Dvec, int32_t d, uint64_t seed, int32_t P, float* sigma_out,
+                               void* stream);
+/* Same, for candidates k_begin .. k_begin+k_count-1 only (row 0 of sigma_out is candidate k_begin):
+ * what one worker of a candidate-sharded job regenerates locally. */
+int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float step, const float* Bfactor,
+                                     const float* Dvec, int32_t d, uint64_t seed, int32_t k_begin,
+                                     int32_t k_count, float* sigma_out, void* stream);
+
+/* Population-batched adapted projection (Algorithm 1 line 7 applied to every candidate's tokens).
+ *   x           [T][d_in] bf16 dev: all candidates' tokens stacked; token t belongs to the candidate
+ *               k with seg_offsets[k] <= t < seg_offsets[k+1];
+ *   seg_offsets [P+1] int32 dev, 0 = o[0] <= o[1] <= ... <= o[P] = T (empty segments allowed);
+ *   sigma       [P][ld_sigma] fp32 dev: candidate k reads sA_k = sigma[k][sA_col .. sA_col+r) and
+ *               sB_k = sigma[k][sB_col .. sB_col+r);
+ *   y           [T][d_out] bf16 dev (written): y_t = W0 x_t + U_B (sB_k .* (M (sA_k .* (V_A^T x_t)))).
+ * Accumulation is fp32 with one rounding to bf16 at the end; the rank-r intermediate is rounded to
+ * bf16 once before the up-projection.  T = 0 is a legal no-op.  The offsets are read on the device
+ * only: out-of-order offsets cannot cause out-of-bounds accesses but give unspecified candidates.
+ * May grow the context's scratch memory (a synchronising allocation) unless essa_reserve covered it. */
+int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* adapter, const void* x, int64_t T,
+                              const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma,
+                              int32_t sA_col, int32_t sB_col, void* y, void* stream);
+
+/* The same operation with HOST buffers: x, seg_offsets, sigma are copied to the device, the
+ * projection runs, y is copied back, and the call returns after `stream` has been synchronised.
+ * seg_offsets are validated on the host (ESSA_ERR_INVALID_ARG if not monotone from 0 to T).
+ * Pinned host memory makes the copies asynchronous with respect to each other; pageable works. */
+int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* adapter, const void* x_host, int64_t T,
+                                   const int32_t* seg_offsets_host, int32_t P, const float* sigma_host,
+                                   int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y_host,
+                                   void* stream);
+
+/* Straightforward CUDA-core (no tensor core, fp32 rank path) evaluation of the same formula, same
+ * arguments as essa_apply_projection.  A cross-check for the tensor-core path at sizes the CPU
+ * oracle cannot cover; never used by essa_apply_projection. */
+int32_t essa_apply_projection_simt(essa_ctx* ctx, const essa_adapter* adapter, const void* x, int64_t T,
+                                   const int32_t* seg_offsets, int32_t P, const float* sigma,
+                                   int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y, void* stream);
+
+/* How essa_apply_projection would schedule a call (host-only arithmetic; needs no device). */
+typedef struct essa_plan {
+  int32_t block_m;       /* tokens per tile                                          */
+  int32_t block_n;       /* output channels per tile                                 */
+  int32_t block_k;       /* reduction elements per pipeline stage                    */
+  int32_t stages;        /* shared-memory pipeline depth                             */
+  int32_t k_blocks;      /* stages' worth of K per tile, including the rank-path slab */
+  int32_t splits;        /* split-K factor (1 = none)                                */
+  int32_t tiles;         /* output tiles (token tiles x channel tiles)               */
+  int32_t grid;          /* CTAs launched by the main kernel                         */
+  int32_t down_splits;   /* split-K factor of the rank-path down-projection kernel   */
+  int32_t down_grid;     /* CTAs launched by the down-projection kernel              */
+  int64_t scratch_bytes; /* device scratch the call needs                            */
+} essa_plan;
+int32_t essa_plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T,
+                             int32_t sm_count, essa_plan* out);
+
+/* Per-kernel device time of essa_apply_projection calls, for roofline reporting.  Between
+ * essa_profile_begin and essa_profile_end every essa_apply_projection call records CUDA events on its
+ * stream before, between and after its two kernel launches (up to max_calls calls; later ones are not
+ * recorded).  essa_profile_end synchronises the device and sums the elapsed times per kernel. */
+typedef struct essa_profile {
+  double rank_down_ms;        /* total time of the rank-down kernel launches            */
+  double base_up_ms;          /* total time of the base-contraction + up-projection launches */
+  int32_t calls;              /* recorded calls (each = one launch of either kernel)    */
+  int32_t dropped;            /* calls made while profiling that did not fit max_calls  */
+} essa_profile;
+int32_t essa_profile_begin(essa_ctx* ctx, int32_t max_calls);
+int32_t essa_profile_end(essa_ctx* ctx, essa_profile* out);
+
+/* Host-side check of segment offsets: 0 = o[0] <= ... <= o[P] = T. Needs no device. */
+int32_t essa_validate_segments(const int32_t* seg_offsets_host, int32_t P, int64_t T);
+
+/* Diagnostics for parity tests (all outputs are device buffers, asynchronous on `stream`). */
+/* words_out[k_count][n_blocks][4] uint32: the raw Philox words of candidates k_begin.. (bit-exact check). */
+int32_t essa_debug_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count,
+                                int32_t n_blocks, uint32_t* words_out, void* stream);
+/* One Philox4x32-10 block for an arbitrary counter and key (host in, host out; synchronous). */
+int32_t essa_debug_philox(essa_ctx* ctx, const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+/* cand_out[t] = candidate index the projection kernels derive for token t (device binary search). */
+int32_t essa_debug_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P, int64_t T,
+                               int32_t* cand_out, void* stream);
+/* The adapter's precomputed core M = V_B^T U_A, copied to host as [r][r] fp32 (synchronous). */
+int32_t essa_debug_core_matrix(essa_ctx* ctx, const essa_adapter* adapter, float* M_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESSA_H_ */

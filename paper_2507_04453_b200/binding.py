@@ -1,0 +1,295 @@
+"""ctypes binding of libessa.so: argument marshalling only.
+
+Every function here forwards to the C entry point of the same name (``essa_`` prefix dropped on the
+methods of :class:`Context`); all arithmetic runs in the library's CUDA kernels.  torch supplies device
+memory (``tensor.data_ptr()``) and streams, nothing else.  There is no fallback: if the library has not
+been built, or no sm_100 GPU is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libessa.so")
+
+ESSA_OK = 0
+ESSA_ERR_INVALID_ARG = -1
+ESSA_ERR_UNSUPPORTED_SHAPE = -2
+ESSA_ERR_ALLOC = -3
+ESSA_ERR_CUDA = -4
+ESSA_ERR_DEVICE_TIMEOUT = -5
+ESSA_ERR_NO_DEVICE = -6
+ESSA_W0_BF16 = 0
+ESSA_W0_INT8_PERCHANNEL = 1
+
+EXPORTED_SYMBOLS = (
+    "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",
+    "essa_reserve", "essa_load_adapter", "essa_free_adapter", "essa_sample_population",
+    "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
+    "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
+    "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
+)
+
+
+class EssaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"essa status {status}: {message}")
+        self.status = status
+
+
+class AdapterDesc(C.Structure):
+    _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("rank", C.c_int32), ("w0_dtype", C.c_int32),
+                ("W0", C.c_void_p), ("w0_scale", C.c_void_p), ("U_A", C.c_void_p), ("V_A", C.c_void_p),
+                ("U_B", C.c_void_p), ("V_B", C.c_void_p), ("on_device", C.c_int32)]
+
+
+class Plan(C.Structure):
+    _fields_ = [("block_m", C.c_int32), ("block_n", C.c_int32), ("block_k", C.c_int32), ("stages", C.c_int32),
+                ("k_blocks", C.c_int32), ("splits", C.c_int32), ("tiles", C.c_int32), ("grid", C.c_int32),
+                ("down_splits", C.c_int32), ("down_grid", C.c_int32), ("scratch_bytes", C.c_int64)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class Profile(C.Structure):
+    _fields_ = [("rank_down_ms", C.c_double), ("base_up_ms", C.c_double), ("calls", C.c_int32), ("dropped", C.c_int32)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen libessa.so (built by ``python -m paper_2507_04453_b200.build``) and declare signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} not built: run `python -m paper_2507_04453_b200.build` (or __graft_entry__.build())")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float
+    sig = {
+        "essa_version": (i32, []),
+        "essa_status_string": (C.c_char_p, [i32]),
+        "essa_create": (i32, [C.POINTER(vp), i32]),
+        "essa_destroy": (i32, [vp]),
+        "essa_last_error": (C.c_char_p, [vp]),
+        "essa_get_status": (i32, [vp, C.POINTER(i32)]),
+        "essa_reserve": (i32, [vp, i64, i32, i32]),
+        "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
+        "essa_free_adapter": (i32, [vp, vp]),
+        "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
+        "essa_sample_population_range": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, vp]),
+        "essa_apply_projection": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
+        "essa_apply_projection_host": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
+        "essa_apply_projection_simt": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
+        "essa_plan_projection": (i32, [i32, i32, i32, i32, i64, i32, C.POINTER(Plan)]),
+        "essa_validate_segments": (i32, [vp, i32, i64]),
+        "essa_debug_stream_words": (i32, [vp, u64, i32, i32, i32, vp, vp]),
+        "essa_debug_philox": (i32, [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]),
+        "essa_debug_segment_map": (i32, [vp, vp, i32, i64, vp, vp]),
+        "essa_debug_core_matrix": (i32, [vp, vp, vp]),
+        "essa_profile_begin": (i32, [vp, i32]),
+        "essa_profile_end": (i32, [vp, C.POINTER(Profile)]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def plan_projection(d_in: int, d_out: int, rank: int, w0_dtype: int, T: int, sm_count: int = 148) -> dict:
+    """essa_plan_projection: the schedule a call would use (host arithmetic, no device needed)."""
+    lib = load_library()
+    p = Plan()
+    st = lib.essa_plan_projection(d_in, d_out, rank, w0_dtype, T, sm_count, C.byref(p))
+    if st != ESSA_OK:
+        raise EssaError(st, lib.essa_status_string(st).decode())
+    return p.as_dict()
+
+
+def validate_segments(seg_offsets, T: int) -> int:
+    """essa_validate_segments on a host int32 array; returns the status code."""
+    lib = load_library()
+    seg = np.ascontiguousarray(seg_offsets, dtype=np.int32)
+    return lib.essa_validate_segments(seg.ctypes.data_as(C.c_void_p), len(seg) - 1, T)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+class AdapterHandle:
+    def __init__(self, ctx: "Context", handle: int, d_in: int, d_out: int, rank: int, w0_dtype: int):
+        self.ctx, self.handle = ctx, handle
+        self.d_in, self.d_out, self.rank, self.w0_dtype = d_in, d_out, rank, w0_dtype
+
+    def free(self):
+        if self.handle:
+            self.ctx._check(self.ctx.lib.essa_free_adapter(self.ctx.handle, self.handle))
+            self.handle = None
+
+
+class Context:
+    """Owns one essa_ctx on a CUDA device."""
+
+    def __init__(self, device: int = 0):
+        import torch
+        self.lib = load_library()
+        self.torch = torch
+        self.device = torch.device("cuda", device)
+        h = C.c_void_p()
+        st = self.lib.essa_create(C.byref(h), device)
+        if st != ESSA_OK:
+            raise EssaError(st, self.lib.essa_status_string(st).decode())
+        self.handle = h.value
+        self.gpu_launches = 0  # kernels of this library enqueued through this context
+
+    # -- plumbing
+    def _check(self, st: int):
+        if st != ESSA_OK:
+            raise EssaError(st, self.lib.essa_last_error(self.handle).decode() or self.lib.essa_status_string(st).decode())
+
+    def close(self):
+        if self.handle:
+            self.lib.essa_destroy(self.handle)
+            self.handle = None
+
+    def get_status(self) -> int:
+        v = C.c_int32(0)
+        self._check(self.lib.essa_get_status(self.handle, C.byref(v)))
+        return v.value
+
+    def reserve(self, max_tokens: int, max_d_in: int, max_d_out: int):
+        self._check(self.lib.essa_reserve(self.handle, max_tokens, max_d_in, max_d_out))
+
+    # -- adapters
+    def load_adapter(self, ad) -> AdapterHandle:
+        """essa_load_adapter from a workloads.Adapter (host arrays; values already bf16/fp16/int8 exact)."""
+        torch = self.torch
+        bf = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16).contiguous()
+        keep = {k: bf(getattr(ad, k)) for k in ("U_A", "V_A", "U_B", "V_B")}
+        if ad.w0_dtype == "bf16":
+            keep["W0"] = bf(ad.W0)
+            dtype, scale_ptr = ESSA_W0_BF16, None
+        else:
+            keep["W0"] = torch.from_numpy(np.ascontiguousarray(ad.W0_q, dtype=np.int8))
+            keep["scale"] = torch.from_numpy(np.ascontiguousarray(ad.W0_scale, dtype=np.float16))
+            dtype, scale_ptr = ESSA_W0_INT8_PERCHANNEL, keep["scale"].data_ptr()
+        desc = AdapterDesc(ad.d_in, ad.d_out, ad.rank, dtype, keep["W0"].data_ptr(), scale_ptr, keep["U_A"].data_ptr(),
+                           keep["V_A"].data_ptr(), keep["U_B"].data_ptr(), keep["V_B"].data_ptr(), 0)
+        h = C.c_void_p()
+        self._check(self.lib.essa_load_adapter(self.handle, C.byref(desc), C.byref(h), _stream(None)))
+        return AdapterHandle(self, h.value, ad.d_in, ad.d_out, ad.rank, dtype)
+
+    def load_adapter_device(self, d_in, d_out, rank, W0, U_A, V_A, U_B, V_B, w0_scale=None) -> AdapterHandle:
+        """essa_load_adapter from device tensors (bf16 bases; W0 bf16, or int8 with fp16 w0_scale)."""
+        dtype = ESSA_W0_BF16 if w0_scale is None else ESSA_W0_INT8_PERCHANNEL
+        desc = AdapterDesc(d_in, d_out, rank, dtype, W0.data_ptr(), _ptr(w0_scale), U_A.data_ptr(), V_A.data_ptr(),
+                           U_B.data_ptr(), V_B.data_ptr(), 1)
+        h = C.c_void_p()
+        self._check(self.lib.essa_load_adapter(self.handle, C.byref(desc), C.byref(h), _stream(None)))
+        return AdapterHandle(self, h.value, d_in, d_out, rank, dtype)
+
+    # -- sampling
+    def sample_population(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, out=None, k_begin: int = 0,
+                          stream=None):
+        """essa_sample_population(_range): sigma[P, d] fp32 on the device."""
+        torch = self.torch
+        d = mean.numel()
+        if out is None:
+            out = torch.empty((P, d), dtype=torch.float32, device=self.device)
+        if k_begin == 0:
+            st = self.lib.essa_sample_population(self.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec), d,
+                                                 seed, P, out.data_ptr(), _stream(stream))
+        else:
+            st = self.lib.essa_sample_population_range(self.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec),
+                                                       d, seed, k_begin, P, out.data_ptr(), _stream(stream))
+        self._check(st)
+        self.gpu_launches += 1 if P > 0 else 0
+        return out
+
+    # -- projection
+    def _proj(self, fn, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream):
+        torch = self.torch
+        T = x.shape[0]
+        P = seg_offsets.numel() - 1
+        if out is None:
+            out = torch.empty((T, adapter.d_out), dtype=torch.bfloat16, device=self.device)
+        st = fn(self.handle, adapter.handle, x.data_ptr() if T else None, T, seg_offsets.data_ptr(), P, sigma.data_ptr(),
+                sigma.stride(0) if sigma.dim() == 2 else sigma.numel(), sA_col, sB_col, out.data_ptr() if T else None,
+                _stream(stream))
+        self._check(st)
+        return out
+
+    def apply_projection(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out=None, stream=None):
+        """essa_apply_projection: y[T, d_out] bf16 (two kernel launches: rank-down, base + up)."""
+        y = self._proj(self.lib.essa_apply_projection, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
+        self.gpu_launches += 2 if x.shape[0] else 0
+        return y
+
+    def apply_projection_simt(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out=None, stream=None):
+        """essa_apply_projection_simt: CUDA-core cross-check of the same formula."""
+        y = self._proj(self.lib.essa_apply_projection_simt, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
+        self.gpu_launches += 2 if x.shape[0] else 0
+        return y
+
+    def apply_projection_host(self, adapter, x_host, seg_offsets_host, sigma_host, sA_col: int, sB_col: int, y_host,
+                              stream=None):
+        """essa_apply_projection_host: host tensors in (bf16 x, int32 offsets, fp32 sigma), host bf16 y out."""
+        T = x_host.shape[0]
+        P = seg_offsets_host.numel() - 1
+        st = self.lib.essa_apply_projection_host(self.handle, adapter.handle, x_host.data_ptr(), T,
+                                                 seg_offsets_host.data_ptr(), P, sigma_host.data_ptr(),
+                                                 sigma_host.stride(0), sA_col, sB_col, y_host.data_ptr(), _stream(stream))
+        self._check(st)
+        self.gpu_launches += 2 if T else 0
+        return y_host
+
+    def profile_begin(self, max_calls: int):
+        """essa_profile_begin: record per-kernel CUDA events inside the following apply_projection calls."""
+        self._check(self.lib.essa_profile_begin(self.handle, max_calls))
+
+    def profile_end(self) -> dict:
+        """essa_profile_end: {rank_down_ms, base_up_ms, calls, dropped} summed over the recorded calls."""
+        p = Profile()
+        self._check(self.lib.essa_profile_end(self.handle, C.byref(p)))
+        return {"rank_down_ms": p.rank_down_ms, "base_up_ms": p.base_up_ms, "calls": p.calls, "dropped": p.dropped}
+
+    # -- diagnostics
+    def debug_philox(self, ctr, key):
+        c = (C.c_uint32 * 4)(*[int(v) for v in ctr])
+        k = (C.c_uint32 * 2)(*[int(v) for v in key])
+        o = (C.c_uint32 * 4)()
+        self._check(self.lib.essa_debug_philox(self.handle, c, k, o))
+        return [int(v) for v in o]
+
+    def debug_stream_words(self, seed: int, k_begin: int, k_count: int, n_blocks: int):
+        torch = self.torch
+        out = torch.empty((k_count, n_blocks, 4), dtype=torch.int32, device=self.device)
+        self._check(self.lib.essa_debug_stream_words(self.handle, seed, k_begin, k_count, n_blocks, out.data_ptr(), _stream(None)))
+        return out
+
+    def debug_segment_map(self, seg_offsets, T: int):
+        torch = self.torch
+        out = torch.empty((T,), dtype=torch.int32, device=self.device)
+        self._check(self.lib.essa_debug_segment_map(self.handle, seg_offsets.data_ptr(), seg_offsets.numel() - 1, T,
+                                                    out.data_ptr() if T else None, _stream(None)))
+        return out
+
+    def debug_core_matrix(self, adapter) -> np.ndarray:
+        M = np.empty((adapter.rank, adapter.rank), dtype=np.float32)
+        self._check(self.lib.essa_debug_core_matrix(self.handle, adapter.handle, M.ctypes.data_as(C.c_void_p)))
+        return M

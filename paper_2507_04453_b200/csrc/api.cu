@@ -1,0 +1,447 @@
+// C ABI of libessa.so: contexts, adapters, argument validation, scratch memory, host-buffer entry point.
+// The operations themselves live in sampler.cu (Section 3, "Evolutionary optimization"), proj_tc.cu and
+// proj_simt.cu (Algorithm 1, line 7).
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace essa {
+
+int32_t fail(essa_ctx* ctx, int32_t code, const std::string& msg) {
+  if (ctx) ctx->last_error = msg;
+  return code;
+}
+
+int32_t check_cuda(essa_ctx* ctx, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return ESSA_OK;
+  return fail(ctx, ESSA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+int32_t ensure_scratch(essa_ctx* ctx, Scratch& s, size_t bytes, bool zero, cudaStream_t stream) {
+  if (bytes <= s.bytes) return ESSA_OK;
+  // Growing replaces the buffer: earlier work that may still use the old one must have finished.
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaDeviceSynchronize (scratch growth)");
+  if (s.ptr) cudaFree(s.ptr);
+  s.ptr = nullptr;
+  s.bytes = 0;
+  size_t cap = bytes + bytes / 4;
+  cap = (cap + 255) & ~size_t(255);
+  e = cudaMalloc(&s.ptr, cap);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, ESSA_ERR_ALLOC, std::string("cudaMalloc of scratch failed: ") + cudaGetErrorString(e));
+  }
+  s.bytes = cap;
+  if (zero) {
+    e = cudaMemsetAsync(s.ptr, 0, cap, stream);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemsetAsync (scratch)");
+  }
+  return ESSA_OK;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void* base, uint64_t rows, uint64_t cols,
+                           uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols, int swizzle_bytes) {
+  if (!ctx->encode_tiled) return fail(ctx, ESSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+  if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (row_stride_bytes & 15) != 0)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "tensor base and row pitch must be 16-byte aligned");
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {row_stride_bytes};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                      : CU_TENSOR_MAP_SWIZZLE_NONE;
+  const CUtensorMapDataType dt = kind == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      out, dt, 2, const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    char buf[160];
+    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed (CUresult %d) rows=%llu cols=%llu box=%ux%u", (int)r,
+             (unsigned long long)rows, (unsigned long long)cols, box_rows, box_cols);
+    return fail(ctx, ESSA_ERR_CUDA, buf);
+  }
+  return ESSA_OK;
+}
+
+namespace {
+
+int32_t validate_projection_args(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,
+                                 int32_t P, const float* sigma, int32_t ld_sigma, int32_t sA_col, int32_t sB_col,
+                                 const void* y) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!a) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: adapter is NULL");
+  if (T < 0 || P < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: negative T or P");
+  if (T == 0) return ESSA_OK;
+  if (P == 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: T > 0 needs at least one candidate");
+  if (!x || !seg || !sigma || !y) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: NULL buffer");
+  if (sA_col < 0 || sB_col < 0 || sA_col + a->rank > ld_sigma || sB_col + a->rank > ld_sigma)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: sigma columns outside the row (ld_sigma)");
+  if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15))
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection: x and y must be 16-byte aligned");
+  return ESSA_OK;
+}
+
+void free_scratch(essa::Scratch& s) {
+  if (s.ptr) cudaFree(s.ptr);
+  s.ptr = nullptr;
+  s.bytes = 0;
+}
+
+}  // namespace
+}  // namespace essa
+
+using namespace essa;
+
+extern "C" {
+
+int32_t essa_version(void) { return 100; }
+
+const char* essa_status_string(int32_t status) {
+  switch (status) {
+    case ESSA_OK: return "ok";
+    case ESSA_ERR_INVALID_ARG: return "invalid argument";
+    case ESSA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case ESSA_ERR_ALLOC: return "allocation failed";
+    case ESSA_ERR_CUDA: return "CUDA error";
+    case ESSA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case ESSA_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+    default: return "unknown status";
+  }
+}
+
+int32_t essa_create(essa_ctx** out, int32_t device) {
+  if (!out) return ESSA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0 || device < 0 || device >= count) {
+    cudaGetLastError();
+    return ESSA_ERR_NO_DEVICE;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess || prop.major != 10) {
+    cudaGetLastError();
+    return ESSA_ERR_NO_DEVICE;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return ESSA_ERR_NO_DEVICE; }
+  essa_ctx* ctx = new (std::nothrow) essa_ctx();
+  if (!ctx) return ESSA_ERR_ALLOC;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    ctx->encode_tiled = fn;
+  else
+    cudaGetLastError();
+  if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return ESSA_ERR_ALLOC;
+  }
+  *out = ctx;
+  return ESSA_OK;
+}
+
+int32_t essa_destroy(essa_ctx* ctx) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  free_scratch(ctx->u_buf);
+  free_scratch(ctx->splitk_ws);
+  free_scratch(ctx->splitk_cnt);
+  free_scratch(ctx->simt_buf);
+  free_scratch(ctx->stage_x);
+  free_scratch(ctx->stage_y);
+  free_scratch(ctx->stage_off);
+  free_scratch(ctx->stage_sigma);
+  for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+  return ESSA_OK;
+}
+
+const char* essa_last_error(essa_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "context is NULL"; }
+
+int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
+  if (!ctx || !device_status) return ESSA_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaDeviceSynchronize");
+  e = cudaMemcpy(device_status, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(status)");
+  if (*device_status != 0) {
+    // A kernel gave up part-way: restore the invariants later calls rely on (zeroed split-K scratch).
+    cudaMemset(ctx->d_status, 0, sizeof(int32_t));
+    if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
+    if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
+  }
+  return ESSA_OK;
+}
+
+int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out) {
+  if (!ctx || max_tokens < 0 || max_d_in < 0 || max_d_out < 0) return ESSA_ERR_INVALID_ARG;
+  int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)max_tokens * kRankPadMax * 2, false, nullptr);
+  if (st != ESSA_OK) return st;
+  // split-K is only used while there are fewer tiles than SMs: at most sm_count tiles of 128 x 256 fp32
+  st = ensure_scratch(ctx, ctx->splitk_ws, (size_t)ctx->sm_count * 128 * 256 * 4, true, nullptr);
+  if (st != ESSA_OK) return st;
+  st = ensure_scratch(ctx, ctx->splitk_cnt, (size_t)ctx->sm_count * 4 * 4, true, nullptr);
+  if (st != ESSA_OK) return st;
+  st = ensure_scratch(ctx, ctx->stage_x, (size_t)max_tokens * max_d_in * 2, false, nullptr);
+  if (st != ESSA_OK) return st;
+  st = ensure_scratch(ctx, ctx->stage_y, (size_t)max_tokens * max_d_out * 2, false, nullptr);
+  if (st != ESSA_OK) return st;
+  return check_cuda(ctx, cudaDeviceSynchronize(), "cudaDeviceSynchronize");
+}
+
+int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapter** out, void* stream_v) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!d || !out) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: NULL descriptor or output");
+  *out = nullptr;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (d->d_in <= 0 || d->d_out <= 0 || d->rank <= 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: sizes must be positive");
+  if (d->rank > ESSA_MAX_RANK) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: rank > 64");
+  if (d->d_in % 64 != 0) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: d_in must be a multiple of 64");
+  if (d->d_out % 8 != 0) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: d_out must be a multiple of 8");
+  if (d->w0_dtype != ESSA_W0_BF16 && d->w0_dtype != ESSA_W0_INT8_PERCHANNEL)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: unknown w0_dtype");
+  if (!d->W0 || !d->U_A || !d->V_A || !d->U_B || !d->V_B) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: NULL matrix");
+  const bool int8 = d->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  if (int8 && !d->w0_scale) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: INT8 W0 needs w0_scale");
+
+  essa_adapter* a = new (std::nothrow) essa_adapter();
+  if (!a) return fail(ctx, ESSA_ERR_ALLOC, "load_adapter: host allocation failed");
+  a->d_in = d->d_in; a->d_out = d->d_out; a->rank = d->rank; a->w0_dtype = d->w0_dtype;
+  a->r_pad = ((d->rank + 15) / 16) * 16;
+  a->ext_blocks = int8 ? 2 : 1;
+  const size_t n = d->d_in, m = d->d_out, r = d->rank;
+  // The INT8 weights are widened once to bf16 (exact: |q| <= 127) for the tensor-core operand; the fp16
+  // per-channel scale is applied to the fp32 accumulator, so the dequantisation is exact.
+  const size_t w0_bytes = m * n * 2;
+  __nv_bfloat16 *dUA = nullptr, *dVB = nullptr;
+  cudaError_t e = cudaSuccess;
+  auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
+  alloc(&a->W0, w0_bytes);
+  if (int8) { alloc((void**)&a->w0_scale, m * 2); alloc((void**)&a->W0q, m * n); }
+  alloc((void**)&a->VAt, (size_t)kRankPadMax * n * 2);
+  alloc((void**)&a->UBp, (size_t)a->ext_blocks * m * kRankPadMax * 2);
+  alloc((void**)&a->U_B, m * r * 2);
+  alloc((void**)&a->V_A, n * r * 2);
+  alloc((void**)&a->M, (size_t)kRankPadMax * kRankPadMax * 4);
+  alloc((void**)&dUA, r * r * 2);
+  alloc((void**)&dVB, r * r * 2);
+  int32_t st = ESSA_OK;
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    st = fail(ctx, ESSA_ERR_ALLOC, std::string("load_adapter: cudaMalloc failed: ") + cudaGetErrorString(e));
+  }
+  const cudaMemcpyKind kind = d->on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  auto copy = [&](void* dst, const void* src, size_t bytes) {
+    if (st == ESSA_OK) st = check_cuda(ctx, cudaMemcpyAsync(dst, src, bytes, kind, stream), "load_adapter: copy");
+  };
+  copy(int8 ? (void*)a->W0q : a->W0, d->W0, int8 ? m * n : w0_bytes);
+  if (int8) copy(a->w0_scale, d->w0_scale, m * 2);
+  copy(a->U_B, d->U_B, m * r * 2);
+  copy(a->V_A, d->V_A, n * r * 2);
+  copy(dUA, d->U_A, r * r * 2);
+  copy(dVB, d->V_B, r * r * 2);
+  if (st == ESSA_OK && int8) st = launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(a->W0), m * n, stream);
+  if (st == ESSA_OK) st = launch_adapter_prep(ctx, a, dUA, dVB, stream);
+  if (st == ESSA_OK) {
+    const uint32_t rows[3] = {64, 128, 256};
+    for (int i = 0; i < 3 && st == ESSA_OK; ++i) {
+      st = make_tensor_map_2d(ctx, &a->tm_W0[i], 0, a->W0, m, n, n * 2, rows[i], 64, 128);
+      for (int e2 = 0; e2 < a->ext_blocks && st == ESSA_OK; ++e2)
+        st = make_tensor_map_2d(ctx, &a->tm_UBp[i][e2], 0, a->UBp + (size_t)e2 * m * kRankPadMax, m, kRankPadMax,
+                                kRankPadMax * 2, rows[i], 64, 128);
+    }
+    if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
+  }
+  // The temporaries (and, with host sources, the caller's buffers) are only needed until the copies and the
+  // preparation kernels have run.
+  if (cudaStreamSynchronize(stream) != cudaSuccess && st == ESSA_OK) st = check_cuda(ctx, cudaGetLastError(), "load_adapter: sync");
+  if (dUA) cudaFree(dUA);
+  if (dVB) cudaFree(dVB);
+  if (st != ESSA_OK) {
+    essa_free_adapter(ctx, a);
+    return st;
+  }
+  *out = a;
+  return ESSA_OK;
+}
+
+int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* a) {
+  if (!ctx || !a) return ESSA_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->M};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  delete a;
+  return ESSA_OK;
+}
+
+static int32_t validate_sampler(essa_ctx* ctx, const float* mean, int32_t d, int32_t k_begin, int32_t k_count,
+                                const float* sigma_out) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (d <= 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population: d must be positive");
+  if (k_count < 0 || k_begin < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population: negative candidate range");
+  if ((int64_t)k_begin + k_count > 0x7fffffffLL) return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population: candidate index overflow");
+  if (k_count > 0 && (!mean || !sigma_out)) return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population: NULL buffer");
+  return ESSA_OK;
+}
+
+int32_t essa_sample_population(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec,
+                               int32_t d, uint64_t seed, int32_t P, float* sigma_out, void* stream) {
+  const int32_t st = validate_sampler(ctx, mean, d, 0, P, sigma_out);
+  if (st != ESSA_OK) return st;
+  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, 0, P, sigma_out, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float step, const float* Bfactor,
+                                     const float* Dvec, int32_t d, uint64_t seed, int32_t k_begin, int32_t k_count,
+                                     float* sigma_out, void* stream) {
+  const int32_t st = validate_sampler(ctx, mean, d, k_begin, k_count, sigma_out);
+  if (st != ESSA_OK) return st;
+  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, k_begin, k_count, sigma_out,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,
+                              int32_t P, const float* sigma, int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y,
+                              void* stream) {
+  const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
+  if (st != ESSA_OK || T == 0) return st;
+  ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  return launch_projection_tc(ctx, a, g, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_apply_projection_simt(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,
+                                   int32_t P, const float* sigma, int32_t ld_sigma, int32_t sA_col, int32_t sB_col,
+                                   void* y, void* stream) {
+  const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
+  if (st != ESSA_OK || T == 0) return st;
+  ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  return launch_projection_simt(ctx, a, g, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* a, const void* x_host, int64_t T,
+                                   const int32_t* seg_host, int32_t P, const float* sigma_host, int32_t ld_sigma,
+                                   int32_t sA_col, int32_t sB_col, void* y_host, void* stream_v) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!a) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: adapter is NULL");
+  if (T < 0 || P < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: negative T or P");
+  if (T == 0) return ESSA_OK;
+  if (!x_host || !seg_host || !sigma_host || !y_host || P == 0)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: NULL buffer or no candidates");
+  if (essa_validate_segments(seg_host, P, T) != ESSA_OK)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: seg_offsets must rise from 0 to T");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  const size_t xb = (size_t)T * a->d_in * 2, yb = (size_t)T * a->d_out * 2, ob = (size_t)(P + 1) * 4,
+               sb = (size_t)P * ld_sigma * 4;
+  int32_t st;
+  if ((st = ensure_scratch(ctx, ctx->stage_x, xb, false, stream)) != ESSA_OK) return st;
+  if ((st = ensure_scratch(ctx, ctx->stage_y, yb, false, stream)) != ESSA_OK) return st;
+  if ((st = ensure_scratch(ctx, ctx->stage_off, ob, false, stream)) != ESSA_OK) return st;
+  if ((st = ensure_scratch(ctx, ctx->stage_sigma, sb, false, stream)) != ESSA_OK) return st;
+  cudaError_t e = cudaMemcpyAsync(ctx->stage_x.ptr, x_host, xb, cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, seg_host, ob, cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, stream);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
+  st = essa_apply_projection(ctx, a, ctx->stage_x.ptr, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
+                             static_cast<const float*>(ctx->stage_sigma.ptr), ld_sigma, sA_col, sB_col, ctx->stage_y.ptr,
+                             stream_v);
+  if (st != ESSA_OK) return st;
+  e = cudaMemcpyAsync(y_host, ctx->stage_y.ptr, yb, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  return check_cuda(ctx, e, "apply_projection_host: D2H");
+}
+
+int32_t essa_plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
+                             essa_plan* out) {
+  if (!out || d_in <= 0 || d_out <= 0 || rank <= 0 || T < 0) return ESSA_ERR_INVALID_ARG;
+  if (rank > ESSA_MAX_RANK || d_in % 64 != 0 || d_out % 8 != 0) return ESSA_ERR_UNSUPPORTED_SHAPE;
+  if (w0_dtype != ESSA_W0_BF16 && w0_dtype != ESSA_W0_INT8_PERCHANNEL) return ESSA_ERR_INVALID_ARG;
+  plan_projection(d_in, d_out, rank, w0_dtype, T, sm_count, out);
+  return ESSA_OK;
+}
+
+int32_t essa_profile_begin(essa_ctx* ctx, int32_t max_calls) {
+  if (!ctx || max_calls < 0) return ESSA_ERR_INVALID_ARG;
+  while (ctx->prof_events.size() < (size_t)max_calls * 3) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "cudaEventCreate");
+    ctx->prof_events.push_back(e);
+  }
+  ctx->prof_calls = 0;
+  ctx->prof_dropped = 0;
+  ctx->prof_on = true;
+  return ESSA_OK;
+}
+
+int32_t essa_profile_end(essa_ctx* ctx, essa_profile* out) {
+  if (!ctx || !out) return ESSA_ERR_INVALID_ARG;
+  ctx->prof_on = false;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaDeviceSynchronize");
+  out->rank_down_ms = out->base_up_ms = 0.0;
+  out->calls = ctx->prof_calls;
+  out->dropped = ctx->prof_dropped;
+  for (int c = 0; c < ctx->prof_calls; ++c) {
+    float a = 0.f, b = 0.f;
+    cudaEvent_t* ev = &ctx->prof_events[(size_t)c * 3];
+    if (cudaEventElapsedTime(&a, ev[0], ev[1]) != cudaSuccess || cudaEventElapsedTime(&b, ev[1], ev[2]) != cudaSuccess)
+      return check_cuda(ctx, cudaGetLastError(), "cudaEventElapsedTime");
+    out->rank_down_ms += a;
+    out->base_up_ms += b;
+  }
+  return ESSA_OK;
+}
+
+int32_t essa_validate_segments(const int32_t* seg, int32_t P, int64_t T) {
+  if (!seg || P < 0 || T < 0) return ESSA_ERR_INVALID_ARG;
+  if (seg[0] != 0) return ESSA_ERR_INVALID_ARG;
+  for (int32_t k = 0; k < P; ++k)
+    if (seg[k + 1] < seg[k]) return ESSA_ERR_INVALID_ARG;
+  return seg[P] == T ? ESSA_OK : ESSA_ERR_INVALID_ARG;
+}
+
+int32_t essa_debug_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count, int32_t n_blocks,
+                                uint32_t* words_out, void* stream) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (k_begin < 0 || k_count < 0 || n_blocks < 0 || ((int64_t)k_count * n_blocks > 0 && !words_out))
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "debug_stream_words: bad arguments");
+  return launch_stream_words(ctx, seed, k_begin, k_count, n_blocks, words_out, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_debug_philox(essa_ctx* ctx, const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  if (!ctx || !ctr || !key || !out) return ESSA_ERR_INVALID_ARG;
+  return launch_philox_once(ctx, ctr, key, out);
+}
+
+int32_t essa_debug_segment_map(essa_ctx* ctx, const int32_t* seg, int32_t P, int64_t T, int32_t* cand_out, void* stream) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (T < 0 || P < 0 || (T > 0 && (P == 0 || !seg || !cand_out)) || T > 0x7fffffffLL)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "debug_segment_map: bad arguments");
+  return launch_segment_map(ctx, seg, P, T, cand_out, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_debug_core_matrix(essa_ctx* ctx, const essa_adapter* a, float* M_host) {
+  if (!ctx || !a || !M_host) return ESSA_ERR_INVALID_ARG;
+  float full[kRankPadMax * kRankPadMax];
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(full, a->M, sizeof full, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "debug_core_matrix");
+  for (int j = 0; j < a->rank; ++j)
+    for (int i = 0; i < a->rank; ++i) M_host[j * a->rank + i] = full[j * kRankPadMax + i];
+  return ESSA_OK;
+}
+
+}  // extern "C"

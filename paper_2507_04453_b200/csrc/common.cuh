@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libessa.so (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "essa.h"
+
+namespace essa {
+
+constexpr int kRankPadMax = 64;  // rank-path operands are stored 64 columns wide (one 128-byte swizzle row)
+
+// Device status word values are the ESSA_ERR_* codes; 0 = nothing recorded.
+struct Scratch {
+  void* ptr = nullptr;
+  size_t bytes = 0;
+};
+
+}  // namespace essa
+
+struct essa_ctx {
+  int device = -1;
+  int sm_count = 0;
+  std::string last_error;
+  int32_t* d_status = nullptr;  // device status word
+  // Scratch owned by the context (grown on demand, never shrunk).
+  essa::Scratch u_buf;        // [T_cap][64] bf16: rank-path vector u_t, zero-padded to 64 columns
+  essa::Scratch splitk_ws;    // fp32 partial tiles for split-K (kept all-zero between calls)
+  essa::Scratch splitk_cnt;   // int32 arrival counters, one per output tile (kept zero between calls)
+  essa::Scratch simt_buf;     // [T_cap][64] fp32: rank-path vector of the CUDA-core cross-check path
+  essa::Scratch stage_x, stage_y, stage_off, stage_sigma;  // device staging of the host-buffer entry point
+  void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // essa_profile_begin/end: three events per recorded call
+  bool prof_on = false;
+  int prof_calls = 0, prof_dropped = 0;
+  std::vector<cudaEvent_t> prof_events;
+};
+
+struct essa_adapter {
+  int d_in = 0, d_out = 0, rank = 0, r_pad = 0, w0_dtype = 0;
+  void* W0 = nullptr;            // [d_out][d_in] bf16 (INT8 storage: the integer codes widened to bf16, unscaled)
+  int8_t* W0q = nullptr;         // [d_out][d_in] int8 codes as given (INT8 storage only)
+  __half* w0_scale = nullptr;    // [d_out] fp16 (INT8)
+  __nv_bfloat16* VAt = nullptr;  // [64][d_in]: V_A^T, rows >= rank are zero (K-major B operand of the down-projection)
+  __nv_bfloat16* UBp = nullptr;  // [ext][d_out][64]: U_B zero-padded to 64 columns; INT8: (U_B/scale) split hi, lo
+  __nv_bfloat16* U_B = nullptr;  // [d_out][rank] as given (CUDA-core path)
+  __nv_bfloat16* V_A = nullptr;  // [d_in][rank] as given (CUDA-core path)
+  float* M = nullptr;            // [64][64] fp32: M = V_B^T U_A zero-padded
+  int ext_blocks = 1;            // rank-path K-slabs appended to the base contraction (1 bf16, 2 INT8)
+  CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256
+  CUtensorMap tm_UBp[3][2];
+  CUtensorMap tm_VAt;
+};
+
+namespace essa {
+
+int32_t fail(essa_ctx* ctx, int32_t code, const std::string& msg);
+int32_t check_cuda(essa_ctx* ctx, cudaError_t e, const char* what);
+int32_t ensure_scratch(essa_ctx* ctx, Scratch& s, size_t bytes, bool zero, cudaStream_t stream);
+
+// kind: 0 = bf16, 1 = uint8/int8.  rows x cols (cols contiguous), box = box_rows x box_cols, swizzle bytes in {0,64,128}.
+int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void* base, uint64_t rows, uint64_t cols,
+                           uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols, int swizzle_bytes);
+
+// sampler.cu
+int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
+                       uint64_t seed, int32_t k_begin, int32_t k_count, float* sigma_out, cudaStream_t stream);
+int32_t launch_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count, int32_t n_blocks,
+                            uint32_t* words_out, cudaStream_t stream);
+int32_t launch_philox_once(essa_ctx* ctx, const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+int32_t launch_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P, int64_t T, int32_t* cand_out,
+                           cudaStream_t stream);
+
+// adapter_prep.cu
+int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream);
+int32_t launch_adapter_prep(essa_ctx* ctx, essa_adapter* a, const __nv_bfloat16* U_A, const __nv_bfloat16* V_B,
+                            cudaStream_t stream);
+
+struct ProjArgs {
+  const __nv_bfloat16* x;
+  int64_t T;
+  const int32_t* seg_offsets;
+  int32_t P;
+  const float* sigma;
+  int32_t ld_sigma, sA_col, sB_col;
+  __nv_bfloat16* y;
+};
+
+// proj_simt.cu / proj_tc.cu
+int32_t launch_projection_simt(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
+int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
+void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
+                     essa_plan* out);
+
+#ifdef __CUDACC__
+// Largest k in [0, P-1] with off[k] <= t (candidate that owns token t; empty segments own nothing).
+// Never reads outside off[0..P]; for offsets that are not monotone the result is some k in range.
+__device__ __forceinline__ int find_candidate(const int32_t* __restrict__ off, int P, int t) {
+  int lo = 0, hi = P;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(off + mid) <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+#endif
+
+}  // namespace essa

@@ -1,0 +1,698 @@
+// Tensor-core path of the population-batched adapted projection (Algorithm 1, line 7, for all candidates
+// at once):   y_t = W0 x_t + U_B u_t,   u_t = sB_k .* (M (sA_k .* (V_A^T x_t))),   k = cand(t),  M = V_B^T U_A.
+//
+// Two launches of one warp-specialised kernel template, both TMA -> shared memory -> tcgen05.mma -> TMEM:
+//   1. rank-down : D[128 tokens][r_pad] = x_tile . V_A^T over K = d_in; the epilogue owns one token per thread
+//                  (TMEM lane), looks up the token's candidate in the segment offsets, applies sA_k, the r x r
+//                  core M (shared memory) and sB_k in registers, and writes u_t as bf16 (64 columns, zero padded).
+//   2. base + up : D[128 tokens][BLOCK_N channels] = [x | u] . [W0 | U_B]^T : the base contraction over
+//                  K = d_in streams W0 once for the whole population, and the rank-r up-projection is one
+//                  more K-slab (two for INT8 W0) of the same accumulation.  Epilogue: fp32 -> (x scale[o]) -> bf16.
+// No per-candidate weight is ever formed; per-candidate state is the 2r singular values read in step 1.
+//
+// Small token counts (decode) use split-K over CTAs: partial tiles are added into an fp32 workspace with
+// vector reductions and the last CTA to arrive for a tile (atomic counter, no spinning) runs the epilogue
+// and re-zeroes the workspace.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocator + MMA issuer (one lane),
+// warps 2..5 = epilogue (warp w may access TMEM lanes 32*(w%4)..+31).  Two TMEM accumulators let the epilogue
+// of one tile overlap the main loop of the next.  Every mbarrier wait is bounded: on expiry the CTA records
+// ESSA_ERR_DEVICE_TIMEOUT in the status word, drains its outstanding copies, frees its TMEM and exits.
+#include "common.cuh"
+
+namespace essa {
+namespace {
+
+constexpr int BLOCK_M = 128;  // tokens per tile (UMMA M)
+constexpr int BLOCK_K = 64;   // 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr long long kWaitLimitCycles = 3000000000LL;  // ~1.5-2 s at B200 clocks
+constexpr int kSmemBudget = 227 * 1024;
+
+enum { EPI_STORE = 0, EPI_RANK = 1 };
+
+struct KParams {
+  int T;           // rows of the activation operand
+  int n_out;       // valid accumulator columns: d_out (EPI_STORE) or r_pad (EPI_RANK)
+  int main_kb;     // d_in / 64
+  int ext_kb;      // rank-path K-slabs appended after the main ones (EPI_STORE only)
+  int ext_ksteps;  // r_pad / 16: UMMA K-steps that matter in a rank-path slab
+  int m_tiles, n_tiles, splits;
+  // EPI_STORE
+  __nv_bfloat16* y;
+  int ldy;
+  const __half* scale;  // per-output-channel scale (INT8 W0) or nullptr
+  // EPI_RANK
+  const int32_t* seg;
+  int P;
+  const float* sigma;
+  int ld_sigma, sA_col, sB_col, r;
+  const float* M;  // [64][64] fp32
+  __nv_bfloat16* u;  // [T][64]
+  // split-K
+  float* ws;
+  int* cnt;
+  int32_t* status;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this or another thread ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c_inner, int c_outer, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(c_inner), "r"(c_outer), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// mbarrier arrives once all MMAs issued so far by this thread have completed (implies fence::before_thread_sync).
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  tmem_ld_wait();
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ float4 ld_cg_v4(const float* addr) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_cg_zero_v4(float* addr) {
+  asm volatile("st.global.cg.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(addr), "f"(0.f) : "memory");
+}
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte swizzle (what TMA wrote):
+// start address >> 4 | stride between 8-row groups (1024 B) >> 4 at bit 32 | descriptor version 1 at bit 46 |
+// layout type 2 (128-byte swizzle) at bit 61.  The leading-dimension offset is unused for this layout.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D = fp32 (bits 4-5 = 1), A = B = bf16 (bits 7-9 = 1, 10-12 = 1), both K-major,
+// N >> 3 at bits 17-22, M >> 4 at bits 24-28.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int BLOCK_N, int EPI>
+struct Cfg {
+  static constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;
+  static constexpr int B_BYTES = BLOCK_N * BLOCK_K * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int M_SMEM_BYTES = (EPI == EPI_RANK) ? BLOCK_N * BLOCK_N * 4 : 0;
+  static constexpr int AUX_BYTES = 1024;  // barriers, TMEM slot, flags
+  static constexpr int STAGES_RAW = (kSmemBudget - 1024 /*alignment slack*/ - AUX_BYTES - M_SMEM_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + M_SMEM_BYTES + AUX_BYTES;
+  // two accumulators, each starting at a power-of-two column offset
+  static constexpr int ACC_STRIDE = BLOCK_N <= 32 ? 32 : BLOCK_N <= 64 ? 64 : BLOCK_N <= 128 ? 128 : 256;
+  static constexpr int TMEM_COLS = 2 * ACC_STRIDE;
+  static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M = 128");
+  static_assert(STAGES >= 2, "pipeline too shallow");
+};
+
+// ------------------------------------------------------------------------------------------------ the kernel
+template <int BLOCK_N, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+essa_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2a,
+               const __grid_constant__ CUtensorMap tmB2b, const KParams p) {
+  using C = Cfg<BLOCK_N, EPI>;
+  constexpr int STAGES = C::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * C::A_BYTES;
+  float* smem_m = reinterpret_cast<float*>(smem + STAGES * C::STAGE_BYTES);
+  uint8_t* aux = smem + STAGES * C::STAGE_BYTES + C::M_SMEM_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aux);  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * STAGES + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  volatile int* epi_abort = reinterpret_cast<volatile int*>(tmem_slot + 3);
+
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
+  const uint32_t bar_tfull = bar_empty + 8 * STAGES, bar_tempty = bar_tfull + 16, bar_drain = bar_tempty + 16;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_kb = p.main_kb + p.ext_kb;
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int items = tiles * p.splits;
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    if (p.ext_kb > 0) { tma_prefetch_desc(&tmA2); tma_prefetch_desc(&tmB2a); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+    mbar_init(bar_drain, 1);
+    *abort_flag = 0;
+    *last_flag = 0;
+    *epi_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  if (EPI == EPI_RANK && warp >= 2) {
+    // core matrix M (zero-padded, row stride 64 in global) -> shared [BLOCK_N][BLOCK_N]
+    for (int idx = threadIdx.x - 64; idx < BLOCK_N * BLOCK_N; idx += kEpiThreads)
+      smem_m[idx] = p.M[(idx / BLOCK_N) * kRankPadMax + (idx % BLOCK_N)];
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // work item w -> (tile, split); tile -> (m_tile, n_tile) with n fastest; split s covers K-blocks [kb0, kb1)
+  auto item_range = [&](int w, int& m_tile, int& n_tile, int& kb0, int& kb1, int& tile) {
+    tile = w / p.splits;
+    const int s = w - tile * p.splits;
+    m_tile = tile / p.n_tiles;
+    n_tile = tile - m_tile * p.n_tiles;
+    const int base = total_kb / p.splits, rem = total_kb % p.splits;
+    kb0 = s * base + min(s, rem);
+    kb1 = kb0 + base + (s < rem ? 1 : 0);
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < items; w += gridDim.x) {
+        int m_tile, n_tile, kb0, kb1, tile;
+        item_range(w, m_tile, n_tile, kb0, kb1, tile);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t fb = bar_full + 8 * stage;
+          mbar_expect_tx(fb, C::STAGE_BYTES);
+          const uint32_t da = smem_u32(smem_a + stage * C::A_BYTES), db = smem_u32(smem_b + stage * C::B_BYTES);
+          if (kb < p.main_kb) {
+            tma_load_2d(da, &tmA, kb * BLOCK_K, m_tile * BLOCK_M, fb);
+            tma_load_2d(db, &tmB, kb * BLOCK_K, n_tile * BLOCK_N, fb);
+          } else {
+            tma_load_2d(da, &tmA2, 0, m_tile * BLOCK_M, fb);
+            tma_load_2d(db, (kb - p.main_kb) == 0 ? &tmB2a : &tmB2b, 0, n_tile * BLOCK_N, fb);
+          }
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // Aborting: let the copies already issued land before the CTA's shared memory is released.
+        const int outstanding = issued < STAGES ? issued : STAGES;
+        int s = stage;
+        uint32_t ph = phase;
+        for (int i = 0; i < outstanding; ++i) {
+          if (--s < 0) { s = STAGES - 1; ph ^= 1; }
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_full + 8 * s, ph) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < items; w += gridDim.x, ++it) {
+        int m_tile, n_tile, kb0, kb1, tile;
+        item_range(w, m_tile, n_tile, kb0, kb1, tile);
+        const int buf = it & 1;
+        const uint32_t use = (uint32_t)(it >> 1);
+        if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * C::ACC_STRIDE);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * C::A_BYTES));
+          const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * C::B_BYTES));
+          const int nk = (kb < p.main_kb) ? (BLOCK_K / UMMA_K) : p.ext_ksteps;
+          for (int k = 0; k < nk; ++k) {
+            // advancing K by 16 bf16 inside the swizzled row = +32 bytes = +2 in the (addr >> 4) field
+            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(bar_empty + 8 * stage);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(bar_tfull + 8 * buf);
+      }
+      if (!ok) {
+        // make sure no MMA is still writing TMEM / reading shared memory when the CTA tears down
+        umma_commit(bar_drain);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < kWaitLimitCycles) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quad = warp & 3;                   // TMEM lane quadrant this warp may access
+    const int row_in_tile = quad * 32 + lane;    // accumulator row (token within the tile) owned by this thread
+    const int epi_tid = threadIdx.x - 64;
+    int it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; ok && w < items; w += gridDim.x, ++it) {
+      int m_tile, n_tile, kb0, kb1, tile;
+      item_range(w, m_tile, n_tile, kb0, kb1, tile);
+      const int buf = it & 1;
+      const uint32_t use = (uint32_t)(it >> 1);
+      // lane 0 polls (bounded); the warp then takes one common decision
+      int got = 1;
+      if (lane == 0) got = mbar_wait(bar_tfull + 8 * buf, use & 1, abort_flag, p.status) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (p.splits > 1) {
+        // the four epilogue warps meet at named barriers below, so they must also agree on aborting
+        epi_bar_sync();
+        if (epi_tid == 0) *epi_abort = *abort_flag;
+        epi_bar_sync();
+        if (*epi_abort) got = 0;
+      }
+      if (!got) { ok = false; break; }
+      while (!mbar_try_wait(bar_tfull + 8 * buf, use & 1)) {}  // already complete: returns at once (acquire for every lane)
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_STRIDE);
+      const int t = m_tile * BLOCK_M + row_in_tile;
+      const bool row_ok = t < p.T;
+      const int col_base = n_tile * BLOCK_N;
+      float* ws_tile = p.ws + (size_t)tile * BLOCK_M * BLOCK_N;  // [BLOCK_N/4][128 rows][4]
+
+      if (p.splits > 1) {
+        // partial tile -> fp32 workspace (coalesced: consecutive rows are 16 bytes apart)
+#pragma unroll 1
+        for (int c = 0; c < BLOCK_N / 16; ++c) {
+          if (col_base + c * 16 >= p.n_out) break;
+          float v[16];
+          tmem_ld16(t_addr + c * 16, v);
+          if (row_ok) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+              red_add_v4(ws_tile + ((size_t)(c * 4 + g) * BLOCK_M + row_in_tile) * 4, v[4 * g], v[4 * g + 1], v[4 * g + 2],
+                         v[4 * g + 3]);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+        __threadfence();
+        epi_bar_sync();
+        if (epi_tid == 0) {
+          const int prev = atomicAdd(p.cnt + tile, 1);
+          const int last = (prev == p.splits - 1);
+          if (last) p.cnt[tile] = 0;  // all arrivals are in; leave the counter clean for the next call
+          *last_flag = last;
+        }
+        epi_bar_sync();
+        const bool last = *last_flag != 0;
+        epi_bar_sync();  // everyone has read the flag before a later item overwrites it
+        if (!last) continue;
+        __threadfence();
+      }
+
+      if constexpr (EPI == EPI_STORE) {
+#pragma unroll 1
+        for (int c = 0; c < BLOCK_N / 16; ++c) {
+          const int col0 = col_base + c * 16;
+          if (col0 >= p.n_out) break;
+          float v[16] = {};
+          if (p.splits > 1) {
+            if (row_ok) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                float* a = ws_tile + ((size_t)(c * 4 + g) * BLOCK_M + row_in_tile) * 4;
+                const float4 f = ld_cg_v4(a);
+                st_cg_zero_v4(a);
+                v[4 * g] = f.x; v[4 * g + 1] = f.y; v[4 * g + 2] = f.z; v[4 * g + 3] = f.w;
+              }
+            }
+          } else {
+            tmem_ld16(t_addr + c * 16, v);
+          }
+          if (row_ok) {
+            if (p.scale != nullptr) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v[i] *= (col0 + i < p.n_out) ? __half2float(__ldg(p.scale + col0 + i)) : 0.f;
+            }
+            __nv_bfloat16* dst = p.y + (size_t)t * p.ldy + col0;
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+              if (col0 + 8 * g < p.n_out) {  // d_out is a multiple of 8: a group of 8 is all in or all out
+                uint4 o;
+                o.x = pack_bf16x2(v[8 * g + 0], v[8 * g + 1]);
+                o.y = pack_bf16x2(v[8 * g + 2], v[8 * g + 3]);
+                o.z = pack_bf16x2(v[8 * g + 4], v[8 * g + 5]);
+                o.w = pack_bf16x2(v[8 * g + 6], v[8 * g + 7]);
+                *reinterpret_cast<uint4*>(dst + 8 * g) = o;
+              }
+            }
+          }
+        }
+      } else {
+        // rank path, one token per thread:  q = sA_k .* p ;  v = M q ;  u = sB_k .* v
+        constexpr int R = BLOCK_N;
+        float q[R];
+#pragma unroll
+        for (int c = 0; c < R / 16; ++c) {
+          float v[16] = {};
+          if (p.splits > 1) {
+            if (row_ok) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                float* a = ws_tile + ((size_t)(c * 4 + g) * BLOCK_M + row_in_tile) * 4;
+                const float4 f = ld_cg_v4(a);
+                st_cg_zero_v4(a);
+                v[4 * g] = f.x; v[4 * g + 1] = f.y; v[4 * g + 2] = f.z; v[4 * g + 3] = f.w;
+              }
+            }
+          } else {
+            tmem_ld16(t_addr + c * 16, v);
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) q[c * 16 + i] = v[i];
+        }
+        if (row_ok) {
+          const int k = find_candidate(p.seg, p.P, t);
+          const float* srow = p.sigma + (size_t)k * p.ld_sigma;
+#pragma unroll
+          for (int i = 0; i < R; ++i) q[i] = (i < p.r) ? q[i] * __ldg(srow + p.sA_col + i) : 0.f;
+          uint32_t packed[kRankPadMax / 2];
+#pragma unroll
+          for (int j2 = 0; j2 < R / 2; ++j2) {
+            float uu[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int j = 2 * j2 + h;
+              float acc = 0.f;
+#pragma unroll
+              for (int i4 = 0; i4 < R / 4; ++i4) {
+                const float4 mm = *reinterpret_cast<const float4*>(smem_m + j * R + 4 * i4);
+                acc = fmaf(mm.x, q[4 * i4], acc);
+                acc = fmaf(mm.y, q[4 * i4 + 1], acc);
+                acc = fmaf(mm.z, q[4 * i4 + 2], acc);
+                acc = fmaf(mm.w, q[4 * i4 + 3], acc);
+              }
+              uu[h] = (j < p.r) ? acc * __ldg(srow + p.sB_col + j) : 0.f;
+            }
+            packed[j2] = pack_bf16x2(uu[0], uu[1]);
+          }
+#pragma unroll
+          for (int j2 = R / 2; j2 < kRankPadMax / 2; ++j2) packed[j2] = 0u;
+          uint4* dst = reinterpret_cast<uint4*>(p.u + (size_t)t * kRankPadMax);
+#pragma unroll
+          for (int g = 0; g < kRankPadMax / 8; ++g)
+            dst[g] = make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
+        }
+      }
+      if (p.splits == 1) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+template <int BLOCK_N, int EPI>
+int32_t launch_one(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2,
+                   const CUtensorMap& tmB2a, const CUtensorMap& tmB2b, const KParams& p, int grid, cudaStream_t stream) {
+  using C = Cfg<BLOCK_N, EPI>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(essa_tc_kernel<BLOCK_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         C::SMEM_BYTES);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_tc_kernel)");
+    attr_done = true;
+  }
+  essa_tc_kernel<BLOCK_N, EPI><<<grid, kThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, tmA2, tmB2a, tmB2b, p);
+  return check_cuda(ctx, cudaGetLastError(), "essa_tc_kernel launch");
+}
+
+int stages_for(int block_n, bool rank_epi) {
+  const int stage_bytes = BLOCK_M * BLOCK_K * 2 + block_n * BLOCK_K * 2;
+  const int m_bytes = rank_epi ? block_n * block_n * 4 : 0;
+  int s = (kSmemBudget - 1024 - 1024 - m_bytes) / stage_bytes;
+  return s > 8 ? 8 : s;
+}
+
+// Relative cost (in SM cycles) of running `tiles` output tiles of width bn with a given split-K factor.
+double schedule_cost(int tiles, int bn, int total_kb, int splits, int sm) {
+  const double load = 2.0 * (BLOCK_M + bn);  // cycles to bring one K-block of A and B from L2 at ~64 B/clk
+  const double mma = 2.0 * bn;               // 4 UMMAs of 128 x bn x 16
+  const double per_kb = load > mma ? load : mma;
+  const int kb_per_item = (total_kb + splits - 1) / splits;
+  const double epilogue = 10.0 * bn * (splits > 1 ? 3.0 : 1.0);
+  const double fixed = 3000.0;  // prologue, pipeline fill, teardown
+  const long long items = (long long)tiles * splits;
+  const double waves = (double)((items + sm - 1) / sm);
+  return waves * (kb_per_item * per_kb + epilogue) + fixed;
+}
+
+}  // namespace
+
+void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
+                     essa_plan* out) {
+  const int sm = sm_count > 0 ? sm_count : 148;
+  const int m_tiles = (int)((T + BLOCK_M - 1) / BLOCK_M);
+  const int main_kb = d_in / BLOCK_K;
+  const int ext = (w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? 2 : 1;
+  const int total_kb = main_kb + ext;
+  const int r_pad = ((rank + 15) / 16) * 16;
+  int best_bn = 256, best_splits = 1;
+  double best = 1e300;
+  const int bns[3] = {256, 128, 64};
+  for (int bi = 0; bi < 3; ++bi) {
+    const int bn = bns[bi];
+    const int n_tiles = (d_out + bn - 1) / bn;
+    const long long tiles = (long long)m_tiles * n_tiles;
+    if (tiles == 0) continue;
+    const int max_splits = tiles >= sm ? 1 : (int)((sm + tiles - 1) / tiles);
+    for (int s = 1; s <= max_splits && s <= total_kb; ++s) {
+      // padded-channel waste counts as extra work
+      const double waste = (double)(n_tiles * bn) / (double)d_out;
+      const double c = schedule_cost((int)(tiles > 0x7fffffff ? 0x7fffffff : tiles), bn, total_kb, s, sm) * (tiles >= sm ? waste : 1.0);
+      if (c < best) { best = c; best_bn = bn; best_splits = s; }
+    }
+  }
+  out->block_m = BLOCK_M;
+  out->block_n = best_bn;
+  out->block_k = BLOCK_K;
+  out->stages = stages_for(best_bn, false);
+  out->k_blocks = total_kb;
+  out->splits = best_splits;
+  const int n_tiles = (d_out + best_bn - 1) / best_bn;
+  out->tiles = m_tiles * n_tiles;
+  const long long items = (long long)out->tiles * best_splits;
+  out->grid = (int)(items < sm ? items : sm);
+  // rank-down kernel: one tile per 128 tokens, N = r_pad; split K until the SMs are covered
+  int ds = 1;
+  if (m_tiles > 0 && m_tiles < sm) {
+    ds = sm / m_tiles;
+    if (ds > main_kb) ds = main_kb;
+    if (ds < 1) ds = 1;
+  }
+  out->down_splits = ds;
+  const long long ditems = (long long)m_tiles * ds;
+  out->down_grid = (int)(ditems < sm ? ditems : sm);
+  int64_t scratch = T * kRankPadMax * 2;
+  if (best_splits > 1) scratch += (int64_t)out->tiles * BLOCK_M * best_bn * 4 + (int64_t)out->tiles * 4;
+  if (ds > 1) scratch += (int64_t)m_tiles * BLOCK_M * r_pad * 4 + (int64_t)m_tiles * 4;
+  out->scratch_bytes = scratch;
+}
+
+int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, cudaStream_t stream) {
+  if (g.T == 0) return ESSA_OK;
+  if (g.T > 0x7fffffffLL - BLOCK_M) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: T too large");
+  essa_plan pl;
+  plan_projection(a->d_in, a->d_out, a->rank, a->w0_dtype, g.T, ctx->sm_count, &pl);
+  const int m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
+
+  int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)g.T * kRankPadMax * 2, false, stream);
+  if (st != ESSA_OK) return st;
+  size_t ws_need = 0, cnt_need = 0;
+  if (pl.splits > 1) { ws_need = (size_t)pl.tiles * BLOCK_M * pl.block_n * 4; cnt_need = (size_t)pl.tiles * 4; }
+  if (pl.down_splits > 1) {
+    ws_need = ws_need > (size_t)m_tiles * BLOCK_M * a->r_pad * 4 ? ws_need : (size_t)m_tiles * BLOCK_M * a->r_pad * 4;
+    cnt_need = cnt_need > (size_t)m_tiles * 4 ? cnt_need : (size_t)m_tiles * 4;
+  }
+  if (ws_need) {
+    st = ensure_scratch(ctx, ctx->splitk_ws, ws_need, true, stream);
+    if (st != ESSA_OK) return st;
+    st = ensure_scratch(ctx, ctx->splitk_cnt, cnt_need, true, stream);
+    if (st != ESSA_OK) return st;
+  }
+  __nv_bfloat16* u = static_cast<__nv_bfloat16*>(ctx->u_buf.ptr);
+
+  CUtensorMap tm_x, tm_u;
+  st = make_tensor_map_2d(ctx, &tm_x, 0, g.x, (uint64_t)g.T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2, BLOCK_M, BLOCK_K, 128);
+  if (st != ESSA_OK) return st;
+  st = make_tensor_map_2d(ctx, &tm_u, 0, u, (uint64_t)g.T, kRankPadMax, kRankPadMax * 2, BLOCK_M, BLOCK_K, 128);
+  if (st != ESSA_OK) return st;
+
+  cudaEvent_t* ev = nullptr;
+  if (ctx->prof_on) {
+    if ((size_t)(ctx->prof_calls + 1) * 3 <= ctx->prof_events.size()) ev = &ctx->prof_events[(size_t)ctx->prof_calls++ * 3];
+    else ++ctx->prof_dropped;
+  }
+  if (ev) cudaEventRecord(ev[0], stream);
+
+  // ---- launch 1: rank-down
+  KParams kp{};
+  kp.T = (int)g.T;
+  kp.n_out = a->r_pad;
+  kp.main_kb = a->d_in / BLOCK_K;
+  kp.ext_kb = 0;
+  kp.ext_ksteps = 0;
+  kp.m_tiles = m_tiles;
+  kp.n_tiles = 1;
+  kp.splits = pl.down_splits;
+  kp.seg = g.seg_offsets;
+  kp.P = g.P;
+  kp.sigma = g.sigma;
+  kp.ld_sigma = g.ld_sigma;
+  kp.sA_col = g.sA_col;
+  kp.sB_col = g.sB_col;
+  kp.r = a->rank;
+  kp.M = a->M;
+  kp.u = u;
+  kp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
+  kp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
+  kp.status = ctx->d_status;
+  switch (a->r_pad) {
+    case 16: st = launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+    case 32: st = launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+    case 48: st = launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+    case 64: st = launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+    default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
+  }
+  if (st != ESSA_OK) return st;
+  if (ev) cudaEventRecord(ev[1], stream);
+
+  // ---- launch 2: base contraction + up-projection
+  KParams mp{};
+  mp.T = (int)g.T;
+  mp.n_out = a->d_out;
+  mp.main_kb = a->d_in / BLOCK_K;
+  mp.ext_kb = a->ext_blocks;
+  mp.ext_ksteps = a->r_pad / UMMA_K;
+  mp.m_tiles = m_tiles;
+  mp.n_tiles = (a->d_out + pl.block_n - 1) / pl.block_n;
+  mp.splits = pl.splits;
+  mp.y = g.y;
+  mp.ldy = a->d_out;
+  mp.scale = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? a->w0_scale : nullptr;
+  mp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
+  mp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
+  mp.status = ctx->d_status;
+  const int bi = pl.block_n == 64 ? 0 : pl.block_n == 128 ? 1 : 2;
+  const CUtensorMap& tmW = a->tm_W0[bi];
+  const CUtensorMap& tmU0 = a->tm_UBp[bi][0];
+  const CUtensorMap& tmU1 = a->tm_UBp[bi][a->ext_blocks > 1 ? 1 : 0];
+  switch (pl.block_n) {
+    case 64: st = launch_one<64, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, pl.grid, stream); break;
+    case 128: st = launch_one<128, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, pl.grid, stream); break;
+    default: st = launch_one<256, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, pl.grid, stream); break;
+  }
+  if (ev) cudaEventRecord(ev[2], stream);
+  return st;
+}
+
+}  // namespace essa

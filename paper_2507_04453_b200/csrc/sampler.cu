@@ -1,0 +1,187 @@
+// Candidate sampling: sigma_k = mean + step * Bfactor (Dvec .* z_k), z_k from a counter-based stream
+// (Section 3, "Evolutionary optimization": x^(k) ~ N(m_t, sigma_t^2 C_t), regenerable from a seed;
+//  Algorithm 1, line 5).  Philox4x32-10 (Salmon et al., SC'11) + Box-Muller, all in this file.
+#include "common.cuh"
+
+namespace essa {
+namespace {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(kPhiloxM0, c.x), lo0 = kPhiloxM0 * c.x;
+    const uint32_t hi1 = __umulhi(kPhiloxM1, c.z), lo1 = kPhiloxM1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += kWeyl0;
+    k.y += kWeyl1;
+  }
+  return c;
+}
+
+// Word -> uniform strictly inside (0,1): (2*(w>>9)+1) * 2^-24; the integer is < 2^24, so the float is exact.
+__device__ __forceinline__ float uniform_open01(uint32_t w) { return static_cast<float>(2u * (w >> 9) + 1u) * 0x1p-24f; }
+
+__device__ __forceinline__ void box_muller(uint32_t w_radius, uint32_t w_angle, float& z0, float& z1) {
+  const float rho = sqrtf(-2.0f * logf(uniform_open01(w_radius)));
+  float s, c;
+  sincospif(2.0f * uniform_open01(w_angle), &s, &c);  // angle = 2*pi*u
+  z0 = rho * c;
+  z1 = rho * s;
+}
+
+// Four standard normals: coordinates 4j..4j+3 of candidate k.
+__device__ __forceinline__ float4 normals_block(uint2 key, uint32_t j, uint32_t k) {
+  const uint4 w = philox4x32_10(make_uint4(j, k, 0u, 0u), key);
+  float4 z;
+  box_muller(w.x, w.y, z.x, z.y);
+  box_muller(w.z, w.w, z.z, z.w);
+  return z;
+}
+
+// Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
+__global__ void sample_diag_kernel(const float* __restrict__ mean, float step, const float* __restrict__ Dvec, int d,
+                                   uint2 key, int k_begin, int k_count, float* __restrict__ sigma_out) {
+  const int nb = (d + 3) >> 2;
+  const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (idx >= (long long)k_count * nb) return;
+  const int kk = (int)(idx / nb), j = (int)(idx % nb);
+  const float4 z = normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk));
+  const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int i = 4 * j + e;
+    if (i < d) {
+      const float w = Dvec ? Dvec[i] * zz[e] : zz[e];
+      sigma_out[(size_t)kk * d + i] = fmaf(step, w, mean[i]);
+    }
+  }
+}
+
+// Full covariance factor.  blockIdx.x = group of kCand candidates, blockIdx.y = tile of kRows rows of Bfactor.
+// Phase 1: w[c][j] = Dvec[j] * z_c[j] into shared memory.  Phase 2: one warp per row i, lanes stride over j,
+// shuffle reduction; lane 0 writes mean[i] + step * acc.
+constexpr int kCand = 4, kRows = 64, kSamplerThreads = 256;
+
+__global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const float* __restrict__ mean, float step,
+                                                                      const float* __restrict__ Bfactor,
+                                                                      const float* __restrict__ Dvec, int d, uint2 key,
+                                                                      int k_begin, int k_count,
+                                                                      float* __restrict__ sigma_out) {
+  extern __shared__ float w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
+  const int nb = (d + 3) >> 2, d4 = nb * 4;
+  const int kk0 = blockIdx.x * kCand;
+  for (int idx = threadIdx.x; idx < kCand * nb; idx += blockDim.x) {
+    const int c = idx / nb, j = idx % nb;
+    float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (kk0 + c < k_count) z = normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk0 + c));
+    const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = 4 * j + e;
+      w_smem[c * d4 + i] = (i < d) ? (Dvec ? Dvec[i] * zz[e] : zz[e]) : 0.f;
+    }
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int row_end = min(d, (int)(blockIdx.y + 1) * kRows);
+  for (int i = blockIdx.y * kRows + warp; i < row_end; i += nwarps) {
+    float acc[kCand];
+#pragma unroll
+    for (int c = 0; c < kCand; ++c) acc[c] = 0.f;
+    const float* brow = Bfactor + (size_t)i * d;
+    for (int j = lane; j < d; j += 32) {
+      const float b = __ldg(brow + j);
+#pragma unroll
+      for (int c = 0; c < kCand; ++c) acc[c] = fmaf(b, w_smem[c * d4 + j], acc[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < kCand; ++c) {
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+    }
+    if (lane == 0) {
+      const float mi = mean[i];
+#pragma unroll
+      for (int c = 0; c < kCand; ++c)
+        if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = fmaf(step, acc[c], mi);
+    }
+  }
+}
+
+__global__ void stream_words_kernel(uint2 key, int k_begin, int k_count, int n_blocks, uint32_t* __restrict__ out) {
+  const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (idx >= (long long)k_count * n_blocks) return;
+  const int kk = (int)(idx / n_blocks), j = (int)(idx % n_blocks);
+  const uint4 w = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)(k_begin + kk), 0u, 0u), key);
+  reinterpret_cast<uint4*>(out)[idx] = w;
+}
+
+__global__ void philox_once_kernel(uint4 ctr, uint2 key, uint32_t* out) {
+  const uint4 w = philox4x32_10(ctr, key);
+  out[0] = w.x; out[1] = w.y; out[2] = w.z; out[3] = w.w;
+}
+
+__global__ void segment_map_kernel(const int32_t* __restrict__ off, int P, int T, int32_t* __restrict__ cand) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < T) cand[t] = find_candidate(off, P, t);
+}
+
+inline uint2 key_of(uint64_t seed) { return make_uint2((uint32_t)(seed & 0xffffffffull), (uint32_t)(seed >> 32)); }
+
+}  // namespace
+
+int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
+                       uint64_t seed, int32_t k_begin, int32_t k_count, float* sigma_out, cudaStream_t stream) {
+  if (k_count == 0) return ESSA_OK;
+  const int nb = (d + 3) / 4;
+  if (Bfactor == nullptr) {
+    const long long total = (long long)k_count * nb;
+    const int threads = 256;
+    const long long blocks = (total + threads - 1) / threads;
+    if (blocks > 0x7fffffffLL) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: P*d too large");
+    sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count,
+                                                                 sigma_out);
+  } else {
+    if (d > 8192) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 8192 with a full covariance factor");
+    const size_t smem = (size_t)kCand * nb * 4 * sizeof(float);
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(sample_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(sample_full_kernel)");
+    }
+    dim3 grid((k_count + kCand - 1) / kCand, (d + kRows - 1) / kRows);
+    sample_full_kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin,
+                                                                k_count, sigma_out);
+  }
+  return check_cuda(ctx, cudaGetLastError(), "sampler launch");
+}
+
+int32_t launch_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count, int32_t n_blocks,
+                            uint32_t* words_out, cudaStream_t stream) {
+  const long long total = (long long)k_count * n_blocks;
+  if (total == 0) return ESSA_OK;
+  stream_words_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(key_of(seed), k_begin, k_count, n_blocks,
+                                                                           words_out);
+  return check_cuda(ctx, cudaGetLastError(), "stream_words launch");
+}
+
+int32_t launch_philox_once(essa_ctx* ctx, const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t* d_out = nullptr;
+  cudaError_t e = cudaMalloc(&d_out, 16);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMalloc");
+  philox_once_kernel<<<1, 1>>>(make_uint4(ctr[0], ctr[1], ctr[2], ctr[3]), make_uint2(key[0], key[1]), d_out);
+  e = cudaMemcpy(out, d_out, 16, cudaMemcpyDeviceToHost);
+  cudaFree(d_out);
+  return check_cuda(ctx, e, "philox_once");
+}
+
+int32_t launch_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P, int64_t T, int32_t* cand_out,
+                           cudaStream_t stream) {
+  if (T == 0) return ESSA_OK;
+  segment_map_kernel<<<(unsigned)((T + 255) / 256), 256, 0, stream>>>(seg_offsets, P, (int)T, cand_out);
+  return check_cuda(ctx, cudaGetLastError(), "segment_map launch");
+}
+
+}  // namespace essa

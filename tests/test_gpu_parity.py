@@ -1,0 +1,266 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Integer work (Philox words, segment map) must match bit for bit; sampled singular values within 1e-6;
+bf16 projection outputs within 2e-2 (4e-2 with INT8 weights) of max(|o|, rms(o)).
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import essa_oracle as orc
+from paper_2507_04453_b200 import workloads as wl
+from tests.parity_utils import TOL_BF16, TOL_INT8, TOL_SIGMA, Case, oracle_weight, sigma_error, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("CUDA device required for -m gpu tests")
+    return torch
+
+
+@pytest.fixture(scope="module")
+def ctx(torch):
+    from paper_2507_04453_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.get_status() == 0, "a kernel recorded a device-side error"
+    c.close()
+
+
+# ------------------------------------------------------------------ integer stream, segment map
+def test_device_philox_known_answers(ctx, philox_kat):
+    for ctr, key, want in philox_kat:
+        assert ctx.debug_philox(ctr, key) == want
+
+
+def test_stream_words_bit_exact(ctx):
+    for seed, k_begin, k_count, nb in [(0, 0, 4, 4), (3, 0, 256, 32), ((0xDEADBEEF << 32) | 0x1234567, 1000, 37, 129)]:
+        got = ctx.debug_stream_words(seed, k_begin, k_count, nb).cpu().numpy().view(np.uint32)
+        want = orc.candidate_stream_words(seed, np.arange(k_begin, k_begin + k_count), nb)
+        assert np.array_equal(got, want)
+
+
+def test_segment_map_bit_exact(torch, ctx):
+    rng = np.random.default_rng(11)
+    cases = [np.array([0, 16, 32, 48, 64]), np.arange(257), wl.make_segments(wl.CONFIGS["4"]),
+             wl.make_segments(wl.CONFIGS["5c"])]
+    for _ in range(5):
+        lens = rng.integers(0, 7, size=rng.integers(1, 300))
+        lens[rng.integers(0, len(lens))] += 1  # at least one token
+        cases.append(np.concatenate([[0], np.cumsum(lens)]))
+    for off in cases:
+        off = off.astype(np.int32)
+        T = int(off[-1])
+        got = ctx.debug_segment_map(to_dev(torch, off), T).cpu().numpy()
+        assert np.array_equal(got, orc.candidate_of_token(off, T))
+
+
+# ------------------------------------------------------------------ sampling
+@pytest.mark.parametrize("name", ["1", "2", "3", "4", "5a"])
+def test_sampled_sigma_matches_oracle(torch, ctx, name):
+    cfg = wl.CONFIGS[name]
+    adapters = [wl.make_adapter(_tiny_like(cfg), i) for i in range(len(cfg.projections))]
+    cma = wl.make_cma_state(_tiny_like(cfg), adapters)
+    want = orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, cfg.P)
+    got = ctx.sample_population(to_dev(torch, cma.mean), cma.step,
+                                None if cma.Bfactor is None else to_dev(torch, cma.Bfactor),
+                                None if cma.Dvec is None else to_dev(torch, cma.Dvec), cma.seed, cfg.P)
+    torch.cuda.synchronize()
+    assert got.shape == (cfg.P, cfg.d)
+    assert sigma_error(got.cpu().numpy(), want) <= TOL_SIGMA
+
+
+def _tiny_like(cfg):
+    """Same rank / P / CMA-ES structure, small matrices (the sampler does not depend on d_model)."""
+    if len(cfg.projections) == 1:
+        return cfg
+    return dataclasses.replace(cfg, projections=wl._qkvo(128, 64))
+
+
+def test_sampler_general_cases(torch, ctx):
+    rng = np.random.default_rng(12)
+    for d, P, full, step, seed in [(1, 1, False, 1.0, 1), (7, 5, True, 0.32, 2), (130, 33, True, 0.32, (9 << 32) + 5),
+                                   (512, 128, True, 0.32, 77), (1792, 64, False, 0.32, 4), (1030, 9, True, 2.0, 8)]:
+        mean = rng.standard_normal(d).astype(np.float32)
+        Dv = rng.uniform(0.5, 1.5, d).astype(np.float32)
+        Bf = (rng.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32) if full else None
+        want = orc.sample_population(mean, np.float32(step), Bf, Dv, seed, P)
+        got = ctx.sample_population(to_dev(torch, mean), step, None if Bf is None else to_dev(torch, Bf),
+                                    to_dev(torch, Dv), seed, P)
+        assert sigma_error(got.cpu().numpy(), want) <= TOL_SIGMA, (d, P, full)
+    # zero candidates is a no-op
+    out = ctx.sample_population(to_dev(torch, np.zeros(4, np.float32)), 1.0, None, None, 0, 0)
+    assert out.shape == (0, 4)
+
+
+def test_sampler_range_regenerates_any_member(torch, ctx):
+    rng = np.random.default_rng(13)
+    d, P = 128, 64
+    mean = to_dev(torch, rng.standard_normal(d).astype(np.float32))
+    Bf = to_dev(torch, np.linalg.qr(rng.standard_normal((d, d)))[0].astype(np.float32))
+    full = ctx.sample_population(mean, 0.05, Bf, None, 5, P).cpu().numpy()
+    part = ctx.sample_population(mean, 0.05, Bf, None, 5, 10, k_begin=37).cpu().numpy()
+    assert np.array_equal(part, full[37:47])  # bit-identical: a member depends on <seed, k> only
+
+
+# ------------------------------------------------------------------ adapter preparation
+def test_core_matrix(torch, ctx):
+    cfg = wl.CONFIGS["1"]
+    ad = wl.make_adapter(cfg, 0)
+    h = ctx.load_adapter(ad)
+    M = ctx.debug_core_matrix(h)
+    want = ad.V_B.astype(np.float64).T @ ad.U_A.astype(np.float64)
+    np.testing.assert_allclose(M, want, rtol=0, atol=2e-6)
+    h.free()
+
+
+# ------------------------------------------------------------------ projection, full outputs vs oracle
+def _check_projection(case, i, tol, paths=("tc", "simt"), candidates=None):
+    x = case.tokens(i)
+    want = case.oracle_projection(i, x, candidates)
+    errs = {}
+    for path in paths:
+        got = case.gpu_projection(i, x, path)
+        assert got.shape == want.shape
+        assert np.isfinite(got).all()
+        errs[path] = orc.relative_error(got, want)
+        assert errs[path] <= tol, (case.cfg.name, case.cfg.projections[i], path, errs[path])
+    return errs
+
+
+def test_config1_full(torch, ctx):
+    case = Case(torch, ctx, wl.CONFIGS["1"])
+    errs = _check_projection(case, 0, TOL_BF16)
+    assert errs["tc"] < 8e-3, errs  # expected ~4e-3: bf16 output rounding + bf16 rank-r intermediate
+    case.close()
+
+
+SCALED = {
+    # name: (base, d_model, d_kv, rank, P, seg_len)
+    "prefill-r16": ("2", 512, 128, 16, 8, 200),     # T = 1600: 12.5 token tiles, 2-4 channel tiles
+    "decode-r16": ("3", 1024, 192, 16, 256, 1),      # T = 256, split-K path, d_kv not a tile multiple
+    "ragged-r32": ("4", 640, 128, 32, 24, 300),      # ragged segments, d_out = 640 = 2.5 x 256
+    "int8-decode-r64": ("5a", 1024, 256, 64, 128, 1),
+    "int8-prefill-r64": ("5b", 768, 128, 64, 16, 100),
+    "int8-mixed-r64": ("5c", 512, 128, 64, 32, 90),
+}
+
+
+@pytest.mark.parametrize("name", list(SCALED))
+def test_scaled_configs_full_outputs(torch, ctx, name):
+    base, dm, dkv, r, P, L = SCALED[name]
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    for i in range(len(cfg.projections)):
+        _check_projection(case, i, tol)
+    case.close()
+
+
+@pytest.mark.parametrize("rank", [1, 3, 8, 17, 33, 48, 64])
+def test_rank_padding(torch, ctx, rank):
+    cfg = wl.scaled_config("1", d_model=256, d_kv=256, rank=rank, P=5, seg_len=37)
+    case = Case(torch, ctx, cfg)
+    _check_projection(case, 0, TOL_BF16)
+    case.close()
+
+
+def test_edge_cases(torch, ctx):
+    cfg = wl.scaled_config("1", d_model=192, d_kv=192, rank=8, P=6, seg_len=1)
+    case = Case(torch, ctx, cfg)
+    ad, h = case.adapters[0], case.handles[0]
+    sA, sB = cfg.sigma_cols(0)
+    W = oracle_weight(ad)
+
+    def run(offsets, T):
+        x = wl.make_tokens(cfg, 0, T)
+        d_off = to_dev(torch, np.asarray(offsets, dtype=np.int32))
+        want = orc.apply_projection(W, ad.U_A, ad.V_A, ad.U_B, ad.V_B, x, offsets, case.sigma32, sA, sB, ad.rank)
+        for fn in (ctx.apply_projection, ctx.apply_projection_simt):
+            got = fn(h, to_dev(torch, x, torch.bfloat16) if T else torch.empty((0, 192), dtype=torch.bfloat16, device="cuda"),
+                     d_off, case.d_sigma, sA, sB)
+            torch.cuda.synchronize()
+            assert got.shape == (T, 192)
+            if T:
+                assert orc.relative_error(got.float().cpu().numpy(), want) <= TOL_BF16
+
+    run([0, 0, 0, 0, 0, 0, 0], 0)            # empty input: legal no-op
+    run([0, 1, 1, 1, 1, 1, 1], 1)            # one token, trailing empty segments
+    run([0, 0, 0, 0, 0, 0, 129], 129)        # leading empty segments, one token past a tile
+    run([0, 127, 128, 129, 129, 300, 385], 385)  # boundaries around the 128-token tile edge, ragged tail
+    case.close()
+
+
+def test_zero_sigma_gives_base_projection_and_is_deterministic(torch, ctx):
+    cfg = wl.scaled_config("2", d_model=512, d_kv=128, rank=16, P=4, seg_len=160)
+    case = Case(torch, ctx, cfg)
+    x = case.tokens(0)
+    dx = to_dev(torch, x, torch.bfloat16)
+    sA, sB = cfg.sigma_cols(0)
+    zero = torch.zeros_like(case.d_sigma)
+    y0 = ctx.apply_projection(case.handles[0], dx, case.d_offsets, zero, sA, sB).float().cpu().numpy()
+    base = x.astype(np.float64) @ oracle_weight(case.adapters[0]).T
+    assert orc.relative_error(y0, base) <= 6e-3  # only the final bf16 rounding
+    # repeated calls are bit-identical (no data race, no dependence on stale TMEM / shared memory)
+    a = ctx.apply_projection(case.handles[0], dx, case.d_offsets, case.d_sigma, sA, sB).clone()
+    for _ in range(3):
+        b = ctx.apply_projection(case.handles[0], dx, case.d_offsets, case.d_sigma, sA, sB)
+        assert torch.equal(a, b)
+    case.close()
+
+
+def test_host_buffer_entry_point(torch, ctx):
+    cfg = wl.scaled_config("4", d_model=256, d_kv=64, rank=32, P=7, seg_len=50)
+    case = Case(torch, ctx, cfg)
+    x = case.tokens(1)
+    sA, sB = cfg.sigma_cols(1)
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    yh = torch.empty((case.T, 64), dtype=torch.bfloat16).pin_memory()
+    ctx.apply_projection_host(case.handles[1], xh, torch.from_numpy(case.offsets), torch.from_numpy(case.sigma32),
+                              sA, sB, yh)
+    want = case.oracle_projection(1, x)
+    assert orc.relative_error(yh.float().numpy(), want) <= TOL_BF16
+    # offsets that do not end at T are rejected on the host
+    from paper_2507_04453_b200.binding import EssaError
+    bad = torch.from_numpy(case.offsets.copy())
+    bad[-1] += 1
+    with pytest.raises(EssaError):
+        ctx.apply_projection_host(case.handles[1], xh, bad, torch.from_numpy(case.sigma32), sA, sB, yh)
+    case.close()
+
+
+def test_argument_validation(torch, ctx):
+    from paper_2507_04453_b200.binding import EssaError
+    cfg = wl.scaled_config("1", d_model=128, d_kv=128, rank=8, P=2, seg_len=4)
+    case = Case(torch, ctx, cfg)
+    x = to_dev(torch, case.tokens(0), torch.bfloat16)
+    with pytest.raises(EssaError):  # sigma columns outside the row
+        ctx.apply_projection(case.handles[0], x, case.d_offsets, case.d_sigma, 12, 8)
+    bad = dataclasses.replace(case.adapters[0], d_in=100)
+    with pytest.raises(EssaError):  # d_in not a multiple of 64
+        ctx.load_adapter(bad)
+    case.close()
+
+
+def test_sampler_to_projection_end_to_end(torch, ctx):
+    """Both chains run on their own: GPU sampler -> GPU projection vs oracle sampler -> oracle projection."""
+    cfg = wl.scaled_config("3", d_model=512, d_kv=128, rank=16, P=64, seg_len=1)
+    case = Case(torch, ctx, cfg)
+    cma = case.cma
+    d_sig = ctx.sample_population(to_dev(torch, cma.mean), cma.step, to_dev(torch, cma.Bfactor), to_dev(torch, cma.Dvec),
+                                  cma.seed, cfg.P)
+    want_sigma = orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, cfg.P)
+    for i in range(4):
+        x = case.tokens(i)
+        ad = case.adapters[i]
+        sA, sB = cfg.sigma_cols(i)
+        y = ctx.apply_projection(case.handles[i], to_dev(torch, x, torch.bfloat16), case.d_offsets, d_sig, sA, sB)
+        want = orc.apply_projection(oracle_weight(ad), ad.U_A, ad.V_A, ad.U_B, ad.V_B, x, case.offsets, want_sigma,
+                                    sA, sB, ad.rank)
+        assert orc.relative_error(y.float().cpu().numpy(), want) <= TOL_BF16
+    case.close()
