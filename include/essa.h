@@ -103,9 +103,10 @@ int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* adapter);
  * (j, k, 0, 0) yields four 32-bit words per block j; word w maps to u = (2*(w>>9)+1)*2^-24 and the
  * word pairs (0,1) and (2,3) give coordinates 4j..4j+3 by Box-Muller
  * (sqrt(-2 ln u0) * {cos, sin}(2 pi u1)).  A candidate therefore depends on <seed, k> only.
+ * The transform and the sum run in fp64 on the device; each entry is rounded to fp32 once.
  *   mean    [d] fp32 dev;  Bfactor [d][d] fp32 dev, row-major, or NULL for identity;
  *   Dvec    [d] fp32 dev or NULL for ones;  sigma_out [P][d] fp32 dev (written).
- * d >= 1; with a non-NULL Bfactor d <= 8192.  P = 0 is a legal no-op. */
+ * d >= 1; with a non-NULL Bfactor d <= 4096.  P = 0 is a legal no-op. */
 int32_t essa_sample_population(essa_ctx* ctx, const float* mean, float step, const float* Bfactor,
                                const float* Dvec, int32_t d, uint64_t seed, int32_t P, float* sigma_out,
                                void* stream);

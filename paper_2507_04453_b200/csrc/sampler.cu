@@ -21,24 +21,24 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
   return c;
 }
 
-// Word -> uniform strictly inside (0,1): (2*(w>>9)+1) * 2^-24; the integer is < 2^24, so the float is exact.
-__device__ __forceinline__ float uniform_open01(uint32_t w) { return static_cast<float>(2u * (w >> 9) + 1u) * 0x1p-24f; }
+// Word -> uniform strictly inside (0,1): (2*(w>>9)+1) * 2^-24 (exact).
+__device__ __forceinline__ double uniform_open01(uint32_t w) { return static_cast<double>(2u * (w >> 9) + 1u) * 0x1p-24; }
 
-__device__ __forceinline__ void box_muller(uint32_t w_radius, uint32_t w_angle, float& z0, float& z1) {
-  const float rho = sqrtf(-2.0f * logf(uniform_open01(w_radius)));
-  float s, c;
-  sincospif(2.0f * uniform_open01(w_angle), &s, &c);  // angle = 2*pi*u
+// The transform and the covariance product run in fp64 and the result is rounded to fp32 once, so the table
+// matches a double-precision evaluation to fp32 rounding for any step size (the work is tiny: P*d normals).
+__device__ __forceinline__ void box_muller(uint32_t w_radius, uint32_t w_angle, double& z0, double& z1) {
+  const double rho = sqrt(-2.0 * log(uniform_open01(w_radius)));
+  double s, c;
+  sincospi(2.0 * uniform_open01(w_angle), &s, &c);  // angle = 2*pi*u
   z0 = rho * c;
   z1 = rho * s;
 }
 
 // Four standard normals: coordinates 4j..4j+3 of candidate k.
-__device__ __forceinline__ float4 normals_block(uint2 key, uint32_t j, uint32_t k) {
+__device__ __forceinline__ void normals_block(uint2 key, uint32_t j, uint32_t k, double (&z)[4]) {
   const uint4 w = philox4x32_10(make_uint4(j, k, 0u, 0u), key);
-  float4 z;
-  box_muller(w.x, w.y, z.x, z.y);
-  box_muller(w.z, w.w, z.z, z.w);
-  return z;
+  box_muller(w.x, w.y, z[0], z[1]);
+  box_muller(w.z, w.w, z[2], z[3]);
 }
 
 // Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
@@ -48,14 +48,14 @@ __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, c
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (idx >= (long long)k_count * nb) return;
   const int kk = (int)(idx / nb), j = (int)(idx % nb);
-  const float4 z = normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk));
-  const float zz[4] = {z.x, z.y, z.z, z.w};
+  double zz[4];
+  normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk), zz);
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
     const int i = 4 * j + e;
     if (i < d) {
-      const float w = Dvec ? Dvec[i] * zz[e] : zz[e];
-      sigma_out[(size_t)kk * d + i] = fmaf(step, w, mean[i]);
+      const double w = Dvec ? (double)Dvec[i] * zz[e] : zz[e];
+      sigma_out[(size_t)kk * d + i] = (float)((double)mean[i] + (double)step * w);
     }
   }
 }
@@ -70,32 +70,31 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
                                                                       const float* __restrict__ Dvec, int d, uint2 key,
                                                                       int k_begin, int k_count,
                                                                       float* __restrict__ sigma_out) {
-  extern __shared__ float w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
+  extern __shared__ double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
   const int nb = (d + 3) >> 2, d4 = nb * 4;
   const int kk0 = blockIdx.x * kCand;
   for (int idx = threadIdx.x; idx < kCand * nb; idx += blockDim.x) {
     const int c = idx / nb, j = idx % nb;
-    float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (kk0 + c < k_count) z = normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk0 + c));
-    const float zz[4] = {z.x, z.y, z.z, z.w};
+    double zz[4] = {0.0, 0.0, 0.0, 0.0};
+    if (kk0 + c < k_count) normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk0 + c), zz);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int i = 4 * j + e;
-      w_smem[c * d4 + i] = (i < d) ? (Dvec ? Dvec[i] * zz[e] : zz[e]) : 0.f;
+      w_smem[c * d4 + i] = (i < d) ? (Dvec ? (double)Dvec[i] * zz[e] : zz[e]) : 0.0;
     }
   }
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   const int row_end = min(d, (int)(blockIdx.y + 1) * kRows);
   for (int i = blockIdx.y * kRows + warp; i < row_end; i += nwarps) {
-    float acc[kCand];
+    double acc[kCand];
 #pragma unroll
-    for (int c = 0; c < kCand; ++c) acc[c] = 0.f;
+    for (int c = 0; c < kCand; ++c) acc[c] = 0.0;
     const float* brow = Bfactor + (size_t)i * d;
     for (int j = lane; j < d; j += 32) {
-      const float b = __ldg(brow + j);
+      const double b = (double)__ldg(brow + j);
 #pragma unroll
-      for (int c = 0; c < kCand; ++c) acc[c] = fmaf(b, w_smem[c * d4 + j], acc[c]);
+      for (int c = 0; c < kCand; ++c) acc[c] = fma(b, w_smem[c * d4 + j], acc[c]);
     }
 #pragma unroll
     for (int c = 0; c < kCand; ++c) {
@@ -103,10 +102,10 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
       for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
     }
     if (lane == 0) {
-      const float mi = mean[i];
+      const double mi = (double)mean[i];
 #pragma unroll
       for (int c = 0; c < kCand; ++c)
-        if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = fmaf(step, acc[c], mi);
+        if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = (float)(mi + (double)step * acc[c]);
     }
   }
 }
@@ -145,8 +144,8 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count,
                                                                  sigma_out);
   } else {
-    if (d > 8192) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 8192 with a full covariance factor");
-    const size_t smem = (size_t)kCand * nb * 4 * sizeof(float);
+    if (d > 4096) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 4096 with a full covariance factor");
+    const size_t smem = (size_t)kCand * nb * 4 * sizeof(double);
     if (smem > 48 * 1024) {
       cudaError_t e = cudaFuncSetAttribute(sample_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(sample_full_kernel)");
