@@ -363,8 +363,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
+    if args.candidates > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, P=args.candidates, name=f"{cfg.name}-P{args.candidates}")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
