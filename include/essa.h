@@ -51,6 +51,7 @@ extern "C" {
 #define ESSA_W0_INT8_PERCHANNEL 1 /* W0[o][i] = q[o][i] * scale[o], q int8, scale fp16 per out-channel */
 
 #define ESSA_MAX_RANK 64
+#define ESSA_STATIC_MAX_TOKENS 4096 /* largest T essa_apply_projection_static accepts */
 
 typedef struct essa_ctx essa_ctx;         /* one per (process, device); not thread-safe */
 typedef struct essa_adapter essa_adapter; /* one per adapted projection matrix          */
@@ -139,6 +140,26 @@ int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* adapter, c
                                    const int32_t* seg_offsets_host, int32_t P, const float* sigma_host,
                                    int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y_host,
                                    void* stream);
+
+/* (No counterpart in the paper: an engineering variant of essa_apply_projection.)
+ * The same operation, same arguments and same result as essa_apply_projection, for callers that must not
+ * allocate device memory when they call: code running while another allocator owns the GPU's memory budget,
+ * or a latency-critical loop that cannot afford the implicit synchronisation of cudaMalloc / cudaFree.  This
+ * entry point calls no cudaMalloc, cudaFree or any other allocating routine: its only scratch (the rank-path
+ * vector u, 128 bytes per token) is a fixed array compiled into the library, ESSA_STATIC_MAX_TOKENS * 128 bytes
+ * = 512 KB, which every GPU that loads the library holds until the process exits.  Split-K is off on this path,
+ * so small token counts run on fewer SMs than essa_apply_projection would use.
+ *   - T > ESSA_STATIC_MAX_TOKENS is rejected with ESSA_ERR_UNSUPPORTED_SHAPE (and a message in
+ *     essa_last_error); use essa_apply_projection for larger batches.
+ *   - The context's device must be the current device, else ESSA_ERR_INVALID_ARG.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that first
+ *     call before any stream capture.
+ *   - All calls, from every context and stream on that GPU, share the one array and it keeps the last call's
+ *     contents.  Nothing in it needs clearing (each call overwrites every entry it later reads), but two calls
+ *     that overlap on the GPU race on it: keep calls to this entry point ordered (one stream, or events). */
+int32_t essa_apply_projection_static(essa_ctx* ctx, const essa_adapter* adapter, const void* x, int64_t T,
+                                     const int32_t* seg_offsets, int32_t P, const float* sigma,
+                                     int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y, void* stream);
 
 /* Straightforward CUDA-core (no tensor core, fp32 rank path) evaluation of the same formula, same
  * arguments as essa_apply_projection.  A cross-check for the tensor-core path at sizes the CPU

@@ -32,6 +32,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
+    "essa_apply_projection_static",
 )
 
 
@@ -87,6 +88,7 @@ def load_library() -> C.CDLL:
         "essa_apply_projection": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_apply_projection_host": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_apply_projection_simt": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
+        "essa_apply_projection_static": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_plan_projection": (i32, [i32, i32, i32, i32, i64, i32, C.POINTER(Plan)]),
         "essa_validate_segments": (i32, [vp, i32, i64]),
         "essa_debug_stream_words": (i32, [vp, u64, i32, i32, i32, vp, vp]),
@@ -237,6 +239,20 @@ class Context:
     def apply_projection(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out=None, stream=None):
         """essa_apply_projection: y[T, d_out] bf16 (two kernel launches: rank-down, base + up)."""
         y = self._proj(self.lib.essa_apply_projection, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
+        self.gpu_launches += 2 if x.shape[0] else 0
+        return y
+
+    def apply_projection_static(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out, stream=None):
+        """essa_apply_projection_static: same result as apply_projection without any device allocation.
+
+        For callers that cannot allocate when they call (another allocator owns the GPU memory, or no implicit
+        synchronisation is tolerable): the library's fixed 512 KB array is the only scratch, so T is limited to
+        ESSA_STATIC_MAX_TOKENS (4096) and `out` must be supplied by the caller (this wrapper allocates nothing).
+        Calls share that array: keep them ordered on the GPU.
+        """
+        if out is None:
+            raise ValueError("apply_projection_static needs a caller-provided output tensor")
+        y = self._proj(self.lib.essa_apply_projection_static, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
         self.gpu_launches += 2 if x.shape[0] else 0
         return y
 

@@ -323,6 +323,16 @@ int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* 
   return launch_projection_tc(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 
+// Allocation-free variant: see the comment above g_static_u in proj_tc.cu.
+int32_t essa_apply_projection_static(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,
+                                     int32_t P, const float* sigma, int32_t ld_sigma, int32_t sA_col, int32_t sB_col,
+                                     void* y, void* stream) {
+  const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
+  if (st != ESSA_OK || T == 0) return st;
+  ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  return launch_projection_tc_static(ctx, a, g, static_cast<cudaStream_t>(stream));
+}
+
 int32_t essa_apply_projection_simt(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,
                                    int32_t P, const float* sigma, int32_t ld_sigma, int32_t sA_col, int32_t sB_col,
                                    void* y, void* stream) {

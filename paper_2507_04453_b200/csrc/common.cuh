@@ -95,6 +95,7 @@ struct ProjArgs {
 // proj_simt.cu / proj_tc.cu
 int32_t launch_projection_simt(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
 int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
+int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
 void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
                      essa_plan* out);
 

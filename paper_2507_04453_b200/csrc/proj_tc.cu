@@ -695,4 +695,109 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   return st;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant (essa_apply_projection_static).
+//
+// Some callers may not allocate device memory at the moment they need a projection: code that runs inside a
+// memory-pool-managed region where every cudaMalloc would fragment or synchronise the pool, a latency-critical
+// serving loop that must never hit an implicit device synchronisation, or a process that has handed the whole
+// GPU memory budget to another allocator.  For them the rank-path vector u (the only scratch the two launches
+// need when split-K is off) lives in this file-scope device array instead of context-owned cudaMalloc memory.
+// Every GPU that loads the library holds these kStaticMaxTokens * 128 bytes (512 KB) until the process exits.
+//
+// In host code the name g_static_u is only a host-side stand-in for the symbol: passing it to a kernel would
+// hand the device a host address.  The device address is obtained once per device with cudaGetSymbolAddress,
+// with that device current, and it is that pointer the kernels (and the TMA tensor map) receive.
+constexpr int kStaticMaxTokens = ESSA_STATIC_MAX_TOKENS;
+static __device__ __align__(256) unsigned char g_static_u[(size_t)kStaticMaxTokens * kRankPadMax * 2];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_u_addr[kMaxDevices] = {};  // device address of g_static_u, per device, set on first use
+
+int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, cudaStream_t stream) {
+  if (g.T == 0) return ESSA_OK;
+  if (g.T > kStaticMaxTokens)
+    return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE,
+                "apply_projection_static: T exceeds ESSA_STATIC_MAX_TOKENS (the fixed scratch holds 4096 tokens); "
+                "use essa_apply_projection");
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != ctx->device || cur < 0 || cur >= kMaxDevices)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_static: the context's device must be the current device");
+  if (g_static_u_addr[cur] == nullptr) {
+    // One-time set-up on this device (not capturable: do the first call before any stream capture).
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_u);
+    if (e != cudaSuccess || p == nullptr) return check_cuda(ctx, e == cudaSuccess ? cudaErrorInvalidSymbol : e, "cudaGetSymbolAddress(g_static_u)");
+    g_static_u_addr[cur] = p;
+  }
+  __nv_bfloat16* u = static_cast<__nv_bfloat16*>(g_static_u_addr[cur]);
+
+  // Same two launches as essa_apply_projection, with split-K off so that u is the only scratch.  Nothing in u has
+  // to start at zero: the rank-down launch writes all 64 columns of every row < T and rows >= T are never read
+  // (the tensor map over u has exactly T rows), so the previous call's contents are simply overwritten.
+  essa_plan pl;
+  plan_projection(a->d_in, a->d_out, a->rank, a->w0_dtype, g.T, ctx->sm_count, &pl);
+  const int m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
+  const int n_tiles = (a->d_out + pl.block_n - 1) / pl.block_n;
+  const int sm = ctx->sm_count > 0 ? ctx->sm_count : 148;
+
+  CUtensorMap tm_x, tm_u;
+  int32_t st = make_tensor_map_2d(ctx, &tm_x, 0, g.x, (uint64_t)g.T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2, BLOCK_M, BLOCK_K, 128);
+  if (st != ESSA_OK) return st;
+  st = make_tensor_map_2d(ctx, &tm_u, 0, u, (uint64_t)g.T, kRankPadMax, kRankPadMax * 2, BLOCK_M, BLOCK_K, 128);
+  if (st != ESSA_OK) return st;
+
+  KParams kp{};
+  kp.T = (int)g.T;
+  kp.n_out = a->r_pad;
+  kp.main_kb = a->d_in / BLOCK_K;
+  kp.m_tiles = m_tiles;
+  kp.n_tiles = 1;
+  kp.splits = 1;
+  kp.seg = g.seg_offsets;
+  kp.P = g.P;
+  kp.sigma = g.sigma;
+  kp.ld_sigma = g.ld_sigma;
+  kp.sA_col = g.sA_col;
+  kp.sB_col = g.sB_col;
+  kp.r = a->rank;
+  kp.M = a->M;
+  kp.u = u;
+  kp.status = ctx->d_status;
+  const int down_grid = m_tiles < sm ? m_tiles : sm;
+  switch (a->r_pad) {
+    case 16: st = launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream); break;
+    case 32: st = launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream); break;
+    case 48: st = launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream); break;
+    case 64: st = launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream); break;
+    default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection_static: bad padded rank");
+  }
+  if (st != ESSA_OK) return st;
+
+  KParams mp{};
+  mp.T = (int)g.T;
+  mp.n_out = a->d_out;
+  mp.main_kb = a->d_in / BLOCK_K;
+  mp.ext_kb = a->ext_blocks;
+  mp.ext_ksteps = a->r_pad / UMMA_K;
+  mp.m_tiles = m_tiles;
+  mp.n_tiles = n_tiles;
+  mp.splits = 1;
+  mp.y = g.y;
+  mp.ldy = a->d_out;
+  mp.scale = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? a->w0_scale : nullptr;
+  mp.status = ctx->d_status;
+  const long long tiles = (long long)m_tiles * n_tiles;
+  const int grid = (int)(tiles < sm ? tiles : sm);
+  const int bi = pl.block_n == 64 ? 0 : pl.block_n == 128 ? 1 : 2;
+  const CUtensorMap& tmW = a->tm_W0[bi];
+  const CUtensorMap& tmU0 = a->tm_UBp[bi][0];
+  const CUtensorMap& tmU1 = a->tm_UBp[bi][a->ext_blocks > 1 ? 1 : 0];
+  switch (pl.block_n) {
+    case 64: return launch_one<64, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, grid, stream);
+    case 128: return launch_one<128, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, grid, stream);
+    default: return launch_one<256, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, grid, stream);
+  }
+}
+
 }  // namespace essa
