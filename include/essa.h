@@ -71,6 +71,8 @@ const char* essa_last_error(essa_ctx* ctx);
 /* Synchronise the device, then read (and clear) the device status word: 0, or the ESSA_ERR_* code a
  * kernel recorded (ESSA_ERR_DEVICE_TIMEOUT if a bounded wait ran out; the affected output is undefined). */
 int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
+/* Number of kernels of this library enqueued through ctx since it was created (host counter). */
+int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);
 /* Pre-size the context's scratch memory (rank-path buffer, split-K workspace, host-call staging) for
  * up to max_tokens tokens and max_d_out output channels so that later calls do not allocate. */
 int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out);
@@ -181,6 +183,10 @@ typedef struct essa_plan {
   int32_t down_splits;   /* split-K factor of the rank-path down-projection kernel   */
   int32_t down_grid;     /* CTAs launched by the down-projection kernel              */
   int64_t scratch_bytes; /* device scratch the call needs                            */
+  int32_t decode;        /* 1: decode schedule (one launch; block_m = W0 rows per CTA, block_n = tokens
+                            per tile, stages = depth of the W0 ring, splits = CTAs of a cluster sharing
+                            the reduction over d_in); 0: prefill */
+  int32_t x_stages;      /* decode schedule: depth of the activation ring; 0 otherwise */
 } essa_plan;
 int32_t essa_plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T,
                              int32_t sm_count, essa_plan* out);

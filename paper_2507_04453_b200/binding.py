@@ -32,7 +32,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
-    "essa_apply_projection_static",
+    "essa_apply_projection_static", "essa_get_launch_count",
 )
 
 
@@ -51,7 +51,8 @@ class AdapterDesc(C.Structure):
 class Plan(C.Structure):
     _fields_ = [("block_m", C.c_int32), ("block_n", C.c_int32), ("block_k", C.c_int32), ("stages", C.c_int32),
                 ("k_blocks", C.c_int32), ("splits", C.c_int32), ("tiles", C.c_int32), ("grid", C.c_int32),
-                ("down_splits", C.c_int32), ("down_grid", C.c_int32), ("scratch_bytes", C.c_int64)]
+                ("down_splits", C.c_int32), ("down_grid", C.c_int32), ("scratch_bytes", C.c_int64),
+                ("decode", C.c_int32), ("x_stages", C.c_int32)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -81,6 +82,7 @@ def load_library() -> C.CDLL:
         "essa_last_error": (C.c_char_p, [vp]),
         "essa_get_status": (i32, [vp, C.POINTER(i32)]),
         "essa_reserve": (i32, [vp, i64, i32, i32]),
+        "essa_get_launch_count": (i32, [vp, C.POINTER(i64)]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -157,7 +159,6 @@ class Context:
         if st != ESSA_OK:
             raise EssaError(st, self.lib.essa_status_string(st).decode())
         self.handle = h.value
-        self.gpu_launches = 0  # kernels of this library enqueued through this context
 
     # -- plumbing
     def _check(self, st: int):
@@ -168,6 +169,13 @@ class Context:
         if self.handle:
             self.lib.essa_destroy(self.handle)
             self.handle = None
+
+    @property
+    def gpu_launches(self) -> int:
+        """essa_get_launch_count: kernels of this library enqueued through this context so far."""
+        v = C.c_int64(0)
+        self._check(self.lib.essa_get_launch_count(self.handle, C.byref(v)))
+        return v.value
 
     def get_status(self) -> int:
         v = C.c_int32(0)
@@ -220,7 +228,6 @@ class Context:
             st = self.lib.essa_sample_population_range(self.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec),
                                                        d, seed, k_begin, P, out.data_ptr(), _stream(stream))
         self._check(st)
-        self.gpu_launches += 1 if P > 0 else 0
         return out
 
     # -- projection
@@ -237,9 +244,8 @@ class Context:
         return out
 
     def apply_projection(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out=None, stream=None):
-        """essa_apply_projection: y[T, d_out] bf16 (two kernel launches: rank-down, base + up)."""
+        """essa_apply_projection: y[T, d_out] bf16 (one launch at decode sizes, else rank-down then base + up)."""
         y = self._proj(self.lib.essa_apply_projection, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
-        self.gpu_launches += 2 if x.shape[0] else 0
         return y
 
     def apply_projection_static(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out, stream=None):
@@ -253,13 +259,11 @@ class Context:
         if out is None:
             raise ValueError("apply_projection_static needs a caller-provided output tensor")
         y = self._proj(self.lib.essa_apply_projection_static, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
-        self.gpu_launches += 2 if x.shape[0] else 0
         return y
 
     def apply_projection_simt(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out=None, stream=None):
         """essa_apply_projection_simt: CUDA-core cross-check of the same formula."""
         y = self._proj(self.lib.essa_apply_projection_simt, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
-        self.gpu_launches += 2 if x.shape[0] else 0
         return y
 
     def apply_projection_host(self, adapter, x_host, seg_offsets_host, sigma_host, sA_col: int, sB_col: int, y_host,
@@ -271,7 +275,6 @@ class Context:
                                                  seg_offsets_host.data_ptr(), P, sigma_host.data_ptr(),
                                                  sigma_host.stride(0), sA_col, sB_col, y_host.data_ptr(), _stream(stream))
         self._check(st)
-        self.gpu_launches += 2 if T else 0
         return y_host
 
     def profile_begin(self, max_calls: int):

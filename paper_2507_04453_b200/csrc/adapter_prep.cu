@@ -62,6 +62,7 @@ __global__ void widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* _
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream) {
   const size_t threads = (count + 3) / 4;
   widen_int8_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(q, out, count);
+  ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "widen_int8 launch");
 }
 
@@ -71,6 +72,7 @@ int32_t launch_adapter_prep(essa_ctx* ctx, essa_adapter* a, const __nv_bfloat16*
   const int tot = a->d_out * kRankPadMax;
   build_ubp_kernel<<<(tot + 255) / 256, 256, 0, stream>>>(a->U_B, a->w0_scale, a->d_out, a->rank, a->ext_blocks, a->UBp);
   build_core_kernel<<<(kRankPadMax * kRankPadMax + 255) / 256, 256, 0, stream>>>(U_A, V_B, a->rank, a->M);
+  ctx->launches += 3;
   return check_cuda(ctx, cudaGetLastError(), "adapter prep launch");
 }
 

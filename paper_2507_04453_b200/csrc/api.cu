@@ -186,6 +186,12 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
   return ESSA_OK;
 }
 
+int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches) {
+  if (!ctx || !launches) return ESSA_ERR_INVALID_ARG;
+  *launches = ctx->launches;
+  return ESSA_OK;
+}
+
 int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out) {
   if (!ctx || max_tokens < 0 || max_d_in < 0 || max_d_out < 0) return ESSA_ERR_INVALID_ARG;
   int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)max_tokens * kRankPadMax * 2, false, nullptr);

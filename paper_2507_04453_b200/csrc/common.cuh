@@ -14,7 +14,8 @@
 
 namespace essa {
 
-constexpr int kRankPadMax = 64;  // rank-path operands are stored 64 columns wide (one 128-byte swizzle row)
+constexpr int kRankPadMax = 64;
+constexpr int kDecodeMaxTokens = 256;  // calls with at most this many tokens use the decode schedule (proj_decode.cu)  // rank-path operands are stored 64 columns wide (one 128-byte swizzle row)
 
 // Device status word values are the ESSA_ERR_* codes; 0 = nothing recorded.
 struct Scratch {
@@ -29,6 +30,7 @@ struct essa_ctx {
   int sm_count = 0;
   std::string last_error;
   int32_t* d_status = nullptr;  // device status word
+  int64_t launches = 0;         // kernels of this library enqueued through this context
   // Scratch owned by the context (grown on demand, never shrunk).
   essa::Scratch u_buf;        // [T_cap][64] bf16: rank-path vector u_t, zero-padded to 64 columns
   essa::Scratch splitk_ws;    // fp32 partial tiles for split-K (kept all-zero between calls)
@@ -98,6 +100,10 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
 int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
 void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
                      essa_plan* out);
+// proj_decode.cu
+bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out);
+int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, const essa_plan& plan,
+                                 cudaStream_t stream);
 
 #ifdef __CUDACC__
 // Largest k in [0, P-1] with off[k] <= t (candidate that owns token t; empty segments own nothing).

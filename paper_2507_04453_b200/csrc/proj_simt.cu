@@ -132,6 +132,7 @@ int32_t launch_projection_simt(essa_ctx* ctx, const essa_adapter* a, const ProjA
   else
     simt_gemm_kernel<false><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0, nullptr, a->U_B,
                                                       u, g.y);
+  ctx->launches += 2;
   return check_cuda(ctx, cudaGetLastError(), "simt projection launch");
 }
 

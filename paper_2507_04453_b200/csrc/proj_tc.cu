@@ -19,6 +19,7 @@
 // of one tile overlap the main loop of the next.  Every mbarrier wait is bounded: on expiry the CTA records
 // ESSA_ERR_DEVICE_TIMEOUT in the status word, drains its outstanding copies, frees its TMEM and exits.
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace essa {
 namespace {
@@ -28,7 +29,6 @@ constexpr int BLOCK_K = 64;   // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr long long kWaitLimitCycles = 3000000000LL;  // ~1.5-2 s at B200 clocks
 constexpr int kSmemBudget = 227 * 1024;
 
 enum { EPI_STORE = 0, EPI_RANK = 1 };
@@ -56,126 +56,6 @@ struct KParams {
   int* cnt;
   int32_t* status;
 };
-
-// ------------------------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the CTA is aborting (this or another thread ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      atomicCAS(status, 0, ESSA_ERR_DEVICE_TIMEOUT);
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c_inner, int c_outer, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(c_inner), "r"(c_outer), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
-  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// mbarrier arrives once all MMAs issued so far by this thread have completed (implies fence::before_thread_sync).
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// 16 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  tmem_ld_wait();
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ float4 ld_cg_v4(const float* addr) {
-  float4 v;
-  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(addr) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_cg_zero_v4(float* addr) {
-  asm volatile("st.global.cg.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(addr), "f"(0.f) : "memory");
-}
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte swizzle (what TMA wrote):
-// start address >> 4 | stride between 8-row groups (1024 B) >> 4 at bit 32 | descriptor version 1 at bit 46 |
-// layout type 2 (128-byte swizzle) at bit 61.  The leading-dimension offset is unused for this layout.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor, kind::f16: D = fp32 (bits 4-5 = 1), A = B = bf16 (bits 7-9 = 1, 10-12 = 1), both K-major,
-// N >> 3 at bits 17-22, M >> 4 at bits 24-28.
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
 
 template <int BLOCK_N, int EPI>
 struct Cfg {
@@ -523,6 +403,7 @@ int32_t launch_one(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
     attr_done = true;
   }
   essa_tc_kernel<BLOCK_N, EPI><<<grid, kThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, tmA2, tmB2a, tmB2b, p);
+  ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "essa_tc_kernel launch");
 }
 
@@ -548,8 +429,10 @@ double schedule_cost(int tiles, int bn, int total_kb, int splits, int sm) {
 
 }  // namespace
 
-void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
-                     essa_plan* out) {
+// Schedule of the two prefill launches (rank-down, base + up).
+static void plan_prefill(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
+                         essa_plan* out) {
+  *out = essa_plan{};
   const int sm = sm_count > 0 ? sm_count : 148;
   const int m_tiles = (int)((T + BLOCK_M - 1) / BLOCK_M);
   const int main_kb = d_in / BLOCK_K;
@@ -598,11 +481,29 @@ void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype
   out->scratch_bytes = scratch;
 }
 
+void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
+                     essa_plan* out) {
+  *out = essa_plan{};
+  if (plan_decode(d_in, d_out, rank, w0_dtype, T, sm_count, out)) return;
+  plan_prefill(d_in, d_out, rank, w0_dtype, T, sm_count, out);
+}
+
 int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, cudaStream_t stream) {
   if (g.T == 0) return ESSA_OK;
   if (g.T > 0x7fffffffLL - BLOCK_M) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: T too large");
   essa_plan pl;
   plan_projection(a->d_in, a->d_out, a->rank, a->w0_dtype, g.T, ctx->sm_count, &pl);
+  if (pl.decode) {
+    cudaEvent_t* dev = nullptr;
+    if (ctx->prof_on) {
+      if ((size_t)(ctx->prof_calls + 1) * 3 <= ctx->prof_events.size()) dev = &ctx->prof_events[(size_t)ctx->prof_calls++ * 3];
+      else ++ctx->prof_dropped;
+    }
+    if (dev) { cudaEventRecord(dev[0], stream); cudaEventRecord(dev[1], stream); }
+    const int32_t dst = launch_projection_decode(ctx, a, g, pl, stream);
+    if (dev) cudaEventRecord(dev[2], stream);
+    return dst;
+  }
   const int m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
 
   int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)g.T * kRankPadMax * 2, false, stream);
@@ -736,7 +637,7 @@ int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const 
   // to start at zero: the rank-down launch writes all 64 columns of every row < T and rows >= T are never read
   // (the tensor map over u has exactly T rows), so the previous call's contents are simply overwritten.
   essa_plan pl;
-  plan_projection(a->d_in, a->d_out, a->rank, a->w0_dtype, g.T, ctx->sm_count, &pl);
+  plan_prefill(a->d_in, a->d_out, a->rank, a->w0_dtype, g.T, ctx->sm_count, &pl);
   const int m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
   const int n_tiles = (a->d_out + pl.block_n - 1) / pl.block_n;
   const int sm = ctx->sm_count > 0 ? ctx->sm_count : 148;

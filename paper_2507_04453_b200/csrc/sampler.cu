@@ -154,6 +154,7 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     sample_full_kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin,
                                                                 k_count, sigma_out);
   }
+  ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "sampler launch");
 }
 
@@ -163,6 +164,7 @@ int32_t launch_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32
   if (total == 0) return ESSA_OK;
   stream_words_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(key_of(seed), k_begin, k_count, n_blocks,
                                                                            words_out);
+  ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "stream_words launch");
 }
 
@@ -171,6 +173,7 @@ int32_t launch_philox_once(essa_ctx* ctx, const uint32_t ctr[4], const uint32_t 
   cudaError_t e = cudaMalloc(&d_out, 16);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMalloc");
   philox_once_kernel<<<1, 1>>>(make_uint4(ctr[0], ctr[1], ctr[2], ctr[3]), make_uint2(key[0], key[1]), d_out);
+  ctx->launches += 1;
   e = cudaMemcpy(out, d_out, 16, cudaMemcpyDeviceToHost);
   cudaFree(d_out);
   return check_cuda(ctx, e, "philox_once");
@@ -180,6 +183,7 @@ int32_t launch_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P,
                            cudaStream_t stream) {
   if (T == 0) return ESSA_OK;
   segment_map_kernel<<<(unsigned)((T + 255) / 256), 256, 0, stream>>>(seg_offsets, P, (int)T, cand_out);
+  ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "segment_map launch");
 }
 

@@ -68,11 +68,27 @@ def test_plan_is_consistent(lib, name):
     dtype = binding.ESSA_W0_INT8_PERCHANNEL if cfg.w0_dtype == "int8" else binding.ESSA_W0_BF16
     for _, n, m in cfg.projections:
         p = binding.plan_projection(n, m, cfg.rank, dtype, T, 148)
+        ext = 2 if dtype else 1
+        assert p["k_blocks"] == n // 64 + ext
+        if T <= 256:
+            # decode schedule: 128 W0 rows per CTA, all tokens in one tile, reduction split over a cluster
+            r_pad = -(-cfg.rank // 16) * 16
+            assert p["decode"] == 1 and p["block_m"] == 128 and p["block_k"] == 64
+            assert p["block_n"] == -(-T // 16) * 16 and p["tiles"] == -(-m // 128)
+            assert p["splits"] in (1, 2, 4, 8) and p["splits"] <= n // 64 and p["grid"] <= 148
+            assert p["grid"] == p["tiles"] * p["splits"] and p["scratch_bytes"] == 0
+            xrows = 128 if p["block_n"] <= 128 else 256
+            x_stage = xrows * 128 + r_pad * 128
+            rings = p["stages"] * 128 * 128 + p["x_stages"] * x_stage
+            assert 1 <= p["stages"] <= 10 and 1 <= p["x_stages"] <= 4
+            assert 1024 + rings + r_pad * r_pad * 4 + 1024 <= 227 * 1024
+            per = -(-(-(-p["block_n"] // p["splits"])) // 16) * 16
+            assert rings >= p["splits"] * 128 * (per + 4) * 4  # the receive buffer overlays the rings
+            continue
+        assert p["decode"] == 0
         assert p["block_m"] == 128 and p["block_k"] == 64 and p["block_n"] in (64, 128, 256)
         m_tiles = -(-T // 128)
         assert p["tiles"] == m_tiles * -(-m // p["block_n"])
-        ext = 2 if dtype else 1
-        assert p["k_blocks"] == n // 64 + ext
         assert 1 <= p["splits"] <= p["k_blocks"]
         assert 1 <= p["grid"] <= 148 and p["grid"] <= p["tiles"] * p["splits"]
         assert 1 <= p["down_splits"] <= n // 64 and 1 <= p["down_grid"] <= 148
