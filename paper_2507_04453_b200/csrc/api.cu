@@ -142,7 +142,18 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
     ctx->encode_tiled = fn;
   else
     cudaGetLastError();
-  if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess) {
+  if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_u, (size_t)kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMemset(ctx->dec_u, 0, (size_t)kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_cnt, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_ppart, (size_t)8 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_grp, (size_t)kDecodeMaxTokens) != cudaSuccess ||
+      cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens) != cudaSuccess) {
+    if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
+    if (ctx->dec_grp) cudaFree(ctx->dec_grp);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->dec_u) cudaFree(ctx->dec_u);
+    if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
     cudaGetLastError();
     delete ctx;
     return ESSA_ERR_ALLOC;
@@ -165,6 +176,10 @@ int32_t essa_destroy(essa_ctx* ctx) {
   free_scratch(ctx->stage_sigma);
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->dec_u) cudaFree(ctx->dec_u);
+  if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
+  if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
+  if (ctx->dec_grp) cudaFree(ctx->dec_grp);
   delete ctx;
   return ESSA_OK;
 }
@@ -182,6 +197,9 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     cudaMemset(ctx->d_status, 0, sizeof(int32_t));
     if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
     if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
+    cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t));
+    cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens);
+    ctx->dec_epoch = 0;
   }
   return ESSA_OK;
 }
@@ -228,6 +246,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   a->d_in = d->d_in; a->d_out = d->d_out; a->rank = d->rank; a->w0_dtype = d->w0_dtype;
   a->r_pad = ((d->rank + 15) / 16) * 16;
   a->ext_blocks = int8 ? 2 : 1;
+  a->vap_cols = a->r_pad <= 16 ? 16 : a->r_pad <= 32 ? 32 : 64;
   const size_t n = d->d_in, m = d->d_out, r = d->rank;
   // The INT8 weights are widened once to bf16 (exact: |q| <= 127) for the tensor-core operand; the fp16
   // per-channel scale is applied to the fp32 accumulator, so the dequantisation is exact.
@@ -241,6 +260,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   alloc((void**)&a->UBp, (size_t)a->ext_blocks * m * kRankPadMax * 2);
   alloc((void**)&a->U_B, m * r * 2);
   alloc((void**)&a->V_A, n * r * 2);
+  alloc((void**)&a->VAp, n * (size_t)a->vap_cols * 2);
   alloc((void**)&a->M, (size_t)kRankPadMax * kRankPadMax * 4);
   alloc((void**)&dUA, r * r * 2);
   alloc((void**)&dVB, r * r * 2);
@@ -287,7 +307,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
 int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* a) {
   if (!ctx || !a) return ESSA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->M};
+  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->VAp, a->M};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   delete a;

@@ -31,6 +31,13 @@ struct essa_ctx {
   std::string last_error;
   int32_t* d_status = nullptr;  // device status word
   int64_t launches = 0;         // kernels of this library enqueued through this context
+  // decode schedule: rank-path vector u of one call, [kDecodeMaxTokens][64] bf16, and the count of rows
+  // published so far (monotonic across calls; dec_epoch is the host's copy of where the next call starts)
+  void* dec_u = nullptr;
+  uint32_t* dec_cnt = nullptr;
+  uint32_t dec_epoch = 0;
+  void* dec_ppart = nullptr;    // [8][kDecodeMaxTokens][64] fp32: per-K-slice partial down-projections
+  int* dec_grp = nullptr;       // [kDecodeMaxTokens / 4] arrival counters of the token groups (kept at zero)
   // Scratch owned by the context (grown on demand, never shrunk).
   essa::Scratch u_buf;        // [T_cap][64] bf16: rank-path vector u_t, zero-padded to 64 columns
   essa::Scratch splitk_ws;    // fp32 partial tiles for split-K (kept all-zero between calls)
@@ -53,6 +60,8 @@ struct essa_adapter {
   __nv_bfloat16* UBp = nullptr;  // [ext][d_out][64]: U_B zero-padded to 64 columns; INT8: (U_B/scale) split hi, lo
   __nv_bfloat16* U_B = nullptr;  // [d_out][rank] as given (CUDA-core path)
   __nv_bfloat16* V_A = nullptr;  // [d_in][rank] as given (CUDA-core path)
+  __nv_bfloat16* VAp = nullptr;  // [d_in][vap_cols]: V_A zero-padded to 16 / 32 / 64 columns (16-byte row chunks)
+  int vap_cols = 0;
   float* M = nullptr;            // [64][64] fp32: M = V_B^T U_A zero-padded
   int ext_blocks = 1;            // rank-path K-slabs appended to the base contraction (1 bf16, 2 INT8)
   CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256

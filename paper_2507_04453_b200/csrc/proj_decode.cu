@@ -5,25 +5,29 @@
 // once, so the roles of the operands are swapped with respect to the prefill kernel: 128 rows of W0 (output
 // channels) are the UMMA M side, all tokens are the N side, and the reduction over d_in is split over the
 // CTAs of a thread-block cluster so that every SM streams a disjoint slice of W0.  One launch does the
-// whole call; there is no global scratch:
+// whole call:
 //
-//   K loop (TMA -> shared -> tcgen05.mma -> TMEM), per 64-wide K block of this CTA's slice:
-//       D_main[128 ch][tokens] += W0_tile . x_tile^T            (base contraction)
-//       D_p[tokens][r_pad]     += x_tile  . V_A_tile            (partial down-projection, same x tile)
-//     W0 tiles come from HBM and need a deep ring (HBM latency x bandwidth), x / V_A tiles are L2 hits and get
-//     a shallow ring of their own, so that most of shared memory holds W0 bytes in flight.
-//   rank core, one token per thread:  u = sB_k .* (M (sA_k .* p))  -> bf16 -> shared, in the swizzled
-//       K-major operand layout.  The map p -> u is linear, so applying it to this CTA's partial p and
-//       summing over the cluster gives the same rank term as applying it to the full p.
-//   up-projection:  D_main += U_B_tile . u^T  (one more UMMA K slab; two for INT8 storage)
+//   base contraction (TMA -> shared -> tcgen05.mma -> TMEM), per 64-wide K block of this CTA's slice:
+//       D[128 ch][tokens] += W0_tile . x_tile^T
+//     A tcgen05.mma of 128 rows costs about the same whatever its width, and a TMA load takes ~2500 cycles even
+//     when it hits L2, so the loop issues only the four wide MMAs per K block and keeps all of shared memory
+//     full of loads in flight (a ring of W0 tiles from HBM, a ring of x tiles from L2).
+//   rank path, on the CUDA cores of the four epilogue warps, which would otherwise idle during the loop:
+//     the first CTAs of the grid each take a few tokens,  p = V_A^T x_t  (16-byte loads, warp-shuffle and
+//     shared-memory reductions),  u = sB_k .* (M (sA_k .* p))  in registers, and publish u_t (bf16) to a small
+//     global buffer followed by a release-increment of a counter.  fp32 throughout.
+//   up-projection: the CTAs of K split 0 wait (bounded) until the counter shows all T rows, TMA-load u as one
+//     more K slab and add  U_B_tile . u^T  (two slabs for INT8 storage) to their accumulator.
 //   cluster reduction: after a cluster barrier (all MMAs of the cluster done, operand buffers dead) every
-//       CTA pushes the s-th slice of tokens of its fp32 partial tile into CTA s's shared memory (distributed
-//       shared memory stores); after a second barrier CTA s sums the slots in fixed rank order (results are
-//       deterministic), applies the INT8 per-channel scale, rounds to bf16 once and stores y.
+//     CTA pushes the s-th slice of tokens of its fp32 partial tile into CTA s's shared memory (distributed
+//     shared memory stores); after a second barrier CTA s sums the slots in fixed rank order (results are
+//     deterministic), applies the INT8 per-channel scale, rounds to bf16 once and stores y.
 //
-// Warp roles (224 threads): warp 0 = W0 / U_B producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 =
-// rank core + epilogue, warp 6 = x / V_A producer.  All mbarrier waits are bounded; a CTA that gives up
-// records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster barriers, frees its TMEM and exits.
+// The producers of u never wait for anything another CTA does, and they are the lowest-numbered CTAs of the
+// grid, so a consumer's wait always ends; it is bounded all the same.  Warp roles (224 threads): warp 0 = W0 /
+// U_B producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue, warp 6 = x / u
+// producer.  A CTA that gives up on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster
+// barriers, frees its TMEM and exits.
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -32,148 +36,334 @@ namespace {
 
 constexpr int DEC_M = 128;       // W0 rows per CTA (UMMA M)
 constexpr int DEC_K = 64;        // 64 bf16 = one 128-byte swizzle row
-constexpr int DEC_TOK = 256;     // tokens per tile (UMMA N limit)
 constexpr int kDecThreads = 224;
 constexpr int kDecSmemBudget = 227 * 1024;
 constexpr int W_TILE_BYTES = DEC_M * DEC_K * 2;  // 16 KB
-constexpr int kMaxWStages = 10, kMaxXStages = 4;
-constexpr int RECV_PAD = 4;      // floats of padding per receive-buffer row (bank-conflict-free 16-byte accesses)
+constexpr int kMaxWStages = 12, kMaxXStages = 6;
+constexpr int kMaxRankTokens = 4;  // tokens one worker CTA takes through the rank path at a time
+constexpr int DEC_AUX_BYTES = 8 * 1024;  // barriers, flags, rank-path reduction buffers
 
 struct DParams {
-  int T;          // tokens in the call
-  int tn;         // UMMA N of a token tile: multiple of 16, <= 256
-  int xrows;      // rows reserved per x stage (128 or 256): the down-projection reads 128-row halves
-  int d_out;
+  int T;          // tokens in the call (<= 256)
+  int tn;         // UMMA N: T rounded up to a multiple of 16
+  int xbox;       // rows per TMA box of the x tile (divides tn)
+  int d_in, d_out;
   int main_kb;    // d_in / 64
-  int m_tiles, tok_tiles, splits;
+  int m_tiles, splits;
   int w_stages, x_stages;
   int ext;        // U_B slabs: 1 (bf16 W0) or 2 (INT8 W0: hi + lo of U_B / scale)
   __nv_bfloat16* y;
   int ldy;
   const __half* scale;
+  // rank path
+  const __nv_bfloat16* x;    // [T][d_in]
+  const __nv_bfloat16* VAp;  // [d_in][vap_cols]
+  int vap_cols;
+  int rank_groups;           // groups of kMaxRankTokens tokens
+  int rank_slices;           // K slices per group; unit w = (group w / slices, slice w % slices)
+  int rank_ctas;             // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
+  int main_ctas;             // CTAs that stream W0 (m_tiles * splits); later CTAs of the grid only do rank units
+  float* p_part;             // [8][256][64] fp32: partial down-projections, one slot per K slice
+  int* grp_count;            // [64] arrivals per group (left at zero)
   const int32_t* seg;
   int P;
   const float* sigma;
   int ld_sigma, sA_col, sB_col, r;
-  const float* M;  // [64][64] fp32
+  const float* M;            // [64][64] fp32
+  __nv_bfloat16* u;          // [256][64] bf16, rows published by the workers
+  uint32_t* u_count;         // rows published so far (monotonic across calls)
+  uint32_t u_target;         // value of *u_count once this call's T rows are in
   int32_t* status;
 };
 
-__host__ __device__ inline int dec_x_stage_bytes(int xrows, int r_pad) { return xrows * 128 + r_pad * 128; }
 // tokens of the receive buffer each CTA of a cluster of `splits` owns: a multiple of 16 so that a 16-token
 // accumulator chunk never straddles two owners
 __host__ __device__ inline int dec_rows_per_owner(int tn, int splits) { return (((tn + splits - 1) / splits) + 15) / 16 * 16; }
 __host__ __device__ inline int dec_recv_bytes(int tn, int splits) {
-  return splits * DEC_M * (dec_rows_per_owner(tn, splits) + RECV_PAD) * 4;
+  return splits * dec_rows_per_owner(tn, splits) * DEC_M * 4;
 }
 
-// Candidate that owns token t.  Equal-length segments (the usual decode and prefill batches) are found by
-// one proportional guess checked against the offsets; anything else falls back to the binary search.
-__device__ __forceinline__ int find_candidate_guess(const int32_t* __restrict__ off, int P, int T, int t) {
-  const int g = min(P - 1, (int)(((long long)t * P) / T));
-  if (__ldg(off + g) <= t && t < __ldg(off + g + 1)) return g;
-  return find_candidate(off, P, t);
+__device__ __forceinline__ void bf16x8_to_float(const uint4& v, float (&f)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
 }
 
-template <int R_PAD>
+// One unit of the rank path, by the 128 epilogue threads of one CTA: the tokens of group `grp` (kMaxRankTokens
+// consecutive tokens) over the input features of K slice `slice` (of p.rank_slices).
+//   partial p = V_A[slice]^T x_t[slice] : thread (rb, cc) owns the 8 columns 8cc..8cc+7 and the row blocks
+//   rb, rb + RBS, ... of 8 input features each (one 16-byte load of x per token, eight of V_A per block, the next
+//   block's loads in flight while this one is multiplied); partial sums meet by xor-shuffles inside a warp and
+//   through shared memory across the four warps, and go to this slice's slot of a global buffer.
+//   The CTA that completes a group (arrival counter) sums the slots in slice order (deterministic), forms
+//   q = sA_k .* p, v = M q (thread j owns coordinate j), u = sB_k .* v, stores the 64-wide bf16 rows and adds
+//   the group's tokens to the published-row count.
+template <int COLS>
+__device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, float* red /*[4][G][COLS]*/,
+                                          float* qbuf /*[G][64]*/, volatile int* flag, int etid) {
+  constexpr int G = kMaxRankTokens;
+  constexpr int TPR = COLS / 8;      // threads per V_A row
+  constexpr int RBS = 128 / TPR;     // row blocks in flight
+  const int cc = etid % TPR, rb = etid / TPR;
+  const int warp_e = etid >> 5, lane = etid & 31;
+  const int t_begin = grp * G;
+  const int g_n = min(G, p.T - t_begin);
+  const int n_blocks = p.d_in / 8;
+  const int b_per = (n_blocks + p.rank_slices - 1) / p.rank_slices;
+  const int b0 = slice * b_per, b1 = min(n_blocks, b0 + b_per);
+  // Candidate lookup for the finishing step: equal-length segments are found by one proportional guess; its two
+  // offsets are requested now and looked at after the loop, so that no load of the loop waits behind them.
+  const int j = etid;
+  int guess[G], off_lo[G], off_hi[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    guess[g] = min(p.P - 1, (int)(((long long)(t_begin + (g < g_n ? g : 0)) * p.P) / p.T));
+    off_lo[g] = __ldg(p.seg + guess[g]);
+    off_hi[g] = __ldg(p.seg + guess[g] + 1);
+  }
+  float acc[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[g][c] = 0.f;
+  uint4 xr[G], vr[8];
+  auto fetch = [&](int b) {
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+      xr[g] = __ldg(reinterpret_cast<const uint4*>(p.x + (size_t)(t_begin + (g < g_n ? g : 0)) * p.d_in) + b);
+    const uint4* vrow = reinterpret_cast<const uint4*>(p.VAp + (size_t)b * 8 * COLS) + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) vr[i] = __ldg(vrow + (size_t)i * TPR);
+  };
+  int b = b0 + rb;
+  if (b < b1) fetch(b);
+  while (b < b1) {
+    float xv[G][8], vv[8][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) bf16x8_to_float(xr[g], xv[g]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) bf16x8_to_float(vr[i], vv[i]);
+    b += RBS;
+    if (b < b1) fetch(b);  // next block's loads fly while this block is multiplied
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(vv[i][c], xv[g][i], acc[g][c]);
+  }
+  // singular values of the tokens' candidates and this thread's row of the core matrix: one round trip, in flight
+  // during the reductions below
+  float s_a[G], s_b[G];
+  float4 mreg[COLS / 4];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    s_a[g] = 0.f; s_b[g] = 0.f;
+    if (j < p.r && g < g_n) {
+      const int t = t_begin + g;
+      const int k = (off_lo[g] <= t && t < off_hi[g]) ? guess[g] : find_candidate(p.seg, p.P, t);
+      const float* srow = p.sigma + (size_t)k * p.ld_sigma;
+      s_a[g] = __ldg(srow + p.sA_col + j);
+      s_b[g] = __ldg(srow + p.sB_col + j);
+    }
+  }
+#pragma unroll
+  for (int i4 = 0; i4 < COLS / 4; ++i4)
+    mreg[i4] = __ldg(reinterpret_cast<const float4*>(p.M + (j < kRankPadMax ? j : 0) * kRankPadMax) + i4);
+  // lanes with equal cc hold partial sums of the same columns: fold lane bits log2(TPR) .. 4
+#pragma unroll
+  for (int off = TPR; off < 32; off <<= 1)
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[g][c] += __shfl_xor_sync(0xffffffffu, acc[g][c], off);
+  if (lane < TPR) {
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) red[(warp_e * G + g) * COLS + 8 * cc + c] = acc[g][c];
+  }
+  epi_bar_sync();
+  bool last = true;
+  if (p.rank_slices > 1) {
+  // this slice's partial p -> its slot  [slice][token][64]
+  for (int idx = etid; idx < G * COLS; idx += 128) {
+    const int g = idx / COLS, c = idx % COLS;
+    if (g < g_n)
+      p.p_part[((size_t)slice * kDecodeMaxTokens + t_begin + g) * kRankPadMax + c] =
+          red[(0 * G + g) * COLS + c] + red[(1 * G + g) * COLS + c] + red[(2 * G + g) * COLS + c] + red[(3 * G + g) * COLS + c];
+  }
+  __threadfence();
+  epi_bar_sync();
+  if (etid == 0) {
+    const int prev = atomicAdd(p.grp_count + grp, 1);
+    const int is_last = prev == p.rank_slices - 1;
+    if (is_last) p.grp_count[grp] = 0;  // every slice has arrived: leave the counter clean for the next call
+    *flag = is_last;
+  }
+  epi_bar_sync();
+  last = *flag != 0;
+  if (last) __threadfence();
+  }
+  if (last) {
+    if (j < kRankPadMax) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float pj = 0.f;
+        if (g < g_n && j < p.r) {
+          if (p.rank_slices > 1) {
+            for (int sl = 0; sl < p.rank_slices; ++sl)
+              pj += ld_cg_f32(p.p_part + ((size_t)sl * kDecodeMaxTokens + t_begin + g) * kRankPadMax + j);
+          } else {
+            pj = red[(0 * G + g) * COLS + j] + red[(1 * G + g) * COLS + j] + red[(2 * G + g) * COLS + j] + red[(3 * G + g) * COLS + j];
+          }
+        }
+        qbuf[g * kRankPadMax + j] = pj * s_a[g];  // sA_k .* p  (zero beyond the rank)
+      }
+    }
+    epi_bar_sync();
+    if (j < kRankPadMax) {
+      float v[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) v[g] = 0.f;
+      if (j < p.r) {
+#pragma unroll
+        for (int i4 = 0; i4 < COLS / 4; ++i4) {
+          const float4 mm = mreg[i4];  // zero beyond the rank
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const float4 qq = *reinterpret_cast<const float4*>(qbuf + g * kRankPadMax + 4 * i4);
+            v[g] = fmaf(mm.x, qq.x, v[g]);
+            v[g] = fmaf(mm.y, qq.y, v[g]);
+            v[g] = fmaf(mm.z, qq.z, v[g]);
+            v[g] = fmaf(mm.w, qq.w, v[g]);
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        if (g < g_n) p.u[(size_t)(t_begin + g) * kRankPadMax + j] = __float2bfloat16(v[g] * s_b[g]);  // sB_k .* (M q)
+    }
+    // publish: every writer's rows are visible device-wide before the count moves
+    __threadfence();
+    epi_bar_sync();
+    if (etid == 0) red_release_add_u32(p.u_count, (uint32_t)g_n);
+  }
+  epi_bar_sync();  // red / qbuf / flag may be reused
+}
+
 __global__ void __launch_bounds__(kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmUB0,
+                   const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmUB0,
                    const __grid_constant__ CUtensorMap tmUB1, const DParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
-  const int x_bytes = p.xrows * 128;
-  const int xs_bytes = dec_x_stage_bytes(p.xrows, R_PAD);
-  uint8_t* smem_w = smem;                       // W0 ring (the U_B slabs are its last items)
-  uint8_t* smem_x = smem + SW * W_TILE_BYTES;   // x / V_A ring
-  uint8_t* smem_u = smem_x;                     // u tile: overlays x stage 0 once the K loop is done
-  float* smem_m = reinterpret_cast<float*>(smem_x + SX * xs_bytes);
-  uint8_t* aux = reinterpret_cast<uint8_t*>(smem_m + R_PAD * R_PAD);
-  // receive buffer of the cluster reduction, [splits][128 ch][per + pad] fp32: overlays both rings, which are
+  const int x_bytes = p.tn * 128;
+  uint8_t* smem_w = smem;                      // W0 ring (the U_B slabs are its last items)
+  uint8_t* smem_x = smem + SW * W_TILE_BYTES;  // x ring (the u tile is its last item)
+  uint8_t* aux = smem_x + SX * x_bytes;
+  // receive buffer of the cluster reduction, [splits][per tokens][128 ch] fp32: overlays both rings, which are
   // dead once every MMA of the cluster has completed
   float* recv = reinterpret_cast<float*>(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* red = reinterpret_cast<float*>(aux + 1024);       // [4][G][64]
+  float* qbuf = red + 4 * kMaxRankTokens * kRankPadMax;    // [G][64]
 
   const uint32_t bar_wfull = smem_u32(bars), bar_wempty = bar_wfull + 8 * kMaxWStages;
   const uint32_t bar_xfull = bar_wempty + 8 * kMaxWStages, bar_xempty = bar_xfull + 8 * kMaxXStages;
-  const uint32_t bar_p = bar_xempty + 8 * kMaxXStages, bar_u = bar_p + 8, bar_d = bar_u + 8, bar_drain = bar_d + 8;
+  const uint32_t bar_d = bar_xempty + 8 * kMaxXStages, bar_drain = bar_d + 8;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = (int)cluster_ctarank();
-  const int item = blockIdx.x / p.splits;
-  const int m_tile = item % p.m_tiles;
-  const int tok_tile = item / p.m_tiles;
+  const bool is_main = (int)blockIdx.x < p.main_ctas;  // later CTAs of the grid only take rank-path units
+  const int m_tile = blockIdx.x / p.splits;
   // this CTA's K blocks [kb0, kb1)
   const int kbase = p.main_kb / p.splits, krem = p.main_kb % p.splits;
   const int kb0 = split * kbase + min(split, krem);
   const int kb1 = kb0 + kbase + (split < krem ? 1 : 0);
-  const int nkb = kb1 - kb0;
-  const int n_w = nkb + p.ext;  // items of the W0 ring: the K blocks, then the U_B slabs
-  const int halves = p.tn > 128 ? 2 : 1;
+  const int nkb = is_main ? kb1 - kb0 : 0;
+  const int n_ext = (is_main && split == 0) ? p.ext : 0;  // K split 0 adds the rank term
+  const int n_w = nkb + n_ext;               // items of the W0 ring: the K blocks, then the U_B slabs
+  const int n_x = nkb + (n_ext ? 1 : 0);     // items of the x ring: the K blocks, then the u tile
   const int per = dec_rows_per_owner(p.tn, p.splits);
-  const int recv_ld = per + RECV_PAD;
-  constexpr uint32_t TMEM_COLS = 512;
-  constexpr uint32_t P_COL = 256;  // D_p halves at columns 256 and 320
-  const uint32_t x_tx = (uint32_t)(p.tn * 128 + R_PAD * 128);
+  constexpr uint32_t TMEM_COLS = 256;
 
-  auto load_w = [&](int i) {  // item i of the W0 ring
+  auto load_w = [&](int i) {  // item i of the W0 ring, as two 64-row boxes
     const int s = i % SW;
     const uint32_t fb = bar_wfull + 8 * s;
     mbar_expect_tx(fb, (uint32_t)W_TILE_BYTES);
     const uint32_t dst = smem_u32(smem_w + s * W_TILE_BYTES);
-    if (i < nkb) tma_load_2d(dst, &tmW, (kb0 + i) * DEC_K, m_tile * DEC_M, fb);
-    else tma_load_2d(dst, (i - nkb) == 0 ? &tmUB0 : &tmUB1, 0, m_tile * DEC_M, fb);
+    const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
+    const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
+    tma_load_2d(dst, tm, col, m_tile * DEC_M, fb);
+    tma_load_2d(dst + 64 * 128, tm, col, m_tile * DEC_M + 64, fb);
   };
-  auto load_x = [&](int i) {  // K block i of the x / V_A ring
+  auto load_x = [&](int i) {  // item i of the x ring
     const int s = i % SX;
     const uint32_t fb = bar_xfull + 8 * s;
-    uint8_t* st = smem_x + s * xs_bytes;
-    mbar_expect_tx(fb, x_tx);
-    tma_load_2d(smem_u32(st), &tmX, (kb0 + i) * DEC_K, tok_tile * DEC_TOK, fb);
-    tma_load_2d(smem_u32(st + x_bytes), &tmV, (kb0 + i) * DEC_K, 0, fb);
+    const uint32_t dst = smem_u32(smem_x + s * x_bytes);
+    mbar_expect_tx(fb, (uint32_t)x_bytes);
+    const CUtensorMap* tm = i < nkb ? &tmX : &tmU;
+    const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
+    for (int r = 0; r < p.tn; r += p.xbox) tma_load_2d(dst + (uint32_t)(r * 128), tm, col, r, fb);
   };
 
-  const int first_w = n_w < SW ? n_w : SW;  // both rings start empty: their first fills need no wait
-  const int first_x = nkb < SX ? nkb : SX;
+  const int first_w = n_w < SW ? n_w : SW;  // the ring starts empty: its first fill needs no wait
   if (threadIdx.x == 0) {
     for (int s = 0; s < SW; ++s) { mbar_init(bar_wfull + 8 * s, 1); mbar_init(bar_wempty + 8 * s, 1); }
     for (int s = 0; s < SX; ++s) { mbar_init(bar_xfull + 8 * s, 1); mbar_init(bar_xempty + 8 * s, 1); }
-    mbar_init(bar_p, 1);
-    mbar_init(bar_u, 128);
     mbar_init(bar_d, 1);
     mbar_init(bar_drain, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // start streaming at once
-    for (int i = 0; i < first_w; ++i) {
-      load_w(i);
-      if (i < first_x) load_x(i);
-    }
+    for (int i = 0; i < first_w; ++i) load_w(i);  // the frozen weights depend on nothing: stream at once
   }
-  if (warp == 1) {
+  if (warp == 1 && is_main) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base = is_main ? *tmem_slot : 0u;
 
   if (warp == 0 || warp == 6) {
     // ------------------------------------------------------------------ TMA producers (W0 ring / x ring)
     if (lane == 0) {
       const bool is_w = warp == 0;
       const int S = is_w ? SW : SX;
-      const int n = is_w ? n_w : nkb;
+      const int n = is_w ? n_w : n_x;
       const uint32_t bar_e = is_w ? bar_wempty : bar_xempty, bar_f = is_w ? bar_wfull : bar_xfull;
-      int issued = is_w ? first_w : first_x;
+      int issued = is_w ? first_w : 0;
       bool ok = true;
       for (int i = issued; i < n; ++i) {
-        if (!mbar_wait(bar_e + 8 * (i % S), (uint32_t)(((i / S) & 1) ^ 1), abort_flag, p.status)) { ok = false; break; }
-        if (is_w) load_w(i); else load_x(i);
+        if (i >= S && !mbar_wait(bar_e + 8 * (i % S), (uint32_t)(((i / S) & 1) ^ 1), abort_flag, p.status)) { ok = false; break; }
+        if (is_w) {
+          load_w(i);
+        } else {
+          if (i == nkb) {
+            // the u tile: wait until the workers have published all T rows (bounded), then order the
+            // async-proxy read after the acquire
+            const long long t0 = clock64();
+            while ((int32_t)(ld_acquire_u32(p.u_count) - p.u_target) < 0) {
+              if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+                ok = false;
+                break;
+              }
+            }
+            if (!ok) break;
+            fence_proxy_async_global();
+          }
+          load_x(i);
+        }
         ++issued;
       }
       if (!ok || *abort_flag) {
@@ -186,45 +376,35 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 && is_main) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc_main = make_idesc(DEC_M, p.tn);
-      constexpr uint32_t idesc_p = make_idesc(128, R_PAD);
+      const uint32_t idesc = make_idesc(DEC_M, p.tn);
       bool ok = true;
       for (int i = 0; i < nkb; ++i) {
         const int sw = i % SW, sx = i % SX;
         if (!mbar_wait(bar_xfull + 8 * sx, (uint32_t)((i / SX) & 1), abort_flag, p.status) ||
             !mbar_wait(bar_wfull + 8 * sw, (uint32_t)((i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        uint8_t* xs = smem_x + sx * xs_bytes;
         const uint64_t dw = make_smem_desc(smem_u32(smem_w + sw * W_TILE_BYTES));
-        const uint64_t dx = make_smem_desc(smem_u32(xs));
-        const uint64_t dv = make_smem_desc(smem_u32(xs + x_bytes));
-        const uint32_t acc0 = i > 0 ? 1u : 0u;
+        const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
 #pragma unroll
-        for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc_main, (acc0 | (uint32_t)k) ? 1u : 0u);
+        for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
         umma_commit(bar_wempty + 8 * sw);
-        for (int h = 0; h < halves; ++h) {
-          // rows h*128 .. h*128+127 of the x tile as the M side: +16 KB = +1024 in the (address >> 4) field
-#pragma unroll
-          for (int k = 0; k < DEC_K / 16; ++k)
-            umma_bf16(tmem_base + P_COL + 64 * h, dx + 1024 * h + 2 * k, dv + 2 * k, idesc_p, (acc0 | (uint32_t)k) ? 1u : 0u);
-        }
         umma_commit(bar_xempty + 8 * sx);
       }
-      if (ok) {
-        umma_commit(bar_p);
-        ok = mbar_wait(bar_u, 0, abort_flag, p.status);
-      }
-      for (int e = 0; ok && e < p.ext; ++e) {
-        const int i = nkb + e;
-        if (!mbar_wait(bar_wfull + 8 * (i % SW), (uint32_t)((i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        const uint64_t dub = make_smem_desc(smem_u32(smem_w + (i % SW) * W_TILE_BYTES));
-        const uint64_t du = make_smem_desc(smem_u32(smem_u));
-#pragma unroll
-        for (int k = 0; k < R_PAD / 16; ++k) umma_bf16(tmem_base, dub + 2 * k, du + 2 * k, idesc_main, 1u);
+      if (ok && n_ext > 0) {
+        // rank term: u tile (x ring item nkb) against the U_B slabs (W0 ring items nkb ..)
+        ok = mbar_wait(bar_xfull + 8 * (nkb % SX), (uint32_t)((nkb / SX) & 1), abort_flag, p.status);
+        const uint64_t du = make_smem_desc(smem_u32(smem_x + (nkb % SX) * x_bytes));
+        const int ksteps = (p.r + 15) / 16;
+        for (int e = 0; ok && e < n_ext; ++e) {
+          const int i = nkb + e;
+          if (!mbar_wait(bar_wfull + 8 * (i % SW), (uint32_t)((i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t dub = make_smem_desc(smem_u32(smem_w + (i % SW) * W_TILE_BYTES));
+          for (int k = 0; k < ksteps; ++k) umma_bf16(tmem_base, dub + 2 * k, du + 2 * k, idesc, 1u);
+        }
       }
       if (ok) {
         umma_commit(bar_d);
@@ -236,99 +416,32 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
   }
 
-  // ------------------------------------------------------------------ warps 2..5: rank core, then the epilogue
+  // ------------------------------------------------------------------ warps 2..5: rank path, then the epilogue
   const int quad = warp & 3;
-  const int row = quad * 32 + lane;  // TMEM lane owned by this thread (warps 2..5 only)
+  const int row = quad * 32 + lane;  // TMEM lane (output channel of the tile) owned by this thread
   const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
   const bool epi = warp >= 2 && warp <= 5;
   int got = 0;
   if (epi) {
-    // While the K loop streams: core matrix -> shared, this thread's candidates and their singular values.
-    constexpr int PRE = (R_PAD <= 32) ? 2 : 1;  // halves whose singular values are fetched ahead of the wait
-    for (int idx = threadIdx.x - 64; idx < R_PAD * R_PAD / 4; idx += 128) {
-      const int r = idx / (R_PAD / 4), c4 = idx % (R_PAD / 4);
-      reinterpret_cast<float4*>(smem_m)[idx] = __ldg(reinterpret_cast<const float4*>(p.M + r * kRankPadMax) + c4);
-    }
-    int cand[2];
-    float sa[PRE][R_PAD], sb[PRE][R_PAD];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int tl = h * 128 + row, t = tok_tile * DEC_TOK + tl;
-      cand[h] = (h < halves && tl < p.tn && t < p.T) ? find_candidate_guess(p.seg, p.P, p.T, t) : -1;
-    }
-    auto load_sigma = [&](int k, float (&a)[R_PAD], float (&b)[R_PAD]) {
-      const float* srow = p.sigma + (size_t)(k < 0 ? 0 : k) * p.ld_sigma;
-#pragma unroll
-      for (int i = 0; i < R_PAD; ++i) {
-        a[i] = (k >= 0 && i < p.r) ? __ldg(srow + p.sA_col + i) : 0.f;
-        b[i] = (k >= 0 && i < p.r) ? __ldg(srow + p.sB_col + i) : 0.f;
-      }
-    };
-#pragma unroll
-    for (int h = 0; h < PRE; ++h) load_sigma(cand[h], sa[h], sb[h]);
-    epi_bar_sync();  // core matrix is in shared memory
-
-    got = 1;
-    if (lane == 0) got = mbar_wait(bar_p, 0, abort_flag, p.status) ? 1 : 0;
-    got = __shfl_sync(0xffffffffu, got, 0);
-    if (got) {
-      while (!mbar_try_wait(bar_p, 0)) {}  // complete: returns at once (acquire for every lane)
-      tc_fence_after();
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (h < halves) {
-          const int tl = h * 128 + row;  // token within the tile
-          if (h >= PRE) load_sigma(cand[h], sa[0], sb[0]);
-          float (&a)[R_PAD] = sa[h < PRE ? h : 0];
-          float (&b)[R_PAD] = sb[h < PRE ? h : 0];
-          float q[R_PAD];
-#pragma unroll
-          for (int c = 0; c < R_PAD / 16; ++c) {
-            float v[16];
-            tmem_ld16(t_lane + P_COL + 64 * h + c * 16, v);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) q[c * 16 + i] = v[i] * a[c * 16 + i];  // sA_k .* p (zero for padding / no token)
-          }
-          if (tl < p.tn) {
-            uint32_t packed[R_PAD / 2];
-#pragma unroll
-            for (int j2 = 0; j2 < R_PAD / 2; ++j2) {
-              float uu[2];
-#pragma unroll
-              for (int hh = 0; hh < 2; ++hh) {
-                const int j = 2 * j2 + hh;
-                float acc = 0.f;
-#pragma unroll
-                for (int i4 = 0; i4 < R_PAD / 4; ++i4) {
-                  const float4 mm = *reinterpret_cast<const float4*>(smem_m + j * R_PAD + 4 * i4);
-                  acc = fmaf(mm.x, q[4 * i4], acc);
-                  acc = fmaf(mm.y, q[4 * i4 + 1], acc);
-                  acc = fmaf(mm.z, q[4 * i4 + 2], acc);
-                  acc = fmaf(mm.w, q[4 * i4 + 3], acc);
-                }
-                uu[hh] = acc * b[j];  // sB_k .* (M q)
-              }
-              packed[j2] = pack_bf16x2(uu[0], uu[1]);
-            }
-            // row tl of the K-major operand: 128 bytes, 16-byte chunk c stored at position c ^ (tl & 7)
-            uint8_t* urow = smem_u + (size_t)tl * 128;
-#pragma unroll
-            for (int c = 0; c < R_PAD / 8; ++c)
-              *reinterpret_cast<uint4*>(urow + ((c ^ (tl & 7)) << 4)) =
-                  make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
-          }
+    const int etid = threadIdx.x - 64;
+    if ((int)blockIdx.x < p.rank_ctas) {
+      // this CTA's units of the rank path, while its K loop streams
+      volatile int* flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+      for (int unit = blockIdx.x; unit < p.rank_groups * p.rank_slices; unit += p.rank_ctas) {
+        const int grp = unit / p.rank_slices, slice = unit % p.rank_slices;
+        switch (p.vap_cols) {
+          case 16: rank_unit<16>(p, grp, slice, red, qbuf, flag, etid); break;
+          case 32: rank_unit<32>(p, grp, slice, red, qbuf, flag, etid); break;
+          default: rank_unit<64>(p, grp, slice, red, qbuf, flag, etid); break;
         }
       }
-      fence_proxy_async_smem();
-      tc_fence_before();
-      mbar_arrive(bar_u);
-      // ---- wait for the accumulator (base + rank term of this K slice)
-      if (lane == 0) got = mbar_wait(bar_d, 0, abort_flag, p.status) ? 1 : 0;
-      got = __shfl_sync(0xffffffffu, got, 0);
-      if (got) {
-        while (!mbar_try_wait(bar_d, 0)) {}
-        tc_fence_after();
-      }
+    }
+    got = is_main ? 1 : 0;
+    if (is_main && lane == 0) got = mbar_wait(bar_d, 0, abort_flag, p.status) ? 1 : 0;
+    got = __shfl_sync(0xffffffffu, got, 0);
+    if (got) {
+      while (!mbar_try_wait(bar_d, 0)) {}  // complete: returns at once (acquire for every lane)
+      tc_fence_after();
     }
   }
 
@@ -338,8 +451,8 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   __syncwarp();
   cluster_sync_all();
   if (epi && got) {
-    // push: token chunk c (16 tokens) of this thread's channel goes to slot `split` of the chunk's owner,
-    // token-contiguous so that four tokens travel per store
+    // push: token chunk c (16 tokens) of this thread's channel goes to slot `split` of the chunk's owner;
+    // a warp writes 128 contiguous bytes (32 channels of one token) per store
     const uint32_t recv_addr = smem_u32(recv);
 #pragma unroll 1
     for (int c = 0; c < p.tn / 16; ++c) {
@@ -347,73 +460,50 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       tmem_ld16(t_lane + c * 16, v);
       const int owner = (c * 16) / per;
       const int j = c * 16 - owner * per;  // first token of the chunk within the owner's slice
-      const uint32_t dst = map_to_cta(recv_addr + (uint32_t)(((split * DEC_M + row) * recv_ld + j) * 4), (uint32_t)owner);
+      const uint32_t dst = map_to_cta(recv_addr + (uint32_t)((((split * per + j) * DEC_M) + row) * 4), (uint32_t)owner);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) st_dsmem_v4(dst + 16 * i, v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+      for (int i = 0; i < 16; ++i) st_dsmem_f32(dst + (uint32_t)(i * DEC_M * 4), v[i]);
     }
     tc_fence_before();
   }
   __syncwarp();
   cluster_sync_all();  // all partial sums have arrived; nobody touches a peer's shared memory after this point
-  if (epi) {
-    // thread = channel: sum the slots in rank order, scale, round, store (a warp writes 64 contiguous bytes per token)
-    const int ch = m_tile * DEC_M + row;
-    const int j_end = min(per, p.tn - split * per);  // tokens of this CTA's slice inside the tile
-    const int t0 = tok_tile * DEC_TOK + split * per;  // first token of the slice
-    const int j_lim = min(j_end, p.T - t0);           // ... and inside the call
-    if (ch < p.d_out) {
-      const float sc = p.scale != nullptr ? __half2float(__ldg(p.scale + ch)) : 1.f;
-      const float* mine = recv + (size_t)row * recv_ld;
-      __nv_bfloat16* ycol = p.y + (size_t)t0 * p.ldy + ch;
-      for (int j = 0; j < j_lim; j += 4) {
-        float4 acc = *reinterpret_cast<const float4*>(mine + j);
-        for (int r = 1; r < p.splits; ++r) {
-          const float4 v = *reinterpret_cast<const float4*>(mine + (size_t)r * DEC_M * recv_ld + j);
+  if (epi && is_main) {
+    // each thread owns 4 consecutive channels; warp ew takes tokens ew, ew + 4, ... of this CTA's slice
+    const int ew = warp - 2;
+    const int t0 = split * per;                             // first token of the slice
+    const int j_lim = min(min(per, p.tn - t0), p.T - t0);    // tokens of the slice inside the call
+    const int ch0 = m_tile * DEC_M + 4 * lane;
+    if (ch0 < p.d_out) {  // d_out is a multiple of 8: a group of 4 channels is all in or all out
+      float sc[4] = {1.f, 1.f, 1.f, 1.f};
+      if (p.scale != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sc[i] = __half2float(__ldg(p.scale + ch0 + i));
+      }
+      const float* mine = recv + 4 * lane;
+      __nv_bfloat16* yrow0 = p.y + (size_t)t0 * p.ldy + ch0;
+      for (int j = ew; j < j_lim; j += 4) {
+        float4 acc = *reinterpret_cast<const float4*>(mine + (size_t)j * DEC_M);
+        for (int r = 1; r < p.splits; ++r) {  // cluster rank order: deterministic
+          const float4 v = *reinterpret_cast<const float4*>(mine + ((size_t)r * per + j) * DEC_M);
           acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
-        const float o[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (j + i < j_lim) ycol[(size_t)(j + i) * p.ldy] = __float2bfloat16(o[i]);
+        uint2 o;
+        o.x = pack_bf16x2(acc.x * sc[0], acc.y * sc[1]);
+        o.y = pack_bf16x2(acc.z * sc[2], acc.w * sc[3]);
+        *reinterpret_cast<uint2*>(yrow0 + (size_t)j * p.ldy) = o;
       }
     }
   }
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 1 && is_main) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
-inline int dec_smem_bytes(int w_stages, int x_stages, int xrows, int r_pad) {
-  return 1024 + w_stages * W_TILE_BYTES + x_stages * dec_x_stage_bytes(xrows, r_pad) + r_pad * r_pad * 4 + 1024;
-}
-
-template <int R_PAD>
-int32_t launch_decode(essa_ctx* ctx, const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmV,
-                      const CUtensorMap& tmUB0, const CUtensorMap& tmUB1, const DParams& p, int smem_bytes,
-                      cudaStream_t stream) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(essa_decode_kernel<R_PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
-    attr_done = true;
-  }
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)(p.m_tiles * p.tok_tiles * p.splits), 1, 1);
-  cfg.blockDim = dim3(kDecThreads, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)smem_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)p.splits;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  ctx->launches += 1;
-  return check_cuda(ctx, cudaLaunchKernelEx(&cfg, essa_decode_kernel<R_PAD>, tmW, tmX, tmV, tmUB0, tmUB1, p),
-                    "essa_decode_kernel launch");
+inline int dec_smem_bytes(int w_stages, int x_stages, int tn) {
+  return 1024 + w_stages * W_TILE_BYTES + x_stages * tn * 128 + DEC_AUX_BYTES;
 }
 
 }  // namespace
@@ -421,30 +511,35 @@ int32_t launch_decode(essa_ctx* ctx, const CUtensorMap& tmW, const CUtensorMap& 
 // Schedule of the decode kernel for T tokens; returns false when the call should use the prefill kernels.
 bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out) {
   if (T <= 0 || T > kDecodeMaxTokens) return false;
+  (void)rank;
   const int sm = sm_count > 0 ? sm_count : 148;
-  const int r_pad = ((rank + 15) / 16) * 16;
   const int ext = (w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? 2 : 1;
-  const int tn = T <= DEC_TOK ? (int)((T + 15) / 16) * 16 : DEC_TOK;
-  const int tok_tiles = (int)((T + DEC_TOK - 1) / DEC_TOK);
-  const int xrows = tn <= 128 ? 128 : 256;
+  const int tn = (int)((T + 15) / 16) * 16;
   const int m_tiles = (d_out + DEC_M - 1) / DEC_M;
   const int main_kb = d_in / DEC_K;
-  const int items = m_tiles * tok_tiles;
   // cluster size: a power of two (packs into a GPC's SMs without stragglers), at most 8 (portable limit)
+  // All clusters must be resident at once (the CTAs that add the rank term wait for rows other CTAs publish, and
+  // a second wave would double the time anyway).  With one CTA per SM, clusters of 4 fill about 132 of 148 SMs
+  // and clusters of 8 about 120 (they may not straddle GPCs).
+  auto resident = [&](int c) { return c >= 8 ? sm * 120 / 148 : c >= 4 ? sm * 132 / 148 : sm; };
   int splits = 1;
-  while (splits * 2 <= 8 && items * splits * 2 <= sm && splits * 2 <= main_kb) splits *= 2;
+  while (splits * 2 <= 8 && m_tiles * splits * 2 <= resident(splits * 2) && splits * 2 <= main_kb) splits *= 2;
   const int kb_per = (main_kb + splits - 1) / splits;
-  // x / V_A tiles are L2 hits: two stages (three when they are small); the rest of shared memory holds W0 in flight
-  const int xs = dec_x_stage_bytes(xrows, r_pad);
-  int x_stages = xs <= 24 * 1024 ? 3 : 2;
-  if (x_stages > kb_per) x_stages = kb_per;
-  int w_stages = (kDecSmemBudget - dec_smem_bytes(0, x_stages, xrows, r_pad)) / W_TILE_BYTES;
+  // Ring depths.  Per K block the tensor core needs ~560 cycles; a tile load takes ~2500 (L2) to ~4000 (HBM)
+  // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
+  const int xb = tn * 128;
+  const int budget = kDecSmemBudget - dec_smem_bytes(0, 0, tn);
+  int x_stages = budget / (W_TILE_BYTES + xb);
+  if (x_stages > kMaxXStages) x_stages = kMaxXStages;
+  if (x_stages > kb_per + 1) x_stages = kb_per + 1;
+  if (x_stages < 1) return false;
+  int w_stages = (budget - x_stages * xb) / W_TILE_BYTES;
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
   if (w_stages > kb_per + ext) w_stages = kb_per + ext;
   if (w_stages < 1) return false;
   // the receive buffer of the cluster reduction overlays both rings
-  while (w_stages * W_TILE_BYTES + x_stages * xs < dec_recv_bytes(tn, splits)) ++w_stages;
-  if (w_stages > kMaxWStages || dec_smem_bytes(w_stages, x_stages, xrows, r_pad) > kDecSmemBudget) return false;
+  while (w_stages * W_TILE_BYTES + x_stages * xb < dec_recv_bytes(tn, splits)) ++w_stages;
+  if (w_stages > kMaxWStages || dec_smem_bytes(w_stages, x_stages, tn) > kDecSmemBudget) return false;
   out->block_m = DEC_M;
   out->block_n = tn;
   out->block_k = DEC_K;
@@ -452,8 +547,8 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
   out->x_stages = x_stages;
   out->k_blocks = main_kb + ext;
   out->splits = splits;
-  out->tiles = items;
-  out->grid = items * splits;
+  out->tiles = m_tiles;
+  out->grid = m_tiles * splits;
   out->down_splits = 0;
   out->down_grid = 0;
   out->scratch_bytes = 0;
@@ -466,11 +561,11 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   DParams p{};
   p.T = (int)g.T;
   p.tn = pl.block_n;
-  p.xrows = p.tn <= 128 ? 128 : 256;
+  p.xbox = (p.tn % 64 == 0) ? 64 : p.tn;
+  p.d_in = a->d_in;
   p.d_out = a->d_out;
   p.main_kb = a->d_in / DEC_K;
   p.m_tiles = (a->d_out + DEC_M - 1) / DEC_M;
-  p.tok_tiles = (int)((g.T + DEC_TOK - 1) / DEC_TOK);
   p.splits = pl.splits;
   p.w_stages = pl.stages;
   p.x_stages = pl.x_stages;
@@ -478,6 +573,51 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   p.y = g.y;
   p.ldy = a->d_out;
   p.scale = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? a->w0_scale : nullptr;
+  p.x = g.x;
+  p.VAp = a->VAp;
+  p.vap_cols = a->vap_cols;
+  // rank path: spread the tokens over the CTAs of the grid, a few tokens each (more per CTA for wide ranks,
+  // whose V_A is large enough that re-reading it per token would crowd L2)
+  const int grid = p.m_tiles * p.splits;
+  // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
+  static int resident_cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  {
+    const int smem_q = kDecSmemBudget;
+    if (resident_cache[p.splits] == 0) {
+      cudaFuncSetAttribute(essa_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
+      cudaLaunchConfig_t q{};
+      q.gridDim = dim3((unsigned)(148 * p.splits), 1, 1);
+      q.blockDim = dim3(kDecThreads, 1, 1);
+      q.dynamicSmemBytes = (size_t)smem_q;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = (unsigned)p.splits;
+      qa[0].val.clusterDim.y = 1;
+      qa[0].val.clusterDim.z = 1;
+      q.attrs = qa;
+      q.numAttrs = 1;
+      int n_clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, essa_decode_kernel, &q) != cudaSuccess || n_clusters <= 0) {
+        cudaGetLastError();
+        n_clusters = 1;  // unknown: only the first cluster is certainly in the first wave
+      }
+      resident_cache[p.splits] = n_clusters;
+    }
+  }
+  // Launch a full wave: the CTAs beyond the W0-streaming ones only take rank-path units.  A unit is a group of
+  // kMaxRankTokens tokens over one K slice; slices multiply the units until the wave is busy (at most 8).
+  const int resident_ctas = resident_cache[p.splits] * p.splits;
+  const int grid_total = grid > resident_ctas ? grid : resident_ctas;
+  p.main_ctas = grid;
+  p.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
+  p.rank_groups = (p.T + kMaxRankTokens - 1) / kMaxRankTokens;
+  int slices = p.rank_ctas / p.rank_groups;
+  if (slices > 8) slices = 8;
+  if (slices > a->d_in / 512) slices = a->d_in / 512;  // at least 64 row blocks per slice
+  if (slices < 1) slices = 1;
+  p.rank_slices = slices;
+  p.p_part = static_cast<float*>(ctx->dec_ppart);
+  p.grp_count = ctx->dec_grp;
   p.seg = g.seg_offsets;
   p.P = g.P;
   p.sigma = g.sigma;
@@ -486,25 +626,45 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   p.sB_col = g.sB_col;
   p.r = a->rank;
   p.M = a->M;
+  p.u = static_cast<__nv_bfloat16*>(ctx->dec_u);
+  p.u_count = ctx->dec_cnt;
+  ctx->dec_epoch += (uint32_t)p.T;
+  p.u_target = ctx->dec_epoch;
   p.status = ctx->d_status;
 
-  CUtensorMap tm_x;
+  CUtensorMap tm_x, tm_u;
   int32_t st = make_tensor_map_2d(ctx, &tm_x, 0, g.x, (uint64_t)g.T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
-                                  (uint32_t)p.tn, DEC_K, 128);
+                                  (uint32_t)p.xbox, DEC_K, 128);
   if (st != ESSA_OK) return st;
-  const int smem_bytes = dec_smem_bytes(p.w_stages, p.x_stages, p.xrows, a->r_pad);
+  st = make_tensor_map_2d(ctx, &tm_u, 0, ctx->dec_u, (uint64_t)kDecodeMaxTokens, kRankPadMax, kRankPadMax * 2,
+                          (uint32_t)p.xbox, DEC_K, 128);
+  if (st != ESSA_OK) return st;
+  const int smem_bytes = dec_smem_bytes(p.w_stages, p.x_stages, p.tn);
   if (smem_bytes > kDecSmemBudget || p.w_stages > kMaxWStages || p.x_stages > kMaxXStages)
     return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: decode schedule exceeds shared memory");
-  const CUtensorMap& tmW = a->tm_W0[1];  // 128-row boxes
-  const CUtensorMap& tmU0 = a->tm_UBp[1][0];
-  const CUtensorMap& tmU1 = a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0];
-  switch (a->r_pad) {
-    case 16: return launch_decode<16>(ctx, tmW, tm_x, a->tm_VAt, tmU0, tmU1, p, smem_bytes, stream);
-    case 32: return launch_decode<32>(ctx, tmW, tm_x, a->tm_VAt, tmU0, tmU1, p, smem_bytes, stream);
-    case 48: return launch_decode<48>(ctx, tmW, tm_x, a->tm_VAt, tmU0, tmU1, p, smem_bytes, stream);
-    case 64: return launch_decode<64>(ctx, tmW, tm_x, a->tm_VAt, tmU0, tmU1, p, smem_bytes, stream);
-    default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(essa_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
+    attr_done = true;
   }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid_total, 1, 1);
+  cfg.blockDim = dim3(kDecThreads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ctx->launches += 1;
+  // 64-row boxes of W0 and of the U_B slabs
+  return check_cuda(ctx, cudaLaunchKernelEx(&cfg, essa_decode_kernel, a->tm_W0[0], tm_x, tm_u, a->tm_UBp[0][0],
+                                            a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0], p),
+                    "essa_decode_kernel launch");
 }
 
 }  // namespace essa
