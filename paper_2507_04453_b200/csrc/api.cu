@@ -147,8 +147,8 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
       cudaMemset(ctx->dec_u, 0, (size_t)kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
       cudaMalloc(&ctx->dec_cnt, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t)) != cudaSuccess ||
       cudaMalloc(&ctx->dec_ppart, (size_t)8 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_grp, (size_t)kDecodeMaxTokens) != cudaSuccess ||
-      cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens) != cudaSuccess) {
+      cudaMalloc(&ctx->dec_grp, (size_t)kDecodeMaxTokens * 2) != cudaSuccess ||
+      cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens * 2) != cudaSuccess) {
     if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
     if (ctx->dec_grp) cudaFree(ctx->dec_grp);
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -198,7 +198,7 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
     if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
     cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t));
-    cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens);
+    cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens * 2);
     ctx->dec_epoch = 0;
   }
   return ESSA_OK;
@@ -289,6 +289,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
         st = make_tensor_map_2d(ctx, &a->tm_UBp[i][e2], 0, a->UBp + (size_t)e2 * m * kRankPadMax, m, kRankPadMax,
                                 kRankPadMax * 2, rows[i], 64, 128);
     }
+    if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q, 1, a->W0q, m, n, n, 128, 64, 0);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
   }
   // The temporaries (and, with host sources, the caller's buffers) are only needed until the copies and the

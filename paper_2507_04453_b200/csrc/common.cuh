@@ -67,6 +67,7 @@ struct essa_adapter {
   CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256
   CUtensorMap tm_UBp[3][2];
   CUtensorMap tm_VAt;
+  CUtensorMap tm_W0q;            // INT8 storage: the codes, 128-row x 64-byte boxes, unswizzled
 };
 
 namespace essa {

@@ -24,9 +24,9 @@
 //     deterministic), applies the INT8 per-channel scale, rounds to bf16 once and stores y.
 //
 // The producers of u never wait for anything another CTA does, and they are the lowest-numbered CTAs of the
-// grid, so a consumer's wait always ends; it is bounded all the same.  Warp roles (224 threads): warp 0 = W0 /
-// U_B producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue, warp 6 = x / u
-// producer.  A CTA that gives up on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster
+// grid, so a consumer's wait always ends; it is bounded all the same.  Warp roles (192 threads): warp 0 = TMA
+// producer of both rings, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue; INT8 storage
+// adds warps 6..11, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster
 // barriers, frees its TMEM and exits.
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -36,11 +36,15 @@ namespace {
 
 constexpr int DEC_M = 128;       // W0 rows per CTA (UMMA M)
 constexpr int DEC_K = 64;        // 64 bf16 = one 128-byte swizzle row
-constexpr int kDecThreads = 224;
+constexpr int kDecThreads = 192;
 constexpr int kDecSmemBudget = 227 * 1024;
 constexpr int W_TILE_BYTES = DEC_M * DEC_K * 2;  // 16 KB
-constexpr int kMaxWStages = 12, kMaxXStages = 6;
-constexpr int kMaxRankTokens = 4;  // tokens one worker CTA takes through the rank path at a time
+constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 6;
+constexpr int kInt8ConvStages = 3;  // converted tiles between the two converting warps and the tensor core
+constexpr int kDecThreadsInt8 = 256;             // + warps 6..7: INT8 -> bf16 converters
+constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored INT8 codes
+constexpr int kMaxRankTokens = 4;  // tokens of one rank-path unit (2 for the widest ranks, which need the registers)
+__host__ __device__ constexpr int rank_group_tokens(int vap_cols) { return vap_cols > 32 ? 2 : kMaxRankTokens; }
 constexpr int DEC_AUX_BYTES = 8 * 1024;  // barriers, flags, rank-path reduction buffers
 
 struct DParams {
@@ -51,6 +55,7 @@ struct DParams {
   int main_kb;    // d_in / 64
   int m_tiles, splits;
   int w_stages, x_stages;
+  int c_stages;   // INT8 storage: depth of the ring of converted (bf16) W0 tiles; 0 for bf16 storage
   int ext;        // U_B slabs: 1 (bf16 W0) or 2 (INT8 W0: hi + lo of U_B / scale)
   __nv_bfloat16* y;
   int ldy;
@@ -64,7 +69,7 @@ struct DParams {
   int rank_ctas;             // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
   int main_ctas;             // CTAs that stream W0 (m_tiles * splits); later CTAs of the grid only do rank units
   float* p_part;             // [8][256][64] fp32: partial down-projections, one slot per K slice
-  int* grp_count;            // [64] arrivals per group (left at zero)
+  int* grp_count;            // [128] arrivals per group (left at zero)
   const int32_t* seg;
   int P;
   const float* sigma;
@@ -92,8 +97,8 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& v, float (&f)[8]) {
   }
 }
 
-// One unit of the rank path, by the 128 epilogue threads of one CTA: the tokens of group `grp` (kMaxRankTokens
-// consecutive tokens) over the input features of K slice `slice` (of p.rank_slices).
+// One unit of the rank path, by the 128 epilogue threads of one CTA: the tokens of group `grp` (G consecutive
+// tokens) over the input features of K slice `slice` (of p.rank_slices).
 //   partial p = V_A[slice]^T x_t[slice] : thread (rb, cc) owns the 8 columns 8cc..8cc+7 and the row blocks
 //   rb, rb + RBS, ... of 8 input features each (one 16-byte load of x per token, eight of V_A per block, the next
 //   block's loads in flight while this one is multiplied); partial sums meet by xor-shuffles inside a warp and
@@ -104,7 +109,7 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& v, float (&f)[8]) {
 template <int COLS>
 __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, float* red /*[4][G][COLS]*/,
                                           float* qbuf /*[G][64]*/, volatile int* flag, int etid) {
-  constexpr int G = kMaxRankTokens;
+  constexpr int G = rank_group_tokens(COLS);
   constexpr int TPR = COLS / 8;      // threads per V_A row
   constexpr int RBS = 128 / TPR;     // row blocks in flight
   const int cc = etid % TPR, rb = etid / TPR;
@@ -129,31 +134,38 @@ __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, 
   for (int g = 0; g < G; ++g)
 #pragma unroll
     for (int c = 0; c < 8; ++c) acc[g][c] = 0.f;
+  // software pipeline at row granularity: as soon as a register of the current block has been unpacked, the same
+  // register is refilled with the next block's data, so a full block of loads is always in flight
   uint4 xr[G], vr[8];
-  auto fetch = [&](int b) {
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-      xr[g] = __ldg(reinterpret_cast<const uint4*>(p.x + (size_t)(t_begin + (g < g_n ? g : 0)) * p.d_in) + b);
-    const uint4* vrow = reinterpret_cast<const uint4*>(p.VAp + (size_t)b * 8 * COLS) + cc;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) vr[i] = __ldg(vrow + (size_t)i * TPR);
-  };
+  auto x_ptr = [&](int g, int b) { return reinterpret_cast<const uint4*>(p.x + (size_t)(t_begin + (g < g_n ? g : 0)) * p.d_in) + b; };
+  auto v_ptr = [&](int i, int b) { return reinterpret_cast<const uint4*>(p.VAp + (size_t)b * 8 * COLS) + cc + (size_t)i * TPR; };
   int b = b0 + rb;
-  if (b < b1) fetch(b);
+  if (b < b1) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) xr[g] = __ldg(x_ptr(g, b));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) vr[i] = __ldg(v_ptr(i, b));
+  }
   while (b < b1) {
-    float xv[G][8], vv[8][8];
+    const int bn = b + RBS;
+    const bool more = bn < b1;
+    float xv[G][8];
 #pragma unroll
-    for (int g = 0; g < G; ++g) bf16x8_to_float(xr[g], xv[g]);
+    for (int g = 0; g < G; ++g) {
+      bf16x8_to_float(xr[g], xv[g]);
+      if (more) xr[g] = __ldg(x_ptr(g, bn));
+    }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) bf16x8_to_float(vr[i], vv[i]);
-    b += RBS;
-    if (b < b1) fetch(b);  // next block's loads fly while this block is multiplied
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 8; ++i) {
+      float vv[8];
+      bf16x8_to_float(vr[i], vv);
+      if (more) vr[i] = __ldg(v_ptr(i, bn));
 #pragma unroll
       for (int g = 0; g < G; ++g)
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(vv[i][c], xv[g][i], acc[g][c]);
+        for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(vv[c], xv[g][i], acc[g][c]);
+    }
+    b = bn;
   }
   // singular values of the tokens' candidates and this thread's row of the core matrix: one round trip, in flight
   // during the reductions below
@@ -255,7 +267,23 @@ __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, 
   epi_bar_sync();  // red / qbuf / flag may be reused
 }
 
-__global__ void __launch_bounds__(kDecThreads, 1)
+// Four INT8 codes (one 32-bit word) -> four bf16 values, exactly and without leaving the 16-bit lanes: for a code
+// byte b, 0x4300 | (b & 0x7f) is the bf16 number 128 + low7(b) and 0x4300 | (b & 0x80) is 128 (b >= 0) or 256
+// (b < 0); their difference low7(b) - 128 sign(b) is the code, and all three numbers fit bf16's eight significant
+// bits, so the packed subtraction is exact.
+__device__ __forceinline__ void int8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t s0 = __byte_perm(w, 0u, 0x4140);  // [b0, 0, b1, 0]
+  const uint32_t s1 = __byte_perm(w, 0u, 0x4342);  // [b2, 0, b3, 0]
+  const uint32_t p0 = (s0 & 0x007f007fu) | 0x43004300u, d0 = (s0 & 0x00800080u) | 0x43004300u;
+  const uint32_t p1 = (s1 & 0x007f007fu) | 0x43004300u, d1 = (s1 & 0x00800080u) | 0x43004300u;
+  const __nv_bfloat162 q0 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p0), *reinterpret_cast<const __nv_bfloat162*>(&d0));
+  const __nv_bfloat162 q1 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p1), *reinterpret_cast<const __nv_bfloat162*>(&d1));
+  lo = *reinterpret_cast<const uint32_t*>(&q0);
+  hi = *reinterpret_cast<const uint32_t*>(&q1);
+}
+
+template <bool INT8>
+__global__ void __launch_bounds__(INT8 ? kDecThreadsInt8 : kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                    const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmUB0,
                    const __grid_constant__ CUtensorMap tmUB1, const DParams p) {
@@ -263,21 +291,25 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
   const int x_bytes = p.tn * 128;
-  uint8_t* smem_w = smem;                      // W0 ring (the U_B slabs are its last items)
-  uint8_t* smem_x = smem + SW * W_TILE_BYTES;  // x ring (the u tile is its last item)
+  constexpr int W_SLOT = INT8 ? RAW_TILE_BYTES : W_TILE_BYTES;
+  const int SC = INT8 ? p.c_stages : 0;
+  uint8_t* smem_w = smem;                      // W0 ring as stored (bf16: the U_B slabs are its last items)
+  uint8_t* smem_c = smem + SW * W_SLOT;        // INT8: ring of converted bf16 tiles (the U_B slabs are its last items)
+  uint8_t* smem_x = smem_c + SC * W_TILE_BYTES;  // x ring (the u tile is its last item)
   uint8_t* aux = smem_x + SX * x_bytes;
   // receive buffer of the cluster reduction, [splits][per tokens][128 ch] fp32: overlays both rings, which are
   // dead once every MMA of the cluster has completed
   float* recv = reinterpret_cast<float*>(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* red = reinterpret_cast<float*>(aux + 1024);       // [4][G][64]
   float* qbuf = red + 4 * kMaxRankTokens * kRankPadMax;    // [G][64]
 
   const uint32_t bar_wfull = smem_u32(bars), bar_wempty = bar_wfull + 8 * kMaxWStages;
   const uint32_t bar_xfull = bar_wempty + 8 * kMaxWStages, bar_xempty = bar_xfull + 8 * kMaxXStages;
-  const uint32_t bar_d = bar_xempty + 8 * kMaxXStages, bar_drain = bar_d + 8;
+  const uint32_t bar_cfull = bar_xempty + 8 * kMaxXStages, bar_cempty = bar_cfull + 8 * kMaxCStages;
+  const uint32_t bar_d = bar_cempty + 8 * kMaxCStages, bar_drain = bar_d + 8;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = (int)cluster_ctarank();
@@ -289,20 +321,33 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const int kb1 = kb0 + kbase + (split < krem ? 1 : 0);
   const int nkb = is_main ? kb1 - kb0 : 0;
   const int n_ext = (is_main && split == 0) ? p.ext : 0;  // K split 0 adds the rank term
-  const int n_w = nkb + n_ext;               // items of the W0 ring: the K blocks, then the U_B slabs
+  const int n_w = INT8 ? nkb : nkb + n_ext;  // items of the W0 ring: the K blocks (bf16: then the U_B slabs)
   const int n_x = nkb + (n_ext ? 1 : 0);     // items of the x ring: the K blocks, then the u tile
   const int per = dec_rows_per_owner(p.tn, p.splits);
   constexpr uint32_t TMEM_COLS = 256;
 
-  auto load_w = [&](int i) {  // item i of the W0 ring, as two 64-row boxes
+  auto load_w = [&](int i) {  // item i of the W0 ring
     const int s = i % SW;
     const uint32_t fb = bar_wfull + 8 * s;
+    mbar_expect_tx(fb, (uint32_t)W_SLOT);
+    const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
+    if (INT8) {  // 128 rows of 64 codes, unswizzled
+      tma_load_2d(dst, &tmW, (kb0 + i) * DEC_K, m_tile * DEC_M, fb);
+    } else {     // two 64-row boxes
+      const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
+      const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
+      tma_load_2d(dst, tm, col, m_tile * DEC_M, fb);
+      tma_load_2d(dst + 64 * 128, tm, col, m_tile * DEC_M + 64, fb);
+    }
+  };
+  auto load_ub = [&](int e) {  // INT8: U_B slab e goes straight into item nkb + e of the converted ring
+    const int s = (nkb + e) % (SC > 0 ? SC : 1);
+    const uint32_t fb = bar_cfull + 8 * s;
     mbar_expect_tx(fb, (uint32_t)W_TILE_BYTES);
-    const uint32_t dst = smem_u32(smem_w + s * W_TILE_BYTES);
-    const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
-    const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
-    tma_load_2d(dst, tm, col, m_tile * DEC_M, fb);
-    tma_load_2d(dst + 64 * 128, tm, col, m_tile * DEC_M + 64, fb);
+    const uint32_t dst = smem_u32(smem_c + s * W_TILE_BYTES);
+    const CUtensorMap* tm = e == 0 ? &tmUB0 : &tmUB1;
+    tma_load_2d(dst, tm, 0, m_tile * DEC_M, fb);
+    tma_load_2d(dst + 64 * 128, tm, 0, m_tile * DEC_M + 64, fb);
   };
   auto load_x = [&](int i) {  // item i of the x ring
     const int s = i % SX;
@@ -318,9 +363,12 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   if (threadIdx.x == 0) {
     for (int s = 0; s < SW; ++s) { mbar_init(bar_wfull + 8 * s, 1); mbar_init(bar_wempty + 8 * s, 1); }
     for (int s = 0; s < SX; ++s) { mbar_init(bar_xfull + 8 * s, 1); mbar_init(bar_xempty + 8 * s, 1); }
+    for (int s = 0; s < SC; ++s) { mbar_init(bar_cfull + 8 * s, 1); mbar_init(bar_cempty + 8 * s, 1); }
     mbar_init(bar_d, 1);
     mbar_init(bar_drain, 1);
     *abort_flag = 0;
+    *reinterpret_cast<volatile int*>(tmem_slot + 3) = 0;  // conversion ticket
+    *reinterpret_cast<volatile int*>(tmem_slot + 4) = 0;  // ... and whose turn it is to claim a slot
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int i = 0; i < first_w; ++i) load_w(i);  // the frozen weights depend on nothing: stream at once
   }
@@ -333,47 +381,53 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = is_main ? *tmem_slot : 0u;
 
-  if (warp == 0 || warp == 6) {
-    // ------------------------------------------------------------------ TMA producers (W0 ring / x ring)
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer: one thread feeds both rings,
+    // issuing whatever has a free slot (each ring in its own order, so the parity waits stay in step)
     if (lane == 0) {
-      const bool is_w = warp == 0;
-      const int S = is_w ? SW : SX;
-      const int n = is_w ? n_w : n_x;
-      const uint32_t bar_e = is_w ? bar_wempty : bar_xempty, bar_f = is_w ? bar_wfull : bar_xfull;
-      int issued = is_w ? first_w : 0;
+      int iw = first_w, ix = 0;  // next item of the W0 ring, of the x ring
       bool ok = true;
-      for (int i = issued; i < n; ++i) {
-        if (i >= S && !mbar_wait(bar_e + 8 * (i % S), (uint32_t)(((i / S) & 1) ^ 1), abort_flag, p.status)) { ok = false; break; }
-        if (is_w) {
-          load_w(i);
-        } else {
-          if (i == nkb) {
-            // the u tile: wait until the workers have published all T rows (bounded), then order the
-            // async-proxy read after the acquire
-            const long long t0 = clock64();
-            while ((int32_t)(ld_acquire_u32(p.u_count) - p.u_target) < 0) {
-              if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
-                atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
-                ok = false;
-                break;
-              }
-            }
-            if (!ok) break;
-            fence_proxy_async_global();
-          }
-          load_x(i);
+      long long t_idle = 0;
+      while (ok && (iw < n_w || ix < n_x)) {
+        bool progress = false;
+        if (iw < n_w && (iw < SW || mbar_test_wait(bar_wempty + 8 * (iw % SW), (uint32_t)(((iw / SW) & 1) ^ 1)))) {
+          load_w(iw++);
+          progress = true;
         }
-        ++issued;
+        if (ix < n_x && (ix < SX || mbar_test_wait(bar_xempty + 8 * (ix % SX), (uint32_t)(((ix / SX) & 1) ^ 1)))) {
+          // the u tile (item nkb) also needs every row published: acquire the count, then order the
+          // async-proxy read after it
+          const bool ready = ix < nkb || (int32_t)(ld_acquire_u32(p.u_count) - p.u_target) >= 0;
+          if (ready) {
+            if (ix == nkb) fence_proxy_async_global();
+            load_x(ix++);
+            progress = true;
+          }
+        }
+        if (progress) {
+          t_idle = 0;
+        } else {
+          const long long now = clock64();
+          if (t_idle == 0) t_idle = now;
+          if (*abort_flag || now - t_idle > kWaitLimitCycles) {
+            *abort_flag = 1;
+            atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+            ok = false;
+          }
+        }
       }
       if (!ok || *abort_flag) {
         // giving up: let the copies already issued land before the CTA's shared memory is released
-        const int outstanding = issued < S ? issued : S;
-        for (int j = 0; j < outstanding; ++j) {
-          const int i = issued - 1 - j;
-          const long long t0 = clock64();
-          while (!mbar_try_wait(bar_f + 8 * (i % S), (uint32_t)((i / S) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
-        }
+        auto drain = [&](int issued, int S, uint32_t bar_f) {
+          const int outstanding = issued < S ? issued : S;
+          for (int j = 0; j < outstanding; ++j) {
+            const int i = issued - 1 - j;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_f + 8 * (i % S), (uint32_t)((i / S) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
+          }
+        };
+        drain(iw, SW, bar_wfull);
+        drain(ix, SX, bar_xfull);
       }
     }
   } else if (warp == 1 && is_main) {
@@ -382,15 +436,17 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const uint32_t idesc = make_idesc(DEC_M, p.tn);
       bool ok = true;
       for (int i = 0; i < nkb; ++i) {
-        const int sw = i % SW, sx = i % SX;
+        const int sw = INT8 ? i % SC : i % SW, sx = i % SX;
+        const uint32_t wf = INT8 ? bar_cfull + 8 * sw : bar_wfull + 8 * sw;
+        const uint32_t wph = (uint32_t)((INT8 ? i / SC : i / SW) & 1);
         if (!mbar_wait(bar_xfull + 8 * sx, (uint32_t)((i / SX) & 1), abort_flag, p.status) ||
-            !mbar_wait(bar_wfull + 8 * sw, (uint32_t)((i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
+            !mbar_wait(wf, wph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint64_t dw = make_smem_desc(smem_u32(smem_w + sw * W_TILE_BYTES));
+        const uint64_t dw = make_smem_desc(smem_u32((INT8 ? smem_c : smem_w) + sw * W_TILE_BYTES));
         const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
 #pragma unroll
         for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-        umma_commit(bar_wempty + 8 * sw);
+        umma_commit((INT8 ? bar_cempty : bar_wempty) + 8 * sw);
         umma_commit(bar_xempty + 8 * sx);
       }
       if (ok && n_ext > 0) {
@@ -400,9 +456,10 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const int ksteps = (p.r + 15) / 16;
         for (int e = 0; ok && e < n_ext; ++e) {
           const int i = nkb + e;
-          if (!mbar_wait(bar_wfull + 8 * (i % SW), (uint32_t)((i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
+          const int su = INT8 ? i % SC : i % SW;
+          if (!mbar_wait((INT8 ? bar_cfull : bar_wfull) + 8 * su, (uint32_t)((INT8 ? i / SC : i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t dub = make_smem_desc(smem_u32(smem_w + (i % SW) * W_TILE_BYTES));
+          const uint64_t dub = make_smem_desc(smem_u32((INT8 ? smem_c : smem_w) + su * W_TILE_BYTES));
           for (int k = 0; k < ksteps; ++k) umma_bf16(tmem_base, dub + 2 * k, du + 2 * k, idesc, 1u);
         }
       }
@@ -415,6 +472,87 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       }
     }
   }
+
+  // ------------------------------------------------------------------ INT8 -> bf16 conversion (INT8 storage only)
+  // Items of the converted ring are handed out to warps 6..7 by a ticket counter in shared memory, so the two
+  // warps work on different tiles at once.  A warp converts a whole tile:
+  // raw tile = 128 rows of 64 codes, row r at byte 64 r; converted tile = the K-major 128-byte-swizzled operand
+  // layout, row r at byte 128 r, 16-byte chunk c at position c ^ (r & 7).  Lane l takes the 16-code chunks
+  // l, l + 32, ... (conflict-free 16-byte reads), two at a time for instruction-level parallelism.  Tickets
+  // nkb .. are the U_B slabs, which arrive ready-made by TMA into the same ring (its slots are reused in item
+  // order, which the ticket order preserves).
+  volatile int* ticket = reinterpret_cast<volatile int*>(tmem_slot + 3);
+  volatile int* turn = reinterpret_cast<volatile int*>(tmem_slot + 4);
+  auto convert_loop = [&]() {
+    const int SCd = SC > 0 ? SC : 1;
+    for (;;) {
+      int i = 0;
+      if (lane == 0) i = atomicAdd(const_cast<int*>(ticket), 1);
+      i = __shfl_sync(0xffffffffu, i, 0);
+      if (i >= nkb + n_ext) break;
+      const int sc = i % SCd;
+      int got_c = 1;
+      if (lane == 0) {
+        // Slots are claimed strictly in ticket order: a parity wait is only meaningful for the oldest waiter (a
+        // warp further ahead than the ring is deep would see the parity of an older phase), so each ticket
+        // holder first waits for its turn, then for its slot, then passes the turn on.
+        const long long t0 = clock64();
+        while (*turn != i) {
+          if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { got_c = 0; break; }
+        }
+        if (got_c) {
+          got_c = (i < SCd || mbar_wait(bar_cempty + 8 * sc, (uint32_t)(((i / SCd) & 1) ^ 1), abort_flag, p.status)) ? 1 : 0;
+          __threadfence_block();
+          *turn = i + 1;
+        }
+        if (!got_c) {
+          *abort_flag = 1;
+          atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+        }
+        if (got_c && i >= nkb) {
+          load_ub(i - nkb);
+          if (*abort_flag) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_cfull + 8 * sc, (uint32_t)((i / SCd) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
+          }
+        }
+        if (got_c && i < nkb) got_c = mbar_wait(bar_wfull + 8 * (i % SW), (uint32_t)((i / SW) & 1), abort_flag, p.status) ? 1 : 0;
+      }
+      got_c = __shfl_sync(0xffffffffu, got_c, 0);
+      if (!got_c) break;
+      if (i >= nkb) continue;
+      const int sr = i % SW;
+      while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}  // complete: acquire for every lane
+      const uint8_t* raw = smem_w + sr * RAW_TILE_BYTES;
+      uint8_t* out = smem_c + sc * W_TILE_BYTES;
+#pragma unroll 2
+      for (int c0 = 0; c0 < RAW_TILE_BYTES / 16; c0 += 64) {
+        uint4 w[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) w[h] = *reinterpret_cast<const uint4*>(raw + (c0 + 32 * h + lane) * 16);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int chunk = c0 + 32 * h + lane;
+          const int r = chunk >> 2, part = chunk & 3;
+          uint4 o0, o1;
+          int8x4_to_bf16x4(w[h].x, o0.x, o0.y);
+          int8x4_to_bf16x4(w[h].y, o0.z, o0.w);
+          int8x4_to_bf16x4(w[h].z, o1.x, o1.y);
+          int8x4_to_bf16x4(w[h].w, o1.z, o1.w);
+          uint8_t* orow = out + r * 128;
+          *reinterpret_cast<uint4*>(orow + (((2 * part) ^ (r & 7)) << 4)) = o0;
+          *reinterpret_cast<uint4*>(orow + (((2 * part + 1) ^ (r & 7)) << 4)) = o1;
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();  // the whole tile is written (and the raw tile read)
+      if (lane == 0) {
+        mbar_arrive(bar_cfull + 8 * sc);
+        mbar_arrive(bar_wempty + 8 * sr);
+      }
+    }
+  };
+  if (INT8 && warp >= 6) convert_loop();
 
   // ------------------------------------------------------------------ warps 2..5: rank path, then the epilogue
   const int quad = warp & 3;
@@ -502,8 +640,12 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   }
 }
 
-inline int dec_smem_bytes(int w_stages, int x_stages, int tn) {
-  return 1024 + w_stages * W_TILE_BYTES + x_stages * tn * 128 + DEC_AUX_BYTES;
+// c_stages > 0 means INT8 storage: the W0 ring holds 8 KB tiles of codes and c_stages converted tiles follow it
+inline int dec_ring_bytes(int w_stages, int c_stages, int x_stages, int tn) {
+  return w_stages * (c_stages > 0 ? RAW_TILE_BYTES : W_TILE_BYTES) + c_stages * W_TILE_BYTES + x_stages * tn * 128;
+}
+inline int dec_smem_bytes(int w_stages, int c_stages, int x_stages, int tn) {
+  return 1024 + dec_ring_bytes(w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
 }
 
 }  // namespace
@@ -527,19 +669,25 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
   const int kb_per = (main_kb + splits - 1) / splits;
   // Ring depths.  Per K block the tensor core needs ~560 cycles; a tile load takes ~2500 (L2) to ~4000 (HBM)
   // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
+  // INT8 storage: W0 tiles travel as 8 KB of codes; a ring of converted bf16 tiles (which also takes the U_B slabs,
+  // loaded into it directly) sits between the converting warps and the tensor core.
+  const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  const int c_stages = int8 ? kInt8ConvStages : 0;
+  const int w_slot = int8 ? RAW_TILE_BYTES : W_TILE_BYTES;
+  const int n_w_items = int8 ? kb_per : kb_per + ext;
   const int xb = tn * 128;
-  const int budget = kDecSmemBudget - dec_smem_bytes(0, 0, tn);
-  int x_stages = budget / (W_TILE_BYTES + xb);
+  const int budget = kDecSmemBudget - dec_smem_bytes(0, c_stages, 0, tn);
+  int x_stages = budget / (w_slot + xb);
   if (x_stages > kMaxXStages) x_stages = kMaxXStages;
   if (x_stages > kb_per + 1) x_stages = kb_per + 1;
   if (x_stages < 1) return false;
-  int w_stages = (budget - x_stages * xb) / W_TILE_BYTES;
+  int w_stages = (budget - x_stages * xb) / w_slot;
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
-  if (w_stages > kb_per + ext) w_stages = kb_per + ext;
+  if (w_stages > n_w_items) w_stages = n_w_items;
   if (w_stages < 1) return false;
-  // the receive buffer of the cluster reduction overlays both rings
-  while (w_stages * W_TILE_BYTES + x_stages * xb < dec_recv_bytes(tn, splits)) ++w_stages;
-  if (w_stages > kMaxWStages || dec_smem_bytes(w_stages, x_stages, tn) > kDecSmemBudget) return false;
+  // the receive buffer of the cluster reduction overlays the rings
+  while (dec_ring_bytes(w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) ++w_stages;
+  if (w_stages > kMaxWStages || dec_smem_bytes(w_stages, c_stages, x_stages, tn) > kDecSmemBudget) return false;
   out->block_m = DEC_M;
   out->block_n = tn;
   out->block_k = DEC_K;
@@ -567,12 +715,14 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   p.main_kb = a->d_in / DEC_K;
   p.m_tiles = (a->d_out + DEC_M - 1) / DEC_M;
   p.splits = pl.splits;
+  const bool int8 = a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   p.w_stages = pl.stages;
   p.x_stages = pl.x_stages;
+  p.c_stages = int8 ? kInt8ConvStages : 0;
   p.ext = a->ext_blocks;
   p.y = g.y;
   p.ldy = a->d_out;
-  p.scale = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? a->w0_scale : nullptr;
+  p.scale = int8 ? a->w0_scale : nullptr;
   p.x = g.x;
   p.VAp = a->VAp;
   p.vap_cols = a->vap_cols;
@@ -580,14 +730,17 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   // whose V_A is large enough that re-reading it per token would crowd L2)
   const int grid = p.m_tiles * p.splits;
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
-  static int resident_cache[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  static int resident_caches[2][9] = {};
+  int* resident_cache = resident_caches[int8 ? 1 : 0];
+  const void* kernel = int8 ? (const void*)essa_decode_kernel<true> : (const void*)essa_decode_kernel<false>;
+  const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
   {
     const int smem_q = kDecSmemBudget;
     if (resident_cache[p.splits] == 0) {
-      cudaFuncSetAttribute(essa_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
       cudaLaunchConfig_t q{};
       q.gridDim = dim3((unsigned)(148 * p.splits), 1, 1);
-      q.blockDim = dim3(kDecThreads, 1, 1);
+      q.blockDim = dim3((unsigned)threads, 1, 1);
       q.dynamicSmemBytes = (size_t)smem_q;
       cudaLaunchAttribute qa[1];
       qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -597,7 +750,7 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
       q.attrs = qa;
       q.numAttrs = 1;
       int n_clusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&n_clusters, essa_decode_kernel, &q) != cudaSuccess || n_clusters <= 0) {
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &q) != cudaSuccess || n_clusters <= 0) {
         cudaGetLastError();
         n_clusters = 1;  // unknown: only the first cluster is certainly in the first wave
       }
@@ -605,12 +758,13 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
     }
   }
   // Launch a full wave: the CTAs beyond the W0-streaming ones only take rank-path units.  A unit is a group of
-  // kMaxRankTokens tokens over one K slice; slices multiply the units until the wave is busy (at most 8).
+  // 4 tokens (2 for ranks above 32) over one K slice; slices multiply the units until the wave is busy (at most 8).
   const int resident_ctas = resident_cache[p.splits] * p.splits;
   const int grid_total = grid > resident_ctas ? grid : resident_ctas;
   p.main_ctas = grid;
   p.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
-  p.rank_groups = (p.T + kMaxRankTokens - 1) / kMaxRankTokens;
+  const int gtok = rank_group_tokens(a->vap_cols);
+  p.rank_groups = (p.T + gtok - 1) / gtok;
   int slices = p.rank_ctas / p.rank_groups;
   if (slices > 8) slices = 8;
   if (slices > a->d_in / 512) slices = a->d_in / 512;  // at least 64 row blocks per slice
@@ -639,18 +793,16 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   st = make_tensor_map_2d(ctx, &tm_u, 0, ctx->dec_u, (uint64_t)kDecodeMaxTokens, kRankPadMax, kRankPadMax * 2,
                           (uint32_t)p.xbox, DEC_K, 128);
   if (st != ESSA_OK) return st;
-  const int smem_bytes = dec_smem_bytes(p.w_stages, p.x_stages, p.tn);
+  const int smem_bytes = dec_smem_bytes(p.w_stages, p.c_stages, p.x_stages, p.tn);
   if (smem_bytes > kDecSmemBudget || p.w_stages > kMaxWStages || p.x_stages > kMaxXStages)
     return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: decode schedule exceeds shared memory");
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(essa_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
+  {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
-    attr_done = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid_total, 1, 1);
-  cfg.blockDim = dim3(kDecThreads, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -661,10 +813,11 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   ctx->launches += 1;
-  // 64-row boxes of W0 and of the U_B slabs
-  return check_cuda(ctx, cudaLaunchKernelEx(&cfg, essa_decode_kernel, a->tm_W0[0], tm_x, tm_u, a->tm_UBp[0][0],
-                                            a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0], p),
-                    "essa_decode_kernel launch");
+  const CUtensorMap& tmU0 = a->tm_UBp[0][0];  // 64-row boxes of the U_B slabs
+  const CUtensorMap& tmU1 = a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0];
+  const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, a->tm_W0q, tm_x, tm_u, tmU0, tmU1, p)
+                             : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, a->tm_W0[0], tm_x, tm_u, tmU0, tmU1, p);
+  return check_cuda(ctx, e, "essa_decode_kernel launch");
 }
 
 }  // namespace essa
