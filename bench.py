@@ -235,7 +235,7 @@ def run_ours(args, cfg):
     # Weights that fit L2 (decode configurations) would be served from it on every step: rotate through enough
     # device copies of the block's adapters that each step streams its W0 from HBM, as a forward pass over many
     # layers does.
-    w_bytes = sum(a.d_in * a.d_out * 2 for a in adapters)  # the tensor-core operand is bf16
+    w_bytes = sum(a.d_in * a.d_out * (1 if cfg.w0_dtype == 'int8' else 2) for a in adapters)  # as stored
     L2_BYTES = 126e6
     copies = 1 if w_bytes > 2 * L2_BYTES else int(np.ceil(2 * L2_BYTES / w_bytes)) + 1
     handle_sets = [[ctx.load_adapter(a) for a in adapters] for _ in range(copies)]
@@ -251,6 +251,8 @@ def run_ours(args, cfg):
     sigma = torch.empty((cfg.P, cfg.d), dtype=torch.float32, device="cuda")
     k_begin = rank * cfg.P  # weak scaling: rank g evaluates candidates [g*P, (g+1)*P) of an N*P population
     ctx.reserve(T, max(a.d_in for a in adapters), max(a.d_out for a in adapters))
+    if cfg.w0_dtype == "int8":
+        ctx.reserve_dequant(max(a.d_in for a in adapters), max(a.d_out for a in adapters))
     stream = torch.cuda.current_stream()
 
     step_no = [0]

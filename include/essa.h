@@ -77,6 +77,10 @@ int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);
  * up to max_tokens tokens and max_d_out output channels so that later calls do not allocate. */
 int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out);
 
+/* Pre-size the context's dequantisation scratch (d_in * d_out bf16) that prefill-sized calls on INT8-stored
+ * adapters use, so that those calls do not allocate.  Needed before essa_apply_projection_static on such adapters. */
+int32_t essa_reserve_dequant(essa_ctx* ctx, int32_t max_d_in, int32_t max_d_out);
+
 /* Frozen data of one adapted projection (Section 3, "LoRA + SVD parameterization"). */
 typedef struct essa_adapter_desc {
   int32_t d_in;     /* n: input features.  Must be a multiple of 64.                           */
@@ -154,6 +158,9 @@ int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* adapter, c
  *   - T > ESSA_STATIC_MAX_TOKENS is rejected with ESSA_ERR_UNSUPPORTED_SHAPE (and a message in
  *     essa_last_error); use essa_apply_projection for larger batches.
  *   - The context's device must be the current device, else ESSA_ERR_INVALID_ARG.
+ *   - Adapters stored as INT8 are dequantised per call into the context's dequantisation scratch; this entry
+ *     point does not grow it and returns ESSA_ERR_ALLOC unless essa_reserve_dequant (or an earlier
+ *     essa_apply_projection on an adapter at least as large) has sized it.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that first
  *     call before any stream capture.
  *   - All calls, from every context and stream on that GPU, share the one array and it keeps the last call's

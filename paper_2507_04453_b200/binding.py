@@ -32,7 +32,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
-    "essa_apply_projection_static", "essa_get_launch_count",
+    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant",
 )
 
 
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
         "essa_get_status": (i32, [vp, C.POINTER(i32)]),
         "essa_reserve": (i32, [vp, i64, i32, i32]),
         "essa_get_launch_count": (i32, [vp, C.POINTER(i64)]),
+        "essa_reserve_dequant": (i32, [vp, i32, i32]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -184,6 +185,10 @@ class Context:
 
     def reserve(self, max_tokens: int, max_d_in: int, max_d_out: int):
         self._check(self.lib.essa_reserve(self.handle, max_tokens, max_d_in, max_d_out))
+
+    def reserve_dequant(self, max_d_in: int, max_d_out: int):
+        """essa_reserve_dequant: pre-size the scratch that prefill calls on INT8-stored adapters dequantise into."""
+        self._check(self.lib.essa_reserve_dequant(self.handle, max_d_in, max_d_out))
 
     # -- adapters
     def load_adapter(self, ad) -> AdapterHandle:

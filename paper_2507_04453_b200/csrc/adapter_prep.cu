@@ -52,23 +52,24 @@ __global__ void build_core_kernel(const __nv_bfloat16* __restrict__ U_A, const _
   M[idx] = acc;
 }
 
-// INT8 codes -> bf16 (exact for |q| <= 127).
+// INT8 codes -> bf16 (exact), 16 codes per thread.  count is a multiple of 64 (d_in is).
 __global__ void widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* __restrict__ out, size_t count) {
-  size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 4;
-  if (i + 3 < count) {
-    const char4 v = *reinterpret_cast<const char4*>(q + i);
-    __nv_bfloat162 lo = __floats2bfloat162_rn((float)v.x, (float)v.y), hi = __floats2bfloat162_rn((float)v.z, (float)v.w);
-    reinterpret_cast<__nv_bfloat162*>(out + i)[0] = lo;
-    reinterpret_cast<__nv_bfloat162*>(out + i)[1] = hi;
-  } else {
-    for (; i < count; ++i) out[i] = __float2bfloat16((float)q[i]);
-  }
+  const size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 16;
+  if (i >= count) return;
+  const uint4 w = *reinterpret_cast<const uint4*>(q + i);
+  uint4 o0, o1;
+  int8x4_to_bf16x4(w.x, o0.x, o0.y);
+  int8x4_to_bf16x4(w.y, o0.z, o0.w);
+  int8x4_to_bf16x4(w.z, o1.x, o1.y);
+  int8x4_to_bf16x4(w.w, o1.z, o1.w);
+  reinterpret_cast<uint4*>(out + i)[0] = o0;
+  reinterpret_cast<uint4*>(out + i)[1] = o1;
 }
 
 }  // namespace
 
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream) {
-  const size_t threads = (count + 3) / 4;
+  const size_t threads = (count + 15) / 16;
   widen_int8_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(q, out, count);
   ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "widen_int8 launch");

@@ -174,6 +174,7 @@ int32_t essa_destroy(essa_ctx* ctx) {
   free_scratch(ctx->stage_y);
   free_scratch(ctx->stage_off);
   free_scratch(ctx->stage_sigma);
+  free_scratch(ctx->w_deq);
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->dec_u) cudaFree(ctx->dec_u);
@@ -226,6 +227,13 @@ int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_
   return check_cuda(ctx, cudaDeviceSynchronize(), "cudaDeviceSynchronize");
 }
 
+int32_t essa_reserve_dequant(essa_ctx* ctx, int32_t max_d_in, int32_t max_d_out) {
+  if (!ctx || max_d_in < 0 || max_d_out < 0) return ESSA_ERR_INVALID_ARG;
+  const int32_t st = ensure_scratch(ctx, ctx->w_deq, (size_t)max_d_in * max_d_out * 2, false, nullptr);
+  if (st != ESSA_OK) return st;
+  return check_cuda(ctx, cudaDeviceSynchronize(), "cudaDeviceSynchronize");
+}
+
 int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapter** out, void* stream_v) {
   if (!ctx) return ESSA_ERR_INVALID_ARG;
   if (!d || !out) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: NULL descriptor or output");
@@ -248,13 +256,14 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   a->ext_blocks = int8 ? 2 : 1;
   a->vap_cols = a->r_pad <= 16 ? 16 : a->r_pad <= 32 ? 32 : 64;
   const size_t n = d->d_in, m = d->d_out, r = d->rank;
-  // The INT8 weights are widened once to bf16 (exact: |q| <= 127) for the tensor-core operand; the fp16
+  // INT8 weights stay stored as codes (1 byte per weight).  The decode kernel converts them to bf16 in shared
+  // memory; a prefill call dequantises them once into the context's scratch before its GEMM.  Either way the fp16
   // per-channel scale is applied to the fp32 accumulator, so the dequantisation is exact.
   const size_t w0_bytes = m * n * 2;
   __nv_bfloat16 *dUA = nullptr, *dVB = nullptr;
   cudaError_t e = cudaSuccess;
   auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
-  alloc(&a->W0, w0_bytes);
+  if (!int8) alloc(&a->W0, w0_bytes);
   if (int8) { alloc((void**)&a->w0_scale, m * 2); alloc((void**)&a->W0q, m * n); }
   alloc((void**)&a->VAt, (size_t)kRankPadMax * n * 2);
   alloc((void**)&a->UBp, (size_t)a->ext_blocks * m * kRankPadMax * 2);
@@ -279,12 +288,11 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   copy(a->V_A, d->V_A, n * r * 2);
   copy(dUA, d->U_A, r * r * 2);
   copy(dVB, d->V_B, r * r * 2);
-  if (st == ESSA_OK && int8) st = launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(a->W0), m * n, stream);
   if (st == ESSA_OK) st = launch_adapter_prep(ctx, a, dUA, dVB, stream);
   if (st == ESSA_OK) {
     const uint32_t rows[3] = {64, 128, 256};
     for (int i = 0; i < 3 && st == ESSA_OK; ++i) {
-      st = make_tensor_map_2d(ctx, &a->tm_W0[i], 0, a->W0, m, n, n * 2, rows[i], 64, 128);
+      if (!int8) st = make_tensor_map_2d(ctx, &a->tm_W0[i], 0, a->W0, m, n, n * 2, rows[i], 64, 128);
       for (int e2 = 0; e2 < a->ext_blocks && st == ESSA_OK; ++e2)
         st = make_tensor_map_2d(ctx, &a->tm_UBp[i][e2], 0, a->UBp + (size_t)e2 * m * kRankPadMax, m, kRankPadMax,
                                 kRankPadMax * 2, rows[i], 64, 128);

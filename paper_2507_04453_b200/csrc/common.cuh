@@ -44,6 +44,7 @@ struct essa_ctx {
   essa::Scratch splitk_cnt;   // int32 arrival counters, one per output tile (kept zero between calls)
   essa::Scratch simt_buf;     // [T_cap][64] fp32: rank-path vector of the CUDA-core cross-check path
   essa::Scratch stage_x, stage_y, stage_off, stage_sigma;  // device staging of the host-buffer entry point
+  essa::Scratch w_deq;        // [d_out][d_in] bf16: INT8 W0 of the current prefill call, dequantised (unscaled) per call
   void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
   // essa_profile_begin/end: three events per recorded call
   bool prof_on = false;
@@ -53,7 +54,7 @@ struct essa_ctx {
 
 struct essa_adapter {
   int d_in = 0, d_out = 0, rank = 0, r_pad = 0, w0_dtype = 0;
-  void* W0 = nullptr;            // [d_out][d_in] bf16 (INT8 storage: the integer codes widened to bf16, unscaled)
+  void* W0 = nullptr;            // [d_out][d_in] bf16 (bf16 storage only)
   int8_t* W0q = nullptr;         // [d_out][d_in] int8 codes as given (INT8 storage only)
   __half* w0_scale = nullptr;    // [d_out] fp16 (INT8)
   __nv_bfloat16* VAt = nullptr;  // [64][d_in]: V_A^T, rows >= rank are zero (K-major B operand of the down-projection)
@@ -64,7 +65,7 @@ struct essa_adapter {
   int vap_cols = 0;
   float* M = nullptr;            // [64][64] fp32: M = V_B^T U_A zero-padded
   int ext_blocks = 1;            // rank-path K-slabs appended to the base contraction (1 bf16, 2 INT8)
-  CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256
+  CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256 (bf16 storage only)
   CUtensorMap tm_UBp[3][2];
   CUtensorMap tm_VAt;
   CUtensorMap tm_W0q;            // INT8 storage: the codes, 128-row x 64-byte boxes, unswizzled
@@ -116,6 +117,21 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
                                  cudaStream_t stream);
 
 #ifdef __CUDACC__
+// Four INT8 codes (one 32-bit word) -> four bf16 values, exactly and without leaving the 16-bit lanes: for a code
+// byte b, 0x4300 | (b & 0x7f) is the bf16 number 128 + low7(b) and 0x4300 | (b & 0x80) is 128 (b >= 0) or 256
+// (b < 0); their difference low7(b) - 128 sign(b) is the code, and all three numbers fit bf16's eight significant
+// bits, so the packed subtraction is exact.
+__device__ __forceinline__ void int8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t s0 = __byte_perm(w, 0u, 0x4140);  // [b0, 0, b1, 0]
+  const uint32_t s1 = __byte_perm(w, 0u, 0x4342);  // [b2, 0, b3, 0]
+  const uint32_t p0 = (s0 & 0x007f007fu) | 0x43004300u, d0 = (s0 & 0x00800080u) | 0x43004300u;
+  const uint32_t p1 = (s1 & 0x007f007fu) | 0x43004300u, d1 = (s1 & 0x00800080u) | 0x43004300u;
+  const __nv_bfloat162 q0 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p0), *reinterpret_cast<const __nv_bfloat162*>(&d0));
+  const __nv_bfloat162 q1 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p1), *reinterpret_cast<const __nv_bfloat162*>(&d1));
+  lo = *reinterpret_cast<const uint32_t*>(&q0);
+  hi = *reinterpret_cast<const uint32_t*>(&q1);
+}
+
 // Largest k in [0, P-1] with off[k] <= t (candidate that owns token t; empty segments own nothing).
 // Never reads outside off[0..P]; for offsets that are not monotone the result is some k in range.
 __device__ __forceinline__ int find_candidate(const int32_t* __restrict__ off, int P, int t) {

@@ -26,8 +26,8 @@
 // The producers of u never wait for anything another CTA does, and they are the lowest-numbered CTAs of the
 // grid, so a consumer's wait always ends; it is bounded all the same.  Warp roles (192 threads): warp 0 = TMA
 // producer of both rings, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue; INT8 storage
-// adds warps 6..11, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster
-// barriers, frees its TMEM and exits.
+// adds warps 6..7, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
+// on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster barriers, frees its TMEM and exits.
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -265,21 +265,6 @@ __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, 
     if (etid == 0) red_release_add_u32(p.u_count, (uint32_t)g_n);
   }
   epi_bar_sync();  // red / qbuf / flag may be reused
-}
-
-// Four INT8 codes (one 32-bit word) -> four bf16 values, exactly and without leaving the 16-bit lanes: for a code
-// byte b, 0x4300 | (b & 0x7f) is the bf16 number 128 + low7(b) and 0x4300 | (b & 0x80) is 128 (b >= 0) or 256
-// (b < 0); their difference low7(b) - 128 sign(b) is the code, and all three numbers fit bf16's eight significant
-// bits, so the packed subtraction is exact.
-__device__ __forceinline__ void int8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
-  const uint32_t s0 = __byte_perm(w, 0u, 0x4140);  // [b0, 0, b1, 0]
-  const uint32_t s1 = __byte_perm(w, 0u, 0x4342);  // [b2, 0, b3, 0]
-  const uint32_t p0 = (s0 & 0x007f007fu) | 0x43004300u, d0 = (s0 & 0x00800080u) | 0x43004300u;
-  const uint32_t p1 = (s1 & 0x007f007fu) | 0x43004300u, d1 = (s1 & 0x00800080u) | 0x43004300u;
-  const __nv_bfloat162 q0 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p0), *reinterpret_cast<const __nv_bfloat162*>(&d0));
-  const __nv_bfloat162 q1 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p1), *reinterpret_cast<const __nv_bfloat162*>(&d1));
-  lo = *reinterpret_cast<const uint32_t*>(&q0);
-  hi = *reinterpret_cast<const uint32_t*>(&q1);
 }
 
 template <bool INT8>

@@ -32,6 +32,8 @@ def test_static_variant_matches_regular_entry_point_twice(base, dm, dkv, r, P, L
     ctx = binding.Context(0)
     cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
     case = Case(torch, ctx, cfg, projections=[0, 1])
+    if cfg.w0_dtype == "int8":
+        ctx.reserve_dequant(dm, dm)  # set-up time: the allocation-free call will not size this scratch itself
     for i in (0, 1):
         x = to_dev(torch, case.tokens(i), torch.bfloat16)
         sA, sB = cfg.sigma_cols(i)
