@@ -715,8 +715,8 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   // whose V_A is large enough that re-reading it per token would crowd L2)
   const int grid = p.m_tiles * p.splits;
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
-  static int resident_caches[2][9] = {};
-  int* resident_cache = resident_caches[int8 ? 1 : 0];
+  static int resident_caches[64][2][9] = {};  // per device, storage type, cluster size
+  int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][int8 ? 1 : 0];
   const void* kernel = int8 ? (const void*)essa_decode_kernel<true> : (const void*)essa_decode_kernel<false>;
   const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
   {

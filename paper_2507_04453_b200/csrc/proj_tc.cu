@@ -395,7 +395,8 @@ template <int BLOCK_N, int EPI>
 int32_t launch_one(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2,
                    const CUtensorMap& tmB2a, const CUtensorMap& tmB2b, const KParams& p, int grid, cudaStream_t stream) {
   using C = Cfg<BLOCK_N, EPI>;
-  static bool attr_done = false;
+  static bool attr_done_dev[64] = {};  // the attribute is per device
+  bool& attr_done = attr_done_dev[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0];
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(essa_tc_kernel<BLOCK_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          C::SMEM_BYTES);
