@@ -256,14 +256,18 @@ def run_ours(args, cfg):
     stream = torch.cuda.current_stream()
 
     step_no = [0]
+    cols = [cfg.sigma_cols(i) for i in range(len(adapters))]
+    block_call = T <= 256 and len(adapters) > 1 and not args.single_calls
 
     def step():
         hs = handle_sets[step_no[0] % copies]
         step_no[0] += 1
         ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, out=sigma, k_begin=k_begin)
-        for i, h in enumerate(hs):
-            sA, sB = cfg.sigma_cols(i)
-            ctx.apply_projection(h, xs[i], d_off, sigma, sA, sB, out=ys[i])
+        if block_call:  # decode sizes: the block's projections share tokens, segments and the table -> one call
+            ctx.apply_block(hs, xs, d_off, sigma, cols, outs=ys)
+        else:
+            for i, h in enumerate(hs):
+                ctx.apply_projection(h, xs[i], d_off, sigma, cols[i][0], cols[i][1], out=ys[i])
 
     def barrier():
         torch.cuda.synchronize()
@@ -336,14 +340,15 @@ def run_ours(args, cfg):
     model = block_roofline(cfg, T, peaks, sustained=not decode)
     calls = max(prof["calls"], 1)
     main_s = prof["base_up_ms"] * 1e-3 / calls  # average launch duration
+    per_call = 1 if block_call else len(handles)  # a block call is one launch for all projections
     if model["bound"] == "tensor":
-        per_launch = model["flops_main"] / len(handles)
+        per_launch = model["flops_main"] / per_call
         achieved, peak, unit = per_launch / main_s / 1e12, peaks["bf16_tflops" if decode else "bf16_tflops_sustained"], "TFLOP/s"
     else:
-        per_launch = model["bytes_main"] / len(handles)
+        per_launch = model["bytes_main"] / per_call
         achieved, peak, unit = per_launch / main_s / 1e9, peaks["hbm_gbs"], "GB/s"
     roofline = {"bound": model["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(args.config), "kernel": "essa_decode_kernel (whole call)" if decode else "essa_tc_kernel<BLOCK_N, EPI_STORE> (base + up)",
+                "traffic": None if block_call else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc_kernel<BLOCK_N, EPI_STORE> (base + up)",
                 "peak_source": f"{peak_src} ({('burst bf16' if decode else 'sustained bf16') if unit == 'TFLOP/s' else 'copy'})",
                 "avg_launch_us": main_s * 1e6, "launches_timed": prof["calls"],
                 "rank_down_avg_us": prof["rank_down_ms"] * 1e3 / calls,
@@ -359,6 +364,8 @@ def run_ours(args, cfg):
                            "l2": "inputs larger than L2 (x, W0 and y of the projections exceed 126 MB per step)"
                                  if copies == 1 else f"weights rotate through {copies} device copies ({copies * w_bytes / 1e6:.0f} MB > 2 x L2): "
                                                      "every step streams W0 from HBM",
+                           "calls_per_step": "essa_sample_population + 1 x essa_apply_block" if block_call
+                                             else f"essa_sample_population + {len(handles)} x essa_apply_projection",
                            "parallelism": f"dp{world} (candidate-sharded, no data-path collective)"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
         print(json.dumps(line), flush=True)
@@ -380,6 +387,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--single-calls", action="store_true",
+                    help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]

@@ -51,6 +51,7 @@ extern "C" {
 #define ESSA_W0_INT8_PERCHANNEL 1 /* W0[o][i] = q[o][i] * scale[o], q int8, scale fp16 per out-channel */
 
 #define ESSA_MAX_RANK 64
+#define ESSA_MAX_BLOCK_ITEMS 4 /* projections one essa_apply_block call takes (q, k, v, o of an attention block) */
 #define ESSA_STATIC_MAX_TOKENS 4096 /* largest T essa_apply_projection_static accepts */
 
 typedef struct essa_ctx essa_ctx;         /* one per (process, device); not thread-safe */
@@ -137,6 +138,21 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
 int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* adapter, const void* x, int64_t T,
                               const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma,
                               int32_t sA_col, int32_t sB_col, void* y, void* stream);
+
+/* Several adapted projections over the SAME tokens, segments and singular-value table in one call: the q, k, v, o
+ * projections of an attention block ("Slice n" of Figure 1: one contiguous block of the table per LoRA matrix).
+ * The result is what n_items calls of essa_apply_projection give (item i reads x_i, writes y_i, uses columns
+ * sA_col_i / sB_col_i of the table).  At decode sizes (T <= 256, all items stored alike, W0 row tiles of the
+ * whole block within one wave of the GPU) the block runs as ONE kernel launch, which is where the time of such
+ * small calls goes; otherwise the items are issued one after the other.  1 <= n_items <= ESSA_MAX_BLOCK_ITEMS. */
+typedef struct essa_block_item {
+  const essa_adapter* adapter;
+  const void* x;           /* [T][d_in] bf16 dev (items may share one x)  */
+  int32_t sA_col, sB_col;  /* columns of this projection's sA / sB in the table */
+  void* y;                 /* [T][d_out] bf16 dev (written)               */
+} essa_block_item;
+int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T,
+                         const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma, void* stream);
 
 /* The same operation with HOST buffers: x, seg_offsets, sigma are copied to the device, the
  * projection runs, y is copied back, and the call returns after `stream` has been synchronised.

@@ -32,7 +32,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
-    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant",
+    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block",
 )
 
 
@@ -46,6 +46,10 @@ class AdapterDesc(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("rank", C.c_int32), ("w0_dtype", C.c_int32),
                 ("W0", C.c_void_p), ("w0_scale", C.c_void_p), ("U_A", C.c_void_p), ("V_A", C.c_void_p),
                 ("U_B", C.c_void_p), ("V_B", C.c_void_p), ("on_device", C.c_int32)]
+
+
+class BlockItem(C.Structure):
+    _fields_ = [("adapter", C.c_void_p), ("x", C.c_void_p), ("sA_col", C.c_int32), ("sB_col", C.c_int32), ("y", C.c_void_p)]
 
 
 class Plan(C.Structure):
@@ -84,6 +88,7 @@ def load_library() -> C.CDLL:
         "essa_reserve": (i32, [vp, i64, i32, i32]),
         "essa_get_launch_count": (i32, [vp, C.POINTER(i64)]),
         "essa_reserve_dequant": (i32, [vp, i32, i32]),
+        "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -252,6 +257,25 @@ class Context:
         """essa_apply_projection: y[T, d_out] bf16 (one launch at decode sizes, else rank-down then base + up)."""
         y = self._proj(self.lib.essa_apply_projection, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream)
         return y
+
+    def apply_block(self, adapters, xs, seg_offsets, sigma, cols, outs=None, stream=None):
+        """essa_apply_block: several projections over the same tokens / segments / sigma table in one call.
+
+        adapters, xs, cols (pairs (sA_col, sB_col)) and outs are parallel sequences; returns the list of outputs."""
+        torch = self.torch
+        T = xs[0].shape[0]
+        P = seg_offsets.numel() - 1
+        n = len(adapters)
+        if outs is None:
+            outs = [torch.empty((T, a.d_out), dtype=torch.bfloat16, device=self.device) for a in adapters]
+        arr = (BlockItem * n)()
+        for i in range(n):
+            arr[i] = BlockItem(adapters[i].handle, xs[i].data_ptr() if T else None, cols[i][0], cols[i][1],
+                               outs[i].data_ptr() if T else None)
+        st = self.lib.essa_apply_block(self.handle, arr, n, T, seg_offsets.data_ptr(), P, sigma.data_ptr(),
+                                       sigma.stride(0) if sigma.dim() == 2 else sigma.numel(), _stream(stream))
+        self._check(st)
+        return outs
 
     def apply_projection_static(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out, stream=None):
         """essa_apply_projection_static: same result as apply_projection without any device allocation.

@@ -143,12 +143,13 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
   else
     cudaGetLastError();
   if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_u, (size_t)kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
-      cudaMemset(ctx->dec_u, 0, (size_t)kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_cnt, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t)) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_ppart, (size_t)8 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_grp, (size_t)kDecodeMaxTokens * 2) != cudaSuccess ||
-      cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens * 2) != cudaSuccess) {
+      cudaMalloc(&ctx->dec_u, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMemset(ctx->dec_u, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_cnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_ppart, (size_t)ESSA_MAX_BLOCK_ITEMS * 8 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_grp, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2) != cudaSuccess ||
+      cudaMemset(ctx->dec_grp, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2) != cudaSuccess) {
     if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
     if (ctx->dec_grp) cudaFree(ctx->dec_grp);
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -198,9 +199,9 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     cudaMemset(ctx->d_status, 0, sizeof(int32_t));
     if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
     if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
-    cudaMemset(ctx->dec_cnt, 0, sizeof(uint32_t));
-    cudaMemset(ctx->dec_grp, 0, (size_t)kDecodeMaxTokens * 2);
-    ctx->dec_epoch = 0;
+    cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
+    cudaMemset(ctx->dec_grp, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2);
+    for (uint32_t& e : ctx->dec_epoch) e = 0;
   }
   return ESSA_OK;
 }
@@ -356,6 +357,44 @@ int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* 
   if (st != ESSA_OK || T == 0) return st;
   ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
   return launch_projection_tc(ctx, a, g, static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg,
+                         int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!items || n_items < 1 || n_items > ESSA_MAX_BLOCK_ITEMS)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_block: 1 .. ESSA_MAX_BLOCK_ITEMS items expected");
+  for (int32_t i = 0; i < n_items; ++i) {
+    const int32_t st = validate_projection_args(ctx, items[i].adapter, items[i].x, T, seg, P, sigma, ld_sigma,
+                                                items[i].sA_col, items[i].sB_col, items[i].y);
+    if (st != ESSA_OK) return st;
+  }
+  if (T == 0) return ESSA_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (T <= kDecodeMaxTokens) {
+    BlockItem bi[ESSA_MAX_BLOCK_ITEMS];
+    for (int32_t i = 0; i < n_items; ++i)
+      bi[i] = BlockItem{items[i].adapter, static_cast<const __nv_bfloat16*>(items[i].x), items[i].sA_col, items[i].sB_col,
+                        static_cast<__nv_bfloat16*>(items[i].y)};
+    cudaEvent_t* ev = nullptr;
+    if (ctx->prof_on) {
+      if ((size_t)(ctx->prof_calls + 1) * 3 <= ctx->prof_events.size()) ev = &ctx->prof_events[(size_t)ctx->prof_calls * 3];
+      else ++ctx->prof_dropped;
+    }
+    if (ev) { cudaEventRecord(ev[0], stream); cudaEventRecord(ev[1], stream); }
+    const int32_t st = launch_block_decode(ctx, bi, n_items, T, seg, P, sigma, ld_sigma, stream);
+    if (st != kBlockNotFused) {
+      if (ev) { cudaEventRecord(ev[2], stream); ++ctx->prof_calls; }
+      return st;
+    }
+  }
+  for (int32_t i = 0; i < n_items; ++i) {
+    ProjArgs g{static_cast<const __nv_bfloat16*>(items[i].x), T, seg, P, sigma, ld_sigma, items[i].sA_col, items[i].sB_col,
+               static_cast<__nv_bfloat16*>(items[i].y)};
+    const int32_t st = launch_projection_tc(ctx, items[i].adapter, g, stream);
+    if (st != ESSA_OK) return st;
+  }
+  return ESSA_OK;
 }
 
 // Allocation-free variant: see the comment above g_static_u in proj_tc.cu.

@@ -35,7 +35,7 @@ struct essa_ctx {
   // published so far (monotonic across calls; dec_epoch is the host's copy of where the next call starts)
   void* dec_u = nullptr;
   uint32_t* dec_cnt = nullptr;
-  uint32_t dec_epoch = 0;
+  uint32_t dec_epoch[ESSA_MAX_BLOCK_ITEMS] = {};  // (one buffer / counter set per projection of a block launch)
   void* dec_ppart = nullptr;    // [8][kDecodeMaxTokens][64] fp32: per-K-slice partial down-projections
   int* dec_grp = nullptr;       // [kDecodeMaxTokens / 4] arrival counters of the token groups (kept at zero)
   // Scratch owned by the context (grown on demand, never shrunk).
@@ -112,6 +112,15 @@ int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const 
 void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
                      essa_plan* out);
 // proj_decode.cu
+struct BlockItem {
+  const essa_adapter* a;
+  const __nv_bfloat16* x;
+  int32_t sA_col, sB_col;
+  __nv_bfloat16* y;
+};
+constexpr int32_t kBlockNotFused = 1;  // launch_block_decode: the block does not fit the one-wave decode schedule
+int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
+                            const float* sigma, int32_t ld_sigma, cudaStream_t stream);
 bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out);
 int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, const essa_plan& plan,
                                  cudaStream_t stream);

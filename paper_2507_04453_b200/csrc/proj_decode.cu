@@ -66,8 +66,6 @@ struct DParams {
   int vap_cols;
   int rank_groups;           // groups of kMaxRankTokens tokens
   int rank_slices;           // K slices per group; unit w = (group w / slices, slice w % slices)
-  int rank_ctas;             // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
-  int main_ctas;             // CTAs that stream W0 (m_tiles * splits); later CTAs of the grid only do rank units
   float* p_part;             // [8][256][64] fp32: partial down-projections, one slot per K slice
   int* grp_count;            // [128] arrivals per group (left at zero)
   const int32_t* seg;
@@ -79,6 +77,21 @@ struct DParams {
   uint32_t* u_count;         // rows published so far (monotonic across calls)
   uint32_t u_target;         // value of *u_count once this call's T rows are in
   int32_t* status;
+};
+
+// A launch covers up to kMaxBlockProj projections that share the tokens, segments and singular-value table (the
+// q, k, v, o of an attention block): each has its own parameter set and tensor maps; CTAs
+// cta_begin[i] .. cta_begin[i+1]-1 stream projection i's W0, rank-path units unit_begin[i] .. belong to it.
+constexpr int kMaxBlockProj = ESSA_MAX_BLOCK_ITEMS;
+struct DBlock {
+  int n_proj;
+  int cta_begin[kMaxBlockProj + 1];   // multiples of the cluster size; cta_begin[n_proj] = W0-streaming CTAs
+  int unit_begin[kMaxBlockProj + 1];  // rank-path units (token group x K slice) per projection
+  int rank_ctas;                      // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
+  DParams proj[kMaxBlockProj];
+};
+struct DMaps {
+  CUtensorMap tm[kMaxBlockProj][5];   // per projection: W0, x, u, U_B slab 0, U_B slab 1
 };
 
 // tokens of the receive buffer each CTA of a cluster of `splits` owns: a multiple of 16 so that a 16-token
@@ -269,9 +282,16 @@ __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, 
 
 template <bool INT8>
 __global__ void __launch_bounds__(INT8 ? kDecThreadsInt8 : kDecThreads, 1)
-essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                   const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmUB0,
-                   const __grid_constant__ CUtensorMap tmUB1, const DParams p) {
+essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ DBlock blk) {
+  // which projection this CTA streams (CTAs past the last one only take rank-path units)
+  int pi = 0;
+  while (pi + 1 < blk.n_proj && (int)blockIdx.x >= blk.cta_begin[pi + 1]) ++pi;
+  const DParams& p = blk.proj[pi];
+  const CUtensorMap& tmW = maps.tm[pi][0];
+  const CUtensorMap& tmX = maps.tm[pi][1];
+  const CUtensorMap& tmU = maps.tm[pi][2];
+  const CUtensorMap& tmUB0 = maps.tm[pi][3];
+  const CUtensorMap& tmUB1 = maps.tm[pi][4];
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
@@ -298,8 +318,8 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = (int)cluster_ctarank();
-  const bool is_main = (int)blockIdx.x < p.main_ctas;  // later CTAs of the grid only take rank-path units
-  const int m_tile = blockIdx.x / p.splits;
+  const bool is_main = (int)blockIdx.x < blk.cta_begin[blk.n_proj];  // later CTAs of the grid only take rank-path units
+  const int m_tile = ((int)blockIdx.x - blk.cta_begin[pi]) / p.splits;
   // this CTA's K blocks [kb0, kb1)
   const int kbase = p.main_kb / p.splits, krem = p.main_kb % p.splits;
   const int kb0 = split * kbase + min(split, krem);
@@ -547,15 +567,19 @@ essa_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   int got = 0;
   if (epi) {
     const int etid = threadIdx.x - 64;
-    if ((int)blockIdx.x < p.rank_ctas) {
-      // this CTA's units of the rank path, while its K loop streams
+    if ((int)blockIdx.x < blk.rank_ctas) {
+      // this CTA's units of the rank path (of any projection of the block), while its K loop streams
       volatile int* flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
-      for (int unit = blockIdx.x; unit < p.rank_groups * p.rank_slices; unit += p.rank_ctas) {
-        const int grp = unit / p.rank_slices, slice = unit % p.rank_slices;
-        switch (p.vap_cols) {
-          case 16: rank_unit<16>(p, grp, slice, red, qbuf, flag, etid); break;
-          case 32: rank_unit<32>(p, grp, slice, red, qbuf, flag, etid); break;
-          default: rank_unit<64>(p, grp, slice, red, qbuf, flag, etid); break;
+      for (int unit = blockIdx.x; unit < blk.unit_begin[blk.n_proj]; unit += blk.rank_ctas) {
+        int pj = 0;
+        while (pj + 1 < blk.n_proj && unit >= blk.unit_begin[pj + 1]) ++pj;
+        const DParams& pr = blk.proj[pj];
+        const int local = unit - blk.unit_begin[pj];
+        const int grp = local / pr.rank_slices, slice = local % pr.rank_slices;
+        switch (pr.vap_cols) {
+          case 16: rank_unit<16>(pr, grp, slice, red, qbuf, flag, etid); break;
+          case 32: rank_unit<32>(pr, grp, slice, red, qbuf, flag, etid); break;
+          default: rank_unit<64>(pr, grp, slice, red, qbuf, flag, etid); break;
         }
       }
     }
@@ -635,50 +659,62 @@ inline int dec_smem_bytes(int w_stages, int c_stages, int x_stages, int tn) {
 
 }  // namespace
 
-// Schedule of the decode kernel for T tokens; returns false when the call should use the prefill kernels.
-bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out) {
-  if (T <= 0 || T > kDecodeMaxTokens) return false;
-  (void)rank;
+// Schedule shared by the projections of one decode launch (n of them, sizes d_in[i] -> d_out[i], same storage type):
+// cluster size, ring depths.  Returns false when the launch would not fit one wave of the GPU.
+static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int8, int64_t T, int sm_count, int* splits_out,
+                              int* w_stages_out, int* x_stages_out, int* m_tiles_total_out) {
+  if (T <= 0 || T > kDecodeMaxTokens || n < 1 || n > kMaxBlockProj) return false;
   const int sm = sm_count > 0 ? sm_count : 148;
-  const int ext = (w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? 2 : 1;
   const int tn = (int)((T + 15) / 16) * 16;
-  const int m_tiles = (d_out + DEC_M - 1) / DEC_M;
-  const int main_kb = d_in / DEC_K;
-  // cluster size: a power of two (packs into a GPC's SMs without stragglers), at most 8 (portable limit)
+  int m_total = 0, min_kb = 1 << 30;
+  for (int i = 0; i < n; ++i) {
+    m_total += (d_out[i] + DEC_M - 1) / DEC_M;
+    if (d_in[i] / DEC_K < min_kb) min_kb = d_in[i] / DEC_K;
+  }
+  // cluster size: a power of two (packs into a GPC's SMs without stragglers), at most 8 (portable limit).
   // All clusters must be resident at once (the CTAs that add the rank term wait for rows other CTAs publish, and
   // a second wave would double the time anyway).  With one CTA per SM, clusters of 4 fill about 132 of 148 SMs
   // and clusters of 8 about 120 (they may not straddle GPCs).
   auto resident = [&](int c) { return c >= 8 ? sm * 120 / 148 : c >= 4 ? sm * 132 / 148 : sm; };
+  if (n > 1 && m_total > resident(1)) return false;
   int splits = 1;
-  while (splits * 2 <= 8 && m_tiles * splits * 2 <= resident(splits * 2) && splits * 2 <= main_kb) splits *= 2;
-  const int kb_per = (main_kb + splits - 1) / splits;
+  while (splits * 2 <= 8 && m_total * splits * 2 <= resident(splits * 2) && splits * 2 <= min_kb) splits *= 2;
   // Ring depths.  Per K block the tensor core needs ~560 cycles; a tile load takes ~2500 (L2) to ~4000 (HBM)
   // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
   // INT8 storage: W0 tiles travel as 8 KB of codes; a ring of converted bf16 tiles (which also takes the U_B slabs,
   // loaded into it directly) sits between the converting warps and the tensor core.
-  const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   const int c_stages = int8 ? kInt8ConvStages : 0;
   const int w_slot = int8 ? RAW_TILE_BYTES : W_TILE_BYTES;
-  const int n_w_items = int8 ? kb_per : kb_per + ext;
   const int xb = tn * 128;
   const int budget = kDecSmemBudget - dec_smem_bytes(0, c_stages, 0, tn);
   int x_stages = budget / (w_slot + xb);
   if (x_stages > kMaxXStages) x_stages = kMaxXStages;
-  if (x_stages > kb_per + 1) x_stages = kb_per + 1;
   if (x_stages < 1) return false;
   int w_stages = (budget - x_stages * xb) / w_slot;
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
-  if (w_stages > n_w_items) w_stages = n_w_items;
   if (w_stages < 1) return false;
   // the receive buffer of the cluster reduction overlays the rings
-  while (dec_ring_bytes(w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) ++w_stages;
-  if (w_stages > kMaxWStages || dec_smem_bytes(w_stages, c_stages, x_stages, tn) > kDecSmemBudget) return false;
+  if (dec_ring_bytes(w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) return false;
+  *splits_out = splits;
+  *w_stages_out = w_stages;
+  *x_stages_out = x_stages;
+  *m_tiles_total_out = m_total;
+  return true;
+}
+
+// Schedule of the decode kernel for one projection of T tokens; returns false when the call should use the prefill kernels.
+bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out) {
+  (void)rank;
+  const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  int splits, w_stages, x_stages, m_tiles;
+  const int di = d_in, dout = d_out;
+  if (!plan_decode_block(1, &di, &dout, int8, T, sm_count, &splits, &w_stages, &x_stages, &m_tiles)) return false;
   out->block_m = DEC_M;
-  out->block_n = tn;
+  out->block_n = (int)((T + 15) / 16) * 16;
   out->block_k = DEC_K;
   out->stages = w_stages;
   out->x_stages = x_stages;
-  out->k_blocks = main_kb + ext;
+  out->k_blocks = d_in / DEC_K + (int8 ? 2 : 1);
   out->splits = splits;
   out->tiles = m_tiles;
   out->grid = m_tiles * splits;
@@ -689,102 +725,130 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
   return true;
 }
 
-int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, const essa_plan& pl,
-                                 cudaStream_t stream) {
-  DParams p{};
-  p.T = (int)g.T;
-  p.tn = pl.block_n;
-  p.xbox = (p.tn % 64 == 0) ? 64 : p.tn;
-  p.d_in = a->d_in;
-  p.d_out = a->d_out;
-  p.main_kb = a->d_in / DEC_K;
-  p.m_tiles = (a->d_out + DEC_M - 1) / DEC_M;
-  p.splits = pl.splits;
-  const bool int8 = a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
-  p.w_stages = pl.stages;
-  p.x_stages = pl.x_stages;
-  p.c_stages = int8 ? kInt8ConvStages : 0;
-  p.ext = a->ext_blocks;
-  p.y = g.y;
-  p.ldy = a->d_out;
-  p.scale = int8 ? a->w0_scale : nullptr;
-  p.x = g.x;
-  p.VAp = a->VAp;
-  p.vap_cols = a->vap_cols;
-  // rank path: spread the tokens over the CTAs of the grid, a few tokens each (more per CTA for wide ranks,
-  // whose V_A is large enough that re-reading it per token would crowd L2)
-  const int grid = p.m_tiles * p.splits;
+// One launch for n projections that share tokens, segments and the singular-value table.  Returns ESSA_OK, an
+// error, or kBlockNotFused (> 0) when the block does not fit the one-wave decode schedule and the caller should
+// issue the projections one by one.
+int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
+                            const float* sigma, int32_t ld_sigma, cudaStream_t stream) {
+  if (n < 1 || n > kMaxBlockProj || T <= 0 || T > kDecodeMaxTokens) return kBlockNotFused;
+  const bool int8 = items[0].a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  int d_in[kMaxBlockProj], d_out[kMaxBlockProj];
+  for (int i = 0; i < n; ++i) {
+    if ((items[i].a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) != int8) return kBlockNotFused;
+    d_in[i] = items[i].a->d_in;
+    d_out[i] = items[i].a->d_out;
+  }
+  int splits, w_stages, x_stages, m_total;
+  if (!plan_decode_block(n, d_in, d_out, int8, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total)) {
+    if (n > 1) return kBlockNotFused;
+    return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: no decode schedule fits shared memory");
+  }
+  const int tn = (int)((T + 15) / 16) * 16;
+  const int c_stages = int8 ? kInt8ConvStages : 0;
+
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
   static int resident_caches[64][2][9] = {};  // per device, storage type, cluster size
   int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][int8 ? 1 : 0];
   const void* kernel = int8 ? (const void*)essa_decode_kernel<true> : (const void*)essa_decode_kernel<false>;
   const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
   {
-    const int smem_q = kDecSmemBudget;
-    if (resident_cache[p.splits] == 0) {
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
-      cudaLaunchConfig_t q{};
-      q.gridDim = dim3((unsigned)(148 * p.splits), 1, 1);
-      q.blockDim = dim3((unsigned)threads, 1, 1);
-      q.dynamicSmemBytes = (size_t)smem_q;
-      cudaLaunchAttribute qa[1];
-      qa[0].id = cudaLaunchAttributeClusterDimension;
-      qa[0].val.clusterDim.x = (unsigned)p.splits;
-      qa[0].val.clusterDim.y = 1;
-      qa[0].val.clusterDim.z = 1;
-      q.attrs = qa;
-      q.numAttrs = 1;
-      int n_clusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &q) != cudaSuccess || n_clusters <= 0) {
-        cudaGetLastError();
-        n_clusters = 1;  // unknown: only the first cluster is certainly in the first wave
-      }
-      resident_cache[p.splits] = n_clusters;
-    }
-  }
-  // Launch a full wave: the CTAs beyond the W0-streaming ones only take rank-path units.  A unit is a group of
-  // 4 tokens (2 for ranks above 32) over one K slice; slices multiply the units until the wave is busy (at most 8).
-  const int resident_ctas = resident_cache[p.splits] * p.splits;
-  const int grid_total = grid > resident_ctas ? grid : resident_ctas;
-  p.main_ctas = grid;
-  p.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
-  const int gtok = rank_group_tokens(a->vap_cols);
-  p.rank_groups = (p.T + gtok - 1) / gtok;
-  int slices = p.rank_ctas / p.rank_groups;
-  if (slices > 8) slices = 8;
-  if (slices > a->d_in / 512) slices = a->d_in / 512;  // at least 64 row blocks per slice
-  if (slices < 1) slices = 1;
-  p.rank_slices = slices;
-  p.p_part = static_cast<float*>(ctx->dec_ppart);
-  p.grp_count = ctx->dec_grp;
-  p.seg = g.seg_offsets;
-  p.P = g.P;
-  p.sigma = g.sigma;
-  p.ld_sigma = g.ld_sigma;
-  p.sA_col = g.sA_col;
-  p.sB_col = g.sB_col;
-  p.r = a->rank;
-  p.M = a->M;
-  p.u = static_cast<__nv_bfloat16*>(ctx->dec_u);
-  p.u_count = ctx->dec_cnt;
-  ctx->dec_epoch += (uint32_t)p.T;
-  p.u_target = ctx->dec_epoch;
-  p.status = ctx->d_status;
-
-  CUtensorMap tm_x, tm_u;
-  int32_t st = make_tensor_map_2d(ctx, &tm_x, 0, g.x, (uint64_t)g.T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
-                                  (uint32_t)p.xbox, DEC_K, 128);
-  if (st != ESSA_OK) return st;
-  st = make_tensor_map_2d(ctx, &tm_u, 0, ctx->dec_u, (uint64_t)kDecodeMaxTokens, kRankPadMax, kRankPadMax * 2,
-                          (uint32_t)p.xbox, DEC_K, 128);
-  if (st != ESSA_OK) return st;
-  const int smem_bytes = dec_smem_bytes(p.w_stages, p.c_stages, p.x_stages, p.tn);
-  if (smem_bytes > kDecSmemBudget || p.w_stages > kMaxWStages || p.x_stages > kMaxXStages)
-    return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: decode schedule exceeds shared memory");
-  {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
   }
+  if (resident_cache[splits] == 0) {
+    cudaLaunchConfig_t q{};
+    q.gridDim = dim3((unsigned)(148 * splits), 1, 1);
+    q.blockDim = dim3((unsigned)threads, 1, 1);
+    q.dynamicSmemBytes = (size_t)kDecSmemBudget;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = (unsigned)splits;
+    qa[0].val.clusterDim.y = 1;
+    qa[0].val.clusterDim.z = 1;
+    q.attrs = qa;
+    q.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &q) != cudaSuccess || n_clusters <= 0) {
+      cudaGetLastError();
+      n_clusters = 1;  // unknown: only the first cluster is certainly in the first wave
+    }
+    resident_cache[splits] = n_clusters;
+  }
+  const int resident_ctas = resident_cache[splits] * splits;
+  const int main_ctas = m_total * splits;
+  if (n > 1 && main_ctas > resident_ctas) return kBlockNotFused;
+  // Launch a full wave: the CTAs beyond the W0-streaming ones only take rank-path units.  A unit is a group of
+  // 4 tokens (2 for ranks above 32) over one K slice; slices multiply the units until the wave is busy (at most 8).
+  const int grid_total = main_ctas > resident_ctas ? main_ctas : resident_ctas;
+
+  DBlock blk{};
+  DMaps maps{};
+  blk.n_proj = n;
+  blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
+  int groups_total = 0;
+  for (int i = 0; i < n; ++i) groups_total += ((int)T + rank_group_tokens(items[i].a->vap_cols) - 1) / rank_group_tokens(items[i].a->vap_cols);
+  int cta = 0, unit = 0;
+  for (int i = 0; i < n; ++i) {
+    const essa_adapter* a = items[i].a;
+    DParams& p = blk.proj[i];
+    p.T = (int)T;
+    p.tn = tn;
+    p.xbox = (tn % 64 == 0) ? 64 : tn;
+    p.d_in = a->d_in;
+    p.d_out = a->d_out;
+    p.main_kb = a->d_in / DEC_K;
+    p.m_tiles = (a->d_out + DEC_M - 1) / DEC_M;
+    p.splits = splits;
+    p.w_stages = w_stages;
+    p.x_stages = x_stages;
+    p.c_stages = c_stages;
+    p.ext = a->ext_blocks;
+    p.y = items[i].y;
+    p.ldy = a->d_out;
+    p.scale = int8 ? a->w0_scale : nullptr;
+    p.x = items[i].x;
+    p.VAp = a->VAp;
+    p.vap_cols = a->vap_cols;
+    const int gtok = rank_group_tokens(a->vap_cols);
+    p.rank_groups = ((int)T + gtok - 1) / gtok;
+    int slices = blk.rank_ctas / groups_total;
+    if (slices > 8) slices = 8;
+    if (slices > a->d_in / 512) slices = a->d_in / 512;  // at least 64 row blocks per slice
+    if (slices < 1) slices = 1;
+    p.rank_slices = slices;
+    p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)i * 8 * kDecodeMaxTokens * kRankPadMax;
+    p.grp_count = ctx->dec_grp + i * (kDecodeMaxTokens / 2);
+    p.seg = seg;
+    p.P = P;
+    p.sigma = sigma;
+    p.ld_sigma = ld_sigma;
+    p.sA_col = items[i].sA_col;
+    p.sB_col = items[i].sB_col;
+    p.r = a->rank;
+    p.M = a->M;
+    p.u = static_cast<__nv_bfloat16*>(ctx->dec_u) + (size_t)i * kDecodeMaxTokens * kRankPadMax;
+    p.u_count = ctx->dec_cnt + i;
+    ctx->dec_epoch[i] += (uint32_t)T;
+    p.u_target = ctx->dec_epoch[i];
+    p.status = ctx->d_status;
+    blk.cta_begin[i] = cta;
+    blk.unit_begin[i] = unit;
+    cta += p.m_tiles * splits;
+    unit += p.rank_groups * p.rank_slices;
+
+    maps.tm[i][0] = int8 ? a->tm_W0q : a->tm_W0[0];  // 64-row boxes of bf16 W0 / 128-row boxes of codes
+    int32_t st = make_tensor_map_2d(ctx, &maps.tm[i][1], 0, items[i].x, (uint64_t)T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
+                                    (uint32_t)p.xbox, DEC_K, 128);
+    if (st != ESSA_OK) return st;
+    st = make_tensor_map_2d(ctx, &maps.tm[i][2], 0, p.u, (uint64_t)kDecodeMaxTokens, kRankPadMax, kRankPadMax * 2,
+                            (uint32_t)p.xbox, DEC_K, 128);
+    if (st != ESSA_OK) return st;
+    maps.tm[i][3] = a->tm_UBp[0][0];  // 64-row boxes of the U_B slabs
+    maps.tm[i][4] = a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0];
+  }
+  for (int i = n; i <= kMaxBlockProj; ++i) { blk.cta_begin[i] = cta; blk.unit_begin[i] = unit; }
+
+  const int smem_bytes = dec_smem_bytes(w_stages, c_stages, x_stages, tn);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid_total, 1, 1);
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
@@ -792,17 +856,23 @@ int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const Pro
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)p.splits;
+  attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   ctx->launches += 1;
-  const CUtensorMap& tmU0 = a->tm_UBp[0][0];  // 64-row boxes of the U_B slabs
-  const CUtensorMap& tmU1 = a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0];
-  const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, a->tm_W0q, tm_x, tm_u, tmU0, tmU1, p)
-                             : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, a->tm_W0[0], tm_x, tm_u, tmU0, tmU1, p);
+  const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, maps, blk)
+                             : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, maps, blk);
   return check_cuda(ctx, e, "essa_decode_kernel launch");
+}
+
+int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, const essa_plan& pl,
+                                 cudaStream_t stream) {
+  (void)pl;
+  const BlockItem item{a, g.x, g.sA_col, g.sB_col, g.y};
+  const int32_t st = launch_block_decode(ctx, &item, 1, g.T, g.seg_offsets, g.P, g.sigma, g.ld_sigma, stream);
+  return st == kBlockNotFused ? fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: no decode schedule for this call") : st;
 }
 
 }  // namespace essa

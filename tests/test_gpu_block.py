@@ -1,0 +1,97 @@
+"""GPU parity of essa_apply_block (the q, k, v, o projections of a block in one call) against the CPU oracle.
+
+At decode sizes the block runs as one launch of the decode kernel; otherwise it degrades to one call per
+projection.  Either way every projection's output must match the oracle like a single call does.
+"""
+import numpy as np
+import pytest
+
+from oracle import essa_oracle as orc
+from paper_2507_04453_b200 import binding, workloads as wl
+from tests.parity_utils import TOL_BF16, TOL_INT8, Case, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("CUDA device required for -m gpu tests")
+    return torch
+
+
+@pytest.fixture(scope="module")
+def ctx(torch):
+    c = binding.Context(0)
+    yield c
+    assert c.get_status() == 0, "a kernel recorded a device-side error"
+    c.close()
+
+
+def _block(torch, ctx, case, candidates=None):
+    cfg = case.cfg
+    n = len(cfg.projections)
+    xs_host = [case.tokens(i) for i in range(n)]
+    xs = [to_dev(torch, x, torch.bfloat16) for x in xs_host]
+    cols = [cfg.sigma_cols(i) for i in range(n)]
+    launches0 = ctx.gpu_launches
+    ys = ctx.apply_block([case.handles[i] for i in range(n)], xs, case.d_offsets, case.d_sigma, cols)
+    torch.cuda.synchronize()
+    launches = ctx.gpu_launches - launches0
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    for i in range(n):
+        got = ys[i].float().cpu().numpy()
+        want = case.oracle_projection(i, xs_host[i], candidates)
+        assert np.isfinite(got).all()
+        err = orc.relative_error(got, want)
+        assert err <= tol, (cfg.name, cfg.projections[i], err)
+    return launches, xs, ys
+
+
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 1024, 192, 16, 256, 1),      # decode block, bf16: one launch
+                                               ("5a", 1024, 256, 64, 128, 1),     # decode block, INT8, rank 64
+                                               ("4", 512, 128, 32, 9, 20),        # ragged segments, T = sum L_k <= 180
+                                               ("2", 256, 64, 16, 3, 100)])       # T = 300: prefill sizes, one call each
+def test_block_matches_oracle(torch, ctx, base, dm, dkv, r, P, L):
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    launches, _, _ = _block(torch, ctx, case)
+    if case.T <= 256:
+        assert launches == 1, "a decode-sized block is one kernel launch"
+    else:
+        assert launches == 2 * len(cfg.projections)
+    case.close()
+
+
+def test_block_equals_single_calls_in_structure_and_is_deterministic(torch, ctx):
+    """Same inputs, two block calls: bit-identical (the cluster reduction and the rank path sum in fixed order)."""
+    cfg = wl.scaled_config("3", d_model=2048, d_kv=256, rank=16, P=200, seg_len=1)
+    case = Case(torch, ctx, cfg)
+    _, xs, ys = _block(torch, ctx, case)
+    first = [y.clone() for y in ys]
+    cols = [cfg.sigma_cols(i) for i in range(4)]
+    for _ in range(3):
+        again = ctx.apply_block([case.handles[i] for i in range(4)], xs, case.d_offsets, case.d_sigma, cols)
+        for a, b in zip(first, again):
+            assert torch.equal(a, b)
+    # single calls take another split of the reduction, so they agree to rounding, not bit for bit
+    for i in range(4):
+        single = ctx.apply_projection(case.handles[i], xs[i], case.d_offsets, case.d_sigma, *cols[i])
+        assert orc.relative_error(first[i].float().cpu().numpy(), single.float().cpu().numpy().astype(np.float64)) <= TOL_BF16
+    case.close()
+
+
+@pytest.mark.parametrize("name,max_cands", [("3", 24), ("5a", 12)])
+def test_block_full_size(torch, ctx, name, max_cands):
+    """The benchmark's decode configurations through the block call, in the launch configuration bench.py times."""
+    cfg = wl.CONFIGS[name]
+    case = Case(torch, ctx, cfg)
+    cands = wl.stratified_candidates(cfg, case.offsets)[:max_cands]
+    launches, xs, ys = _block(torch, ctx, case, cands)
+    assert launches == 1
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    for i in range(4):  # every element against the CUDA-core path
+        ref = ctx.apply_projection_simt(case.handles[i], xs[i], case.d_offsets, case.d_sigma, *cfg.sigma_cols(i))
+        assert orc.relative_error(ys[i].float().cpu().numpy(), ref.float().cpu().numpy().astype(np.float64)) <= tol
+    case.close()
