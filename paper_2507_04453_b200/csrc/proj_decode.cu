@@ -280,6 +280,37 @@ __device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, 
   epi_bar_sync();  // red / qbuf / flag may be reused
 }
 
+// Sum token rows j0, j0 + 4, ... < j_end of this CTA's slice over the NS receive slots (cluster rank order:
+// deterministic), scale, round to bf16, store; four tokens per pass so that their loads overlap.
+// recv layout: [slot][per][128 channels] fp32; each thread owns 4 consecutive channels.
+template <int NS>
+__device__ __forceinline__ void sum_store(const float* mine, int per, int j0, int j_end, const float (&sc)[4],
+                                          __nv_bfloat16* yrow0, int ldy) {
+  for (int j = j0; j < j_end; j += 16) {
+    float4 acc[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int jj = min(j + 4 * u, j_end - 1);  // clamped rows are loaded twice and stored once
+      acc[u] = *reinterpret_cast<const float4*>(mine + (size_t)jj * DEC_M);
+#pragma unroll
+      for (int r = 1; r < NS; ++r) {
+        const float4 v = *reinterpret_cast<const float4*>(mine + ((size_t)r * per + jj) * DEC_M);
+        acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int jj = j + 4 * u;
+      if (jj < j_end) {
+        uint2 o;
+        o.x = pack_bf16x2(acc[u].x * sc[0], acc[u].y * sc[1]);
+        o.y = pack_bf16x2(acc[u].z * sc[2], acc[u].w * sc[3]);
+        *reinterpret_cast<uint2*>(yrow0 + (size_t)jj * ldy) = o;
+      }
+    }
+  }
+}
+
 template <bool INT8>
 __global__ void __launch_bounds__(INT8 ? kDecThreadsInt8 : kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ DBlock blk) {
@@ -629,16 +660,12 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       }
       const float* mine = recv + 4 * lane;
       __nv_bfloat16* yrow0 = p.y + (size_t)t0 * p.ldy + ch0;
-      for (int j = ew; j < j_lim; j += 4) {
-        float4 acc = *reinterpret_cast<const float4*>(mine + (size_t)j * DEC_M);
-        for (int r = 1; r < p.splits; ++r) {  // cluster rank order: deterministic
-          const float4 v = *reinterpret_cast<const float4*>(mine + ((size_t)r * per + j) * DEC_M);
-          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        uint2 o;
-        o.x = pack_bf16x2(acc.x * sc[0], acc.y * sc[1]);
-        o.y = pack_bf16x2(acc.z * sc[2], acc.w * sc[3]);
-        *reinterpret_cast<uint2*>(yrow0 + (size_t)j * p.ldy) = o;
+      const int ldy = p.ldy;
+      switch (p.splits) {
+        case 1: sum_store<1>(mine, per, ew, j_lim, sc, yrow0, ldy); break;
+        case 2: sum_store<2>(mine, per, ew, j_lim, sc, yrow0, ldy); break;
+        case 4: sum_store<4>(mine, per, ew, j_lim, sc, yrow0, ldy); break;
+        default: sum_store<8>(mine, per, ew, j_lim, sc, yrow0, ldy); break;
       }
     }
   }
