@@ -228,6 +228,8 @@ def run_ours(args, cfg):
     peaks, peak_src = load_peaks()
 
     ctx = binding.Context(local_rank)
+    if args.pair_tiles >= 0:
+        ctx.set_option(binding.ESSA_OPT_PAIR_TILES, args.pair_tiles)
     adapters = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
     offsets = wl.make_segments(cfg)
     T = int(offsets[-1])
@@ -387,6 +389,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pair-tiles", type=int, default=-1, help="override ESSA_OPT_PAIR_TILES (0 / 1)")
     ap.add_argument("--single-calls", action="store_true",
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")

@@ -72,6 +72,11 @@ const char* essa_last_error(essa_ctx* ctx);
 /* Synchronise the device, then read (and clear) the device status word: 0, or the ESSA_ERR_* code a
  * kernel recorded (ESSA_ERR_DEVICE_TIMEOUT if a bounded wait ran out; the affected output is undefined). */
 int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
+/* Scheduling options of a context.
+ *   ESSA_OPT_PAIR_TILES (0 / 1): run the base + up step of prefill-sized calls (T >= 512, 256-channel tiles) on
+ *   256-token x 256-channel tiles shared by pairs of CTAs (tcgen05 cta_group::2) instead of 128 x 256 tiles per CTA. */
+#define ESSA_OPT_PAIR_TILES 1
+int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);
 /* Pre-size the context's scratch memory (rank-path buffer, split-K workspace, host-call staging) for

@@ -25,6 +25,7 @@ ESSA_ERR_DEVICE_TIMEOUT = -5
 ESSA_ERR_NO_DEVICE = -6
 ESSA_W0_BF16 = 0
 ESSA_W0_INT8_PERCHANNEL = 1
+ESSA_OPT_PAIR_TILES = 1
 
 EXPORTED_SYMBOLS = (
     "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",
@@ -32,7 +33,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
-    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block",
+    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_set_option",
 )
 
 
@@ -88,6 +89,7 @@ def load_library() -> C.CDLL:
         "essa_reserve": (i32, [vp, i64, i32, i32]),
         "essa_get_launch_count": (i32, [vp, C.POINTER(i64)]),
         "essa_reserve_dequant": (i32, [vp, i32, i32]),
+        "essa_set_option": (i32, [vp, i32, i32]),
         "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
@@ -190,6 +192,10 @@ class Context:
 
     def reserve(self, max_tokens: int, max_d_in: int, max_d_out: int):
         self._check(self.lib.essa_reserve(self.handle, max_tokens, max_d_in, max_d_out))
+
+    def set_option(self, option: int, value: int):
+        """essa_set_option (ESSA_OPT_PAIR_TILES = 1)."""
+        self._check(self.lib.essa_set_option(self.handle, option, value))
 
     def reserve_dequant(self, max_d_in: int, max_d_out: int):
         """essa_reserve_dequant: pre-size the scratch that prefill calls on INT8-stored adapters dequantise into."""

@@ -206,6 +206,14 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
   return ESSA_OK;
 }
 
+int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  switch (option) {
+    case ESSA_OPT_PAIR_TILES: ctx->pair_tiles = value != 0; return ESSA_OK;
+    default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
+  }
+}
+
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches) {
   if (!ctx || !launches) return ESSA_ERR_INVALID_ARG;
   *launches = ctx->launches;

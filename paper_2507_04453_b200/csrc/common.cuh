@@ -31,6 +31,7 @@ struct essa_ctx {
   std::string last_error;
   int32_t* d_status = nullptr;  // device status word
   int64_t launches = 0;         // kernels of this library enqueued through this context
+  bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
   // decode schedule: rank-path vector u of one call, [kDecodeMaxTokens][64] bf16, and the count of rows
   // published so far (monotonic across calls; dec_epoch is the host's copy of where the next call starts)
   void* dec_u = nullptr;
@@ -111,6 +112,10 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
 int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, cudaStream_t stream);
 void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
                      essa_plan* out);
+// proj_tc2.cu
+int32_t launch_base_up_pair(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2,
+                            const CUtensorMap& tmB2a, const CUtensorMap& tmB2b, int T, int d_out, int main_kb, int ext_kb,
+                            int ext_ksteps, __nv_bfloat16* y, const __half* scale, cudaStream_t stream);
 // proj_decode.cu
 struct BlockItem {
   const essa_adapter* a;

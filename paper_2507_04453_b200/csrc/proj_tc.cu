@@ -535,6 +535,8 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     else ++ctx->prof_dropped;
   }
   if (ev) cudaEventRecord(ev[0], stream);
+  // large prefill calls run base + up on 256 x 256 CTA-pair tiles
+  const bool use_pairs = ctx->pair_tiles && pl.block_n == 256 && pl.splits == 1 && g.T >= 512;
 
   // ---- INT8 storage: dequantise the codes (unscaled, exact) into the context's scratch for this call's GEMM
   CUtensorMap tm_wdeq;
@@ -545,7 +547,7 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     st = launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr), cnt, stream);
     if (st != ESSA_OK) return st;
     st = make_tensor_map_2d(ctx, &tm_wdeq, 0, ctx->w_deq.ptr, (uint64_t)a->d_out, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
-                            (uint32_t)pl.block_n, BLOCK_K, 128);
+                            (uint32_t)(use_pairs ? 128 : pl.block_n), BLOCK_K, 128);
     if (st != ESSA_OK) return st;
   }
 
@@ -597,6 +599,13 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   mp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
   mp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
   mp.status = ctx->d_status;
+  if (use_pairs) {
+    const CUtensorMap& tmW128 = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? tm_wdeq : a->tm_W0[1];
+    st = launch_base_up_pair(ctx, tm_x, tmW128, tm_u, a->tm_UBp[1][0], a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0], (int)g.T,
+                             a->d_out, a->d_in / BLOCK_K, a->ext_blocks, a->r_pad / UMMA_K, g.y, mp.scale, stream);
+    if (ev) cudaEventRecord(ev[2], stream);
+    return st;
+  }
   const int bi = pl.block_n == 64 ? 0 : pl.block_n == 128 ? 1 : 2;
   const CUtensorMap& tmW = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? tm_wdeq : a->tm_W0[bi];
   const CUtensorMap& tmU0 = a->tm_UBp[bi][0];
