@@ -61,52 +61,93 @@ __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, c
 }
 
 // Full covariance factor.  blockIdx.x = group of kCand candidates, blockIdx.y = tile of kRows rows of Bfactor.
-// Phase 1: w[c][j] = Dvec[j] * z_c[j] into shared memory.  Phase 2: one warp per row i, lanes stride over j,
-// shuffle reduction; lane 0 writes mean[i] + step * acc.
+// Phase 1: w[c][j] = Dvec[j] * z_c[j] into shared memory (every block regenerates its candidates' normals).
+// Phase 2: a warp owns eight rows at once: lane = 4 * row + quarter, each quarter of a row's lanes strides over
+// the columns (16-byte loads when the rows are 16-byte aligned), so a row's sum is finished by two shuffle steps
+// and all eight rows' loads are in flight together; the quarter-0 lane writes mean[i] + step * acc.
 constexpr int kCand = 4, kRows = 64, kSamplerThreads = 256;
 
+template <bool VEC>
 __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const float* __restrict__ mean, float step,
                                                                       const float* __restrict__ Bfactor,
                                                                       const float* __restrict__ Dvec, int d, uint2 key,
                                                                       int k_begin, int k_count,
                                                                       float* __restrict__ sigma_out) {
-  extern __shared__ double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
+  extern __shared__ __align__(16) double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
   const int nb = (d + 3) >> 2, d4 = nb * 4;
   const int kk0 = blockIdx.x * kCand;
-  for (int idx = threadIdx.x; idx < kCand * nb; idx += blockDim.x) {
-    const int c = idx / nb, j = idx % nb;
-    double zz[4] = {0.0, 0.0, 0.0, 0.0};
-    if (kk0 + c < k_count) normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk0 + c), zz);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = lane >> 2, q = lane & 3;
+  const int i = blockIdx.y * kRows + warp * 8 + r;
+  const bool live = i < d;
+  const float* brow = Bfactor + (size_t)(live ? i : d - 1) * d;  // idle lanes re-read the last row and drop the sum
+  // the first 128 columns of the row are requested before the normals are generated, so the loads' latency
+  // hides behind the transform
+  constexpr int kPrefetch = 8;
+  float4 pre[kPrefetch];
+  if (VEC) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int i = 4 * j + e;
-      w_smem[c * d4 + i] = (i < d) ? (Dvec ? (double)Dvec[i] * zz[e] : zz[e]) : 0.0;
+    for (int u = 0; u < kPrefetch; ++u) {
+      const int j0 = 4 * q + 16 * u;
+      pre[u] = (j0 < d) ? __ldg(reinterpret_cast<const float4*>(brow + j0)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
+  // one thread per Box-Muller pair: coordinates 4j + 2h, 4j + 2h + 1 of candidate c (both halves of a block
+  // recompute the block's four words, which costs far less than the transform)
+  for (int idx = threadIdx.x; idx < kCand * nb * 2; idx += blockDim.x) {
+    const int c = idx / (nb * 2), jh = idx % (nb * 2), j = jh >> 1, h = jh & 1;
+    double z0 = 0.0, z1 = 0.0;
+    if (kk0 + c < k_count) {
+      const uint4 w = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)(k_begin + kk0 + c), 0u, 0u), key);
+      box_muller(h ? w.z : w.x, h ? w.w : w.y, z0, z1);
+    }
+    const int i0 = 4 * j + 2 * h;
+    w_smem[c * d4 + i0] = (i0 < d) ? (Dvec ? (double)Dvec[i0] * z0 : z0) : 0.0;
+    w_smem[c * d4 + i0 + 1] = (i0 + 1 < d) ? (Dvec ? (double)Dvec[i0 + 1] * z1 : z1) : 0.0;
+  }
   __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  const int row_end = min(d, (int)(blockIdx.y + 1) * kRows);
-  for (int i = blockIdx.y * kRows + warp; i < row_end; i += nwarps) {
-    double acc[kCand];
+  double acc[kCand];
 #pragma unroll
-    for (int c = 0; c < kCand; ++c) acc[c] = 0.0;
-    const float* brow = Bfactor + (size_t)i * d;
-    for (int j = lane; j < d; j += 32) {
+  for (int c = 0; c < kCand; ++c) acc[c] = 0.0;
+  if (VEC) {  // d % 4 == 0 and Bfactor 16-byte aligned
+    auto consume = [&](const float4& b4, int j0) {
+      const double b[4] = {(double)b4.x, (double)b4.y, (double)b4.z, (double)b4.w};
+#pragma unroll
+      for (int c = 0; c < kCand; ++c) {
+        const double2 w01 = *reinterpret_cast<const double2*>(w_smem + c * d4 + j0);
+        const double2 w23 = *reinterpret_cast<const double2*>(w_smem + c * d4 + j0 + 2);
+        acc[c] = fma(b[0], w01.x, acc[c]);
+        acc[c] = fma(b[1], w01.y, acc[c]);
+        acc[c] = fma(b[2], w23.x, acc[c]);
+        acc[c] = fma(b[3], w23.y, acc[c]);
+      }
+    };
+#pragma unroll
+    for (int u = 0; u < kPrefetch; ++u) {
+      const int j0 = 4 * q + 16 * u;
+      if (j0 < d) consume(pre[u], j0);
+    }
+#pragma unroll 8
+    for (int j0 = 4 * q + 16 * kPrefetch; j0 < d; j0 += 16)
+      consume(__ldg(reinterpret_cast<const float4*>(brow + j0)), j0);
+  } else {
+#pragma unroll 4
+    for (int j = q; j < d; j += 4) {
       const double b = (double)__ldg(brow + j);
 #pragma unroll
       for (int c = 0; c < kCand; ++c) acc[c] = fma(b, w_smem[c * d4 + j], acc[c]);
     }
+  }
 #pragma unroll
-    for (int c = 0; c < kCand; ++c) {
+  for (int c = 0; c < kCand; ++c) {
+    acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], 1);
+    acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], 2);
+  }
+  if (live && q == 0) {
+    const double mi = (double)mean[i];
 #pragma unroll
-      for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
-    }
-    if (lane == 0) {
-      const double mi = (double)mean[i];
-#pragma unroll
-      for (int c = 0; c < kCand; ++c)
-        if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = (float)(mi + (double)step * acc[c]);
-    }
+    for (int c = 0; c < kCand; ++c)
+      if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = (float)(mi + (double)step * acc[c]);
   }
 }
 
@@ -146,13 +187,15 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
   } else {
     if (d > 4096) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 4096 with a full covariance factor");
     const size_t smem = (size_t)kCand * nb * 4 * sizeof(double);
+    const bool vec = (d % 4 == 0) && (reinterpret_cast<uintptr_t>(Bfactor) % 16 == 0);
+    auto kernel = vec ? sample_full_kernel<true> : sample_full_kernel<false>;
     if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(sample_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(sample_full_kernel)");
     }
     dim3 grid((k_count + kCand - 1) / kCand, (d + kRows - 1) / kRows);
-    sample_full_kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin,
-                                                                k_count, sigma_out);
+    kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin, k_count,
+                                                    sigma_out);
   }
   ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "sampler launch");
