@@ -147,11 +147,11 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
       cudaMemset(ctx->dec_u, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
       cudaMalloc(&ctx->dec_cnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
       cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_ppart, (size_t)ESSA_MAX_BLOCK_ITEMS * 8 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_grp, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2) != cudaSuccess ||
-      cudaMemset(ctx->dec_grp, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2) != cudaSuccess) {
+      cudaMalloc(&ctx->dec_ppart, (size_t)ESSA_MAX_BLOCK_ITEMS * 32 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_pcnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess) {
     if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
-    if (ctx->dec_grp) cudaFree(ctx->dec_grp);
+    if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->dec_u) cudaFree(ctx->dec_u);
     if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
@@ -181,7 +181,7 @@ int32_t essa_destroy(essa_ctx* ctx) {
   if (ctx->dec_u) cudaFree(ctx->dec_u);
   if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
   if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
-  if (ctx->dec_grp) cudaFree(ctx->dec_grp);
+  if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
   delete ctx;
   return ESSA_OK;
 }
@@ -200,8 +200,9 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
     if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
     cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
-    cudaMemset(ctx->dec_grp, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * 2);
+    cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
     for (uint32_t& e : ctx->dec_epoch) e = 0;
+    for (uint32_t& e : ctx->dec_pepoch) e = 0;
   }
   return ESSA_OK;
 }

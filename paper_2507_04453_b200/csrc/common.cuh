@@ -37,8 +37,9 @@ struct essa_ctx {
   void* dec_u = nullptr;
   uint32_t* dec_cnt = nullptr;
   uint32_t dec_epoch[ESSA_MAX_BLOCK_ITEMS] = {};  // (one buffer / counter set per projection of a block launch)
-  void* dec_ppart = nullptr;    // [8][kDecodeMaxTokens][64] fp32: per-K-slice partial down-projections
-  int* dec_grp = nullptr;       // [kDecodeMaxTokens / 4] arrival counters of the token groups (kept at zero)
+  void* dec_ppart = nullptr;    // [32][kDecodeMaxTokens][64] fp32 per projection: per-slice partial down-projections
+  uint32_t* dec_pcnt = nullptr; // slices delivered so far, per projection (monotonic; dec_pepoch is the host's copy)
+  uint32_t dec_pepoch[ESSA_MAX_BLOCK_ITEMS] = {};
   // Scratch owned by the context (grown on demand, never shrunk).
   essa::Scratch u_buf;        // [T_cap][64] bf16: rank-path vector u_t, zero-padded to 64 columns
   essa::Scratch splitk_ws;    // fp32 partial tiles for split-K (kept all-zero between calls)

@@ -12,10 +12,16 @@
 //     A tcgen05.mma of 128 rows costs about the same whatever its width, and a TMA load takes ~2500 cycles even
 //     when it hits L2, so the loop issues only the four wide MMAs per K block and keeps all of shared memory
 //     full of loads in flight (a ring of W0 tiles from HBM, a ring of x tiles from L2).
-//   rank path, on the CUDA cores of the four epilogue warps, which would otherwise idle during the loop:
-//     the first CTAs of the grid each take a few tokens,  p = V_A^T x_t  (16-byte loads, warp-shuffle and
-//     shared-memory reductions),  u = sB_k .* (M (sA_k .* p))  in registers, and publish u_t (bf16) to a small
-//     global buffer followed by a release-increment of a counter.  fp32 throughout.
+//   rank path.  Down-projection p = V_A^T x on the tensor core, as a by-product of the loop: the x tiles are in
+//     shared memory anyway, so for a few K blocks (a "slice") a CTA also loads the matching 64-column tile of
+//     V_A^T and issues a second MMA with the same x descriptor into a second accumulator,
+//     P[rank row][token] += V_A^T_tile . x_tile^T.  The slices of a projection are spread over its CTAs (each
+//     CTA starts its K loop at its own slice, so the slices finish within the first few K blocks); an owner's
+//     epilogue warps copy the fp32 partial to a per-slice slot in global memory and count an arrival.
+//     Finishing step, on the CUDA cores of the epilogue warps (idle during the loop): the first CTAs of the
+//     grid each take groups of 8 tokens, wait (bounded) for all slices, sum the slots in slice order,
+//     u = sB_k .* (M (sA_k .* p)) in fp32, and publish u_t (bf16) to a small global buffer followed by a
+//     release-increment of a counter.
 //   up-projection: the CTAs of K split 0 wait (bounded) until the counter shows all T rows, TMA-load u as one
 //     more K slab and add  U_B_tile . u^T  (two slabs for INT8 storage) to their accumulator.
 //   cluster reduction: after a cluster barrier (all MMAs of the cluster done, operand buffers dead) every
@@ -23,8 +29,8 @@
 //     shared memory stores); after a second barrier CTA s sums the slots in fixed rank order (results are
 //     deterministic), applies the INT8 per-channel scale, rounds to bf16 once and stores y.
 //
-// The producers of u never wait for anything another CTA does, and they are the lowest-numbered CTAs of the
-// grid, so a consumer's wait always ends; it is bounded all the same.  Warp roles (192 threads): warp 0 = TMA
+// Slice owners never wait for another CTA before they deliver, the finishing CTAs wait only for the owners, and
+// both are low-numbered CTAs of the first wave, so every wait ends; all are bounded all the same.  Warp roles (192 threads): warp 0 = TMA
 // producer of both rings, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue; INT8 storage
 // adds warps 6..7, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
 // on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster barriers, frees its TMEM and exits.
@@ -43,9 +49,13 @@ constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 6;
 constexpr int kInt8ConvStages = 3;  // converted tiles between the two converting warps and the tensor core
 constexpr int kDecThreadsInt8 = 256;             // + warps 6..7: INT8 -> bf16 converters
 constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored INT8 codes
-constexpr int kMaxRankTokens = 4;  // tokens of one rank-path unit (2 for the widest ranks, which need the registers)
-__host__ __device__ constexpr int rank_group_tokens(int vap_cols) { return vap_cols > 32 ? 2 : kMaxRankTokens; }
-constexpr int DEC_AUX_BYTES = 8 * 1024;  // barriers, flags, rank-path reduction buffers
+constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
+static_assert(kFinishTokens == 8, "finish_unit loads four tokens per thread as one float4");
+constexpr int kMaxPSlices = 32;    // slots of partial down-projections per projection
+constexpr int kVatStages = 2;      // ring of V_A^T tiles (used only during a CTA's slice)
+constexpr int VAT_SLOT_BYTES = kRankPadMax * DEC_K * 2;  // 8 KB: up to 64 rank rows of 64 input features
+constexpr int DEC_AUX_BYTES = 8 * 1024;  // barriers, flags, finishing-step buffers
+constexpr uint32_t TMEM_P_COL = 256;     // the down-projection accumulator sits behind the main one
 
 struct DParams {
   int T;          // tokens in the call (<= 256)
@@ -61,13 +71,13 @@ struct DParams {
   int ldy;
   const __half* scale;
   // rank path
-  const __nv_bfloat16* x;    // [T][d_in]
-  const __nv_bfloat16* VAp;  // [d_in][vap_cols]
-  int vap_cols;
-  int rank_groups;           // groups of kMaxRankTokens tokens
-  int rank_slices;           // K slices per group; unit w = (group w / slices, slice w % slices)
-  float* p_part;             // [8][256][64] fp32: partial down-projections, one slot per K slice
-  int* grp_count;            // [128] arrivals per group (left at zero)
+  int r_pad;                 // rank rows of a V_A^T tile (the TMA box): 16 / 32 / 48 / 64
+  int p_c;                   // K blocks per slice: CTA (m_tile j, split s) owns local K blocks [j p_c, (j+1) p_c)
+  int p_per_split;           // slots reserved per split (slot = split * p_per_split + j)
+  int rank_groups;           // finishing units: groups of kFinishTokens tokens
+  float* p_part;             // [kMaxPSlices][64 rank rows][256 tokens] fp32: partial down-projections, one slot per slice
+  uint32_t* p_count;         // slices delivered so far (monotonic across calls)
+  uint32_t p_target;         // value of *p_count once this call's slices are all in
   const int32_t* seg;
   int P;
   const float* sigma;
@@ -91,7 +101,7 @@ struct DBlock {
   DParams proj[kMaxBlockProj];
 };
 struct DMaps {
-  CUtensorMap tm[kMaxBlockProj][5];   // per projection: W0, x, u, U_B slab 0, U_B slab 1
+  CUtensorMap tm[kMaxBlockProj][6];   // per projection: W0, x, u, U_B slab 0, U_B slab 1, V_A^T
 };
 
 // tokens of the receive buffer each CTA of a cluster of `splits` owns: a multiple of 16 so that a 16-token
@@ -101,183 +111,103 @@ __host__ __device__ inline int dec_recv_bytes(int tn, int splits) {
   return splits * dec_rows_per_owner(tn, splits) * DEC_M * 4;
 }
 
-__device__ __forceinline__ void bf16x8_to_float(const uint4& v, float (&f)[8]) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+// One finishing unit of the rank path, by the 128 epilogue threads of one CTA: tokens t0 .. t0 + 7 of a projection.
+// Thread (h, j) = (etid / 64, etid % 64) owns rank coordinate j of the tokens t0 + 4h .. t0 + 4h + 3: it sums the
+// slices' partial p_j (one 16-byte load per slice: the slots are stored [rank row][token]) in slice order
+// (deterministic), forms q = sA_k .* p; after a barrier v_j = (M q)_j with its
+// row of the core matrix, u_j = sB_k,j v_j, stored as bf16; then the group's tokens are added to the published-row
+// count.  Everything that does not depend on the slices (candidate lookup, singular values, the row of M) is
+// requested before the wait for them.  Returns false when the wait gave up.
+__device__ __forceinline__ bool finish_unit(const DParams& p, int grp, float* qbuf /*[kFinishTokens][64]*/, volatile int* flag,
+                                            volatile int* abort_flag, int etid) {
+  constexpr int TPT = kFinishTokens / 2;  // tokens per thread
+  const int j = etid & 63, h = etid >> 6;
+  const int t0 = grp * kFinishTokens;
+  const int g_n = min(kFinishTokens, p.T - t0);
+  // equal-length segments are found by one proportional guess, checked against its two offsets
+  float s_a[TPT], s_b[TPT];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = __uint_as_float(w[i] << 16);
-    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
-}
-
-// One unit of the rank path, by the 128 epilogue threads of one CTA: the tokens of group `grp` (G consecutive
-// tokens) over the input features of K slice `slice` (of p.rank_slices).
-//   partial p = V_A[slice]^T x_t[slice] : thread (rb, cc) owns the 8 columns 8cc..8cc+7 and the row blocks
-//   rb, rb + RBS, ... of 8 input features each (one 16-byte load of x per token, eight of V_A per block, the next
-//   block's loads in flight while this one is multiplied); partial sums meet by xor-shuffles inside a warp and
-//   through shared memory across the four warps, and go to this slice's slot of a global buffer.
-//   The CTA that completes a group (arrival counter) sums the slots in slice order (deterministic), forms
-//   q = sA_k .* p, v = M q (thread j owns coordinate j), u = sB_k .* v, stores the 64-wide bf16 rows and adds
-//   the group's tokens to the published-row count.
-template <int COLS>
-__device__ __forceinline__ void rank_unit(const DParams& p, int grp, int slice, float* red /*[4][G][COLS]*/,
-                                          float* qbuf /*[G][64]*/, volatile int* flag, int etid) {
-  constexpr int G = rank_group_tokens(COLS);
-  constexpr int TPR = COLS / 8;      // threads per V_A row
-  constexpr int RBS = 128 / TPR;     // row blocks in flight
-  const int cc = etid % TPR, rb = etid / TPR;
-  const int warp_e = etid >> 5, lane = etid & 31;
-  const int t_begin = grp * G;
-  const int g_n = min(G, p.T - t_begin);
-  const int n_blocks = p.d_in / 8;
-  const int b_per = (n_blocks + p.rank_slices - 1) / p.rank_slices;
-  const int b0 = slice * b_per, b1 = min(n_blocks, b0 + b_per);
-  // Candidate lookup for the finishing step: equal-length segments are found by one proportional guess; its two
-  // offsets are requested now and looked at after the loop, so that no load of the loop waits behind them.
-  const int j = etid;
-  int guess[G], off_lo[G], off_hi[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    guess[g] = min(p.P - 1, (int)(((long long)(t_begin + (g < g_n ? g : 0)) * p.P) / p.T));
-    off_lo[g] = __ldg(p.seg + guess[g]);
-    off_hi[g] = __ldg(p.seg + guess[g] + 1);
-  }
-  float acc[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g)
-#pragma unroll
-    for (int c = 0; c < 8; ++c) acc[g][c] = 0.f;
-  // software pipeline at row granularity: as soon as a register of the current block has been unpacked, the same
-  // register is refilled with the next block's data, so a full block of loads is always in flight
-  uint4 xr[G], vr[8];
-  auto x_ptr = [&](int g, int b) { return reinterpret_cast<const uint4*>(p.x + (size_t)(t_begin + (g < g_n ? g : 0)) * p.d_in) + b; };
-  auto v_ptr = [&](int i, int b) { return reinterpret_cast<const uint4*>(p.VAp + (size_t)b * 8 * COLS) + cc + (size_t)i * TPR; };
-  int b = b0 + rb;
-  if (b < b1) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) xr[g] = __ldg(x_ptr(g, b));
-#pragma unroll
-    for (int i = 0; i < 8; ++i) vr[i] = __ldg(v_ptr(i, b));
-  }
-  while (b < b1) {
-    const int bn = b + RBS;
-    const bool more = bn < b1;
-    float xv[G][8];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      bf16x8_to_float(xr[g], xv[g]);
-      if (more) xr[g] = __ldg(x_ptr(g, bn));
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float vv[8];
-      bf16x8_to_float(vr[i], vv);
-      if (more) vr[i] = __ldg(v_ptr(i, bn));
-#pragma unroll
-      for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(vv[c], xv[g][i], acc[g][c]);
-    }
-    b = bn;
-  }
-  // singular values of the tokens' candidates and this thread's row of the core matrix: one round trip, in flight
-  // during the reductions below
-  float s_a[G], s_b[G];
-  float4 mreg[COLS / 4];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
+  for (int g = 0; g < TPT; ++g) {
     s_a[g] = 0.f; s_b[g] = 0.f;
-    if (j < p.r && g < g_n) {
-      const int t = t_begin + g;
-      const int k = (off_lo[g] <= t && t < off_hi[g]) ? guess[g] : find_candidate(p.seg, p.P, t);
+    const int tl = TPT * h + g;
+    if (tl < g_n && j < p.r) {
+      const int t = t0 + tl;
+      const int guess = min(p.P - 1, (int)(((long long)t * p.P) / p.T));
+      const int lo = __ldg(p.seg + guess), hi = __ldg(p.seg + guess + 1);
+      const int k = (lo <= t && t < hi) ? guess : find_candidate(p.seg, p.P, t);
       const float* srow = p.sigma + (size_t)k * p.ld_sigma;
       s_a[g] = __ldg(srow + p.sA_col + j);
       s_b[g] = __ldg(srow + p.sB_col + j);
     }
   }
+  float4 mreg[kRankPadMax / 4];  // row j of M (zero beyond the rank)
 #pragma unroll
-  for (int i4 = 0; i4 < COLS / 4; ++i4)
-    mreg[i4] = __ldg(reinterpret_cast<const float4*>(p.M + (j < kRankPadMax ? j : 0) * kRankPadMax) + i4);
-  // lanes with equal cc hold partial sums of the same columns: fold lane bits log2(TPR) .. 4
-#pragma unroll
-  for (int off = TPR; off < 32; off <<= 1)
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) acc[g][c] += __shfl_xor_sync(0xffffffffu, acc[g][c], off);
-  if (lane < TPR) {
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) red[(warp_e * G + g) * COLS + 8 * cc + c] = acc[g][c];
-  }
-  epi_bar_sync();
-  bool last = true;
-  if (p.rank_slices > 1) {
-  // this slice's partial p -> its slot  [slice][token][64]
-  for (int idx = etid; idx < G * COLS; idx += 128) {
-    const int g = idx / COLS, c = idx % COLS;
-    if (g < g_n)
-      p.p_part[((size_t)slice * kDecodeMaxTokens + t_begin + g) * kRankPadMax + c] =
-          red[(0 * G + g) * COLS + c] + red[(1 * G + g) * COLS + c] + red[(2 * G + g) * COLS + c] + red[(3 * G + g) * COLS + c];
-  }
-  __threadfence();
-  epi_bar_sync();
+  for (int i4 = 0; i4 < kRankPadMax / 4; ++i4) mreg[i4] = __ldg(reinterpret_cast<const float4*>(p.M + j * kRankPadMax) + i4);
+  // all slices delivered?
   if (etid == 0) {
-    const int prev = atomicAdd(p.grp_count + grp, 1);
-    const int is_last = prev == p.rank_slices - 1;
-    if (is_last) p.grp_count[grp] = 0;  // every slice has arrived: leave the counter clean for the next call
-    *flag = is_last;
+    int ok = 1;
+    const long long w0 = clock64();
+    while ((int32_t)(ld_acquire_u32(p.p_count) - p.p_target) < 0) {
+      if (*abort_flag || clock64() - w0 > kWaitLimitCycles) { ok = 0; break; }
+    }
+    if (!ok) {
+      *abort_flag = 1;
+      atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+    }
+    *flag = ok;
   }
   epi_bar_sync();
-  last = *flag != 0;
-  if (last) __threadfence();
-  }
-  if (last) {
-    if (j < kRankPadMax) {
+  const bool ok = *flag != 0;
+  if (ok) {
+    float pj[TPT];
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float pj = 0.f;
-        if (g < g_n && j < p.r) {
-          if (p.rank_slices > 1) {
-            for (int sl = 0; sl < p.rank_slices; ++sl)
-              pj += ld_cg_f32(p.p_part + ((size_t)sl * kDecodeMaxTokens + t_begin + g) * kRankPadMax + j);
-          } else {
-            pj = red[(0 * G + g) * COLS + j] + red[(1 * G + g) * COLS + j] + red[(2 * G + g) * COLS + j] + red[(3 * G + g) * COLS + j];
-          }
+    for (int g = 0; g < TPT; ++g) pj[g] = 0.f;
+    if (j < p.r) {
+      // slot sp * p_per_split + sl exists when slice sl of split sp does; eight loads in flight at a time
+      const int kbase = p.main_kb / p.splits, krem = p.main_kb % p.splits;
+      const int n_flat = p.splits * p.p_per_split;
+      const float* base = p.p_part + (size_t)j * kDecodeMaxTokens + t0 + TPT * h;
+      for (int i0 = 0; i0 < n_flat; i0 += 8) {
+        float4 v4[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int idx = i0 + u;
+          const int sp = idx / p.p_per_split, sl = idx - sp * p.p_per_split;
+          const bool valid = idx < n_flat && sl * p.p_c < kbase + (sp < krem ? 1 : 0);
+          v4[u] = valid ? ld_cg_f32x4(base + (size_t)idx * kRankPadMax * kDecodeMaxTokens) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        qbuf[g * kRankPadMax + j] = pj * s_a[g];  // sA_k .* p  (zero beyond the rank)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { pj[0] += v4[u].x; pj[1] += v4[u].y; pj[2] += v4[u].z; pj[3] += v4[u].w; }
       }
     }
+#pragma unroll
+    for (int g = 0; g < TPT; ++g) qbuf[(TPT * h + g) * kRankPadMax + j] = pj[g] * s_a[g];  // sA_k .* p  (zero beyond the rank)
     epi_bar_sync();
-    if (j < kRankPadMax) {
-      float v[G];
+    float v[TPT];
 #pragma unroll
-      for (int g = 0; g < G; ++g) v[g] = 0.f;
-      if (j < p.r) {
+    for (int g = 0; g < TPT; ++g) v[g] = 0.f;
 #pragma unroll
-        for (int i4 = 0; i4 < COLS / 4; ++i4) {
-          const float4 mm = mreg[i4];  // zero beyond the rank
+    for (int i4 = 0; i4 < kRankPadMax / 4; ++i4) {
+      const float4 mm = mreg[i4];
 #pragma unroll
-          for (int g = 0; g < G; ++g) {
-            const float4 qq = *reinterpret_cast<const float4*>(qbuf + g * kRankPadMax + 4 * i4);
-            v[g] = fmaf(mm.x, qq.x, v[g]);
-            v[g] = fmaf(mm.y, qq.y, v[g]);
-            v[g] = fmaf(mm.z, qq.z, v[g]);
-            v[g] = fmaf(mm.w, qq.w, v[g]);
-          }
-        }
+      for (int g = 0; g < TPT; ++g) {
+        const float4 qq = *reinterpret_cast<const float4*>(qbuf + (TPT * h + g) * kRankPadMax + 4 * i4);
+        v[g] = fmaf(mm.x, qq.x, v[g]);
+        v[g] = fmaf(mm.y, qq.y, v[g]);
+        v[g] = fmaf(mm.z, qq.z, v[g]);
+        v[g] = fmaf(mm.w, qq.w, v[g]);
       }
-#pragma unroll
-      for (int g = 0; g < G; ++g)
-        if (g < g_n) p.u[(size_t)(t_begin + g) * kRankPadMax + j] = __float2bfloat16(v[g] * s_b[g]);  // sB_k .* (M q)
     }
+#pragma unroll
+    for (int g = 0; g < TPT; ++g)
+      if (TPT * h + g < g_n) p.u[(size_t)(t0 + TPT * h + g) * kRankPadMax + j] = __float2bfloat16(v[g] * s_b[g]);  // sB_k .* (M q)
     // publish: every writer's rows are visible device-wide before the count moves
     __threadfence();
     epi_bar_sync();
     if (etid == 0) red_release_add_u32(p.u_count, (uint32_t)g_n);
   }
-  epi_bar_sync();  // red / qbuf / flag may be reused
+  epi_bar_sync();  // qbuf / flag may be reused
+  return ok;
 }
 
 // Sum token rows j0, j0 + 4, ... < j_end of this CTA's slice over the NS receive slots (cluster rank order:
@@ -323,29 +253,33 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const CUtensorMap& tmU = maps.tm[pi][2];
   const CUtensorMap& tmUB0 = maps.tm[pi][3];
   const CUtensorMap& tmUB1 = maps.tm[pi][4];
+  const CUtensorMap& tmV = maps.tm[pi][5];
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
   const int x_bytes = p.tn * 128;
   constexpr int W_SLOT = INT8 ? RAW_TILE_BYTES : W_TILE_BYTES;
   const int SC = INT8 ? p.c_stages : 0;
-  uint8_t* smem_w = smem;                      // W0 ring as stored (bf16: the U_B slabs are its last items)
-  uint8_t* smem_c = smem + SW * W_SLOT;        // INT8: ring of converted bf16 tiles (the U_B slabs are its last items)
+  // V_A^T tiles first: their MMA descriptor spans 128 rows, of which only the r_pad rows of the TMA box are data
+  // (the accumulator rows beyond are never read), so the 16 KB it covers must lie inside the allocation
+  uint8_t* smem_v = smem;
+  uint8_t* smem_w = smem_v + kVatStages * VAT_SLOT_BYTES;  // W0 ring as stored (bf16: the U_B slabs are its last items)
+  uint8_t* smem_c = smem_w + SW * W_SLOT;      // INT8: ring of converted bf16 tiles (the U_B slabs are its last items)
   uint8_t* smem_x = smem_c + SC * W_TILE_BYTES;  // x ring (the u tile is its last item)
   uint8_t* aux = smem_x + SX * x_bytes;
   // receive buffer of the cluster reduction, [splits][per tokens][128 ch] fp32: overlays both rings, which are
   // dead once every MMA of the cluster has completed
   float* recv = reinterpret_cast<float*>(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2 + 2 * kVatStages + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* red = reinterpret_cast<float*>(aux + 1024);       // [4][G][64]
-  float* qbuf = red + 4 * kMaxRankTokens * kRankPadMax;    // [G][64]
+  float* qbuf = reinterpret_cast<float*>(aux + 1024);      // [kFinishTokens][64]
 
   const uint32_t bar_wfull = smem_u32(bars), bar_wempty = bar_wfull + 8 * kMaxWStages;
   const uint32_t bar_xfull = bar_wempty + 8 * kMaxWStages, bar_xempty = bar_xfull + 8 * kMaxXStages;
   const uint32_t bar_cfull = bar_xempty + 8 * kMaxXStages, bar_cempty = bar_cfull + 8 * kMaxCStages;
   const uint32_t bar_d = bar_cempty + 8 * kMaxCStages, bar_drain = bar_d + 8;
+  const uint32_t bar_vfull = bar_drain + 8, bar_vempty = bar_vfull + 8 * kVatStages, bar_p = bar_vempty + 8 * kVatStages;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = (int)cluster_ctarank();
@@ -360,7 +294,12 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const int n_w = INT8 ? nkb : nkb + n_ext;  // items of the W0 ring: the K blocks (bf16: then the U_B slabs)
   const int n_x = nkb + (n_ext ? 1 : 0);     // items of the x ring: the K blocks, then the u tile
   const int per = dec_rows_per_owner(p.tn, p.splits);
-  constexpr uint32_t TMEM_COLS = 256;
+  constexpr uint32_t TMEM_COLS = 512;  // main accumulator (up to 256 tokens) + down-projection accumulator
+  // The K loop starts at this CTA's slice of the down-projection and wraps around: item i is local K block
+  // (r0 + i) mod nkb, and the first c_own items also feed the second accumulator.
+  const int r0 = nkb > 0 ? (m_tile * p.p_c) % nkb : 0;
+  const int c_own = (is_main && m_tile * p.p_c < nkb) ? min(p.p_c, nkb - m_tile * p.p_c) : 0;
+  auto kcol = [&](int i) { const int l = r0 + i; return (kb0 + (l >= nkb ? l - nkb : l)) * DEC_K; };
 
   auto load_w = [&](int i) {  // item i of the W0 ring
     const int s = i % SW;
@@ -368,10 +307,10 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     mbar_expect_tx(fb, (uint32_t)W_SLOT);
     const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
     if (INT8) {  // 128 rows of 64 codes, unswizzled
-      tma_load_2d(dst, &tmW, (kb0 + i) * DEC_K, m_tile * DEC_M, fb);
+      tma_load_2d(dst, &tmW, kcol(i), m_tile * DEC_M, fb);
     } else {     // two 64-row boxes
       const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
-      const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
+      const int col = i < nkb ? kcol(i) : 0;
       tma_load_2d(dst, tm, col, m_tile * DEC_M, fb);
       tma_load_2d(dst + 64 * 128, tm, col, m_tile * DEC_M + 64, fb);
     }
@@ -391,8 +330,14 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const uint32_t dst = smem_u32(smem_x + s * x_bytes);
     mbar_expect_tx(fb, (uint32_t)x_bytes);
     const CUtensorMap* tm = i < nkb ? &tmX : &tmU;
-    const int col = i < nkb ? (kb0 + i) * DEC_K : 0;
+    const int col = i < nkb ? kcol(i) : 0;
     for (int r = 0; r < p.tn; r += p.xbox) tma_load_2d(dst + (uint32_t)(r * 128), tm, col, r, fb);
+  };
+  auto load_v = [&](int i) {  // V_A^T tile of item i < c_own: r_pad rank rows x 64 input features
+    const int s = i % kVatStages;
+    const uint32_t fb = bar_vfull + 8 * s;
+    mbar_expect_tx(fb, (uint32_t)(p.r_pad * 128));
+    tma_load_2d(smem_u32(smem_v + s * VAT_SLOT_BYTES), &tmV, kcol(i), 0, fb);
   };
 
   const int first_w = n_w < SW ? n_w : SW;  // the ring starts empty: its first fill needs no wait
@@ -402,6 +347,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     for (int s = 0; s < SC; ++s) { mbar_init(bar_cfull + 8 * s, 1); mbar_init(bar_cempty + 8 * s, 1); }
     mbar_init(bar_d, 1);
     mbar_init(bar_drain, 1);
+    for (int s = 0; s < kVatStages; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 1); }
+    mbar_init(bar_p, 1);
     *abort_flag = 0;
     *reinterpret_cast<volatile int*>(tmem_slot + 3) = 0;  // conversion ticket
     *reinterpret_cast<volatile int*>(tmem_slot + 4) = 0;  // ... and whose turn it is to claim a slot
@@ -421,11 +368,15 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     // ------------------------------------------------------------------ TMA producer: one thread feeds both rings,
     // issuing whatever has a free slot (each ring in its own order, so the parity waits stay in step)
     if (lane == 0) {
-      int iw = first_w, ix = 0;  // next item of the W0 ring, of the x ring
+      int iw = first_w, ix = 0, iv = 0;  // next item of the W0 ring, of the x ring, of the V_A^T ring
       bool ok = true;
       long long t_idle = 0;
-      while (ok && (iw < n_w || ix < n_x)) {
+      while (ok && (iw < n_w || ix < n_x || iv < c_own)) {
         bool progress = false;
+        if (iv < c_own && (iv < kVatStages || mbar_test_wait(bar_vempty + 8 * (iv % kVatStages), (uint32_t)(((iv / kVatStages) & 1) ^ 1)))) {
+          load_v(iv++);
+          progress = true;
+        }
         if (iw < n_w && (iw < SW || mbar_test_wait(bar_wempty + 8 * (iw % SW), (uint32_t)(((iw / SW) & 1) ^ 1)))) {
           load_w(iw++);
           progress = true;
@@ -464,6 +415,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         };
         drain(iw, SW, bar_wfull);
         drain(ix, SX, bar_xfull);
+        drain(iv, kVatStages, bar_vfull);
       }
     }
   } else if (warp == 1 && is_main) {
@@ -482,6 +434,17 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
 #pragma unroll
         for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        if (i < c_own) {
+          // this CTA's slice of the down-projection: V_A^T tile against the same x tile, second accumulator
+          const int sv = i % kVatStages;
+          if (!mbar_wait(bar_vfull + 8 * sv, (uint32_t)((i / kVatStages) & 1), abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t dv = make_smem_desc(smem_u32(smem_v + sv * VAT_SLOT_BYTES));
+#pragma unroll
+          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base + TMEM_P_COL, dv + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          umma_commit(bar_vempty + 8 * sv);
+          if (i == c_own - 1) umma_commit(bar_p);  // the slice is complete
+        }
         umma_commit((INT8 ? bar_cempty : bar_wempty) + 8 * sw);
         umma_commit(bar_xempty + 8 * sx);
       }
@@ -598,20 +561,41 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   int got = 0;
   if (epi) {
     const int etid = threadIdx.x - 64;
+    volatile int* flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+    if (c_own > 0) {
+      // this CTA's slice of the down-projection: accumulator rows (rank index) x columns (token) -> its slot
+      int have = 0;
+      if (lane == 0) have = mbar_wait(bar_p, 0, abort_flag, p.status) ? 1 : 0;
+      have = __shfl_sync(0xffffffffu, have, 0);
+      if (have) {
+        while (!mbar_try_wait(bar_p, 0)) {}  // complete: returns at once (acquire for every lane)
+        tc_fence_after();
+        if (quad * 32 < p.r_pad) {
+          float* slot = p.p_part + (size_t)(split * p.p_per_split + m_tile) * kDecodeMaxTokens * kRankPadMax;
+#pragma unroll 1
+          for (int c = 0; c < p.tn / 16; ++c) {
+            float v[16];
+            tmem_ld16(t_lane + TMEM_P_COL + c * 16, v);
+            if (row < p.r_pad) {  // [rank row][token]; columns of tokens beyond T are zero (their x rows are)
+              float4* dst = reinterpret_cast<float4*>(slot + (size_t)row * kDecodeMaxTokens + c * 16);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+          }
+          tc_fence_before();
+        }
+        __threadfence();
+        epi_bar_sync();
+        if (etid == 0) red_release_add_u32(p.p_count, 1u);
+      }
+    }
     if ((int)blockIdx.x < blk.rank_ctas) {
-      // this CTA's units of the rank path (of any projection of the block), while its K loop streams
-      volatile int* flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
-      for (int unit = blockIdx.x; unit < blk.unit_begin[blk.n_proj]; unit += blk.rank_ctas) {
+      // this CTA's finishing units of the rank path (of any projection of the block), while its K loop streams
+      bool fine = true;
+      for (int unit = blockIdx.x; fine && unit < blk.unit_begin[blk.n_proj]; unit += blk.rank_ctas) {
         int pj = 0;
         while (pj + 1 < blk.n_proj && unit >= blk.unit_begin[pj + 1]) ++pj;
-        const DParams& pr = blk.proj[pj];
-        const int local = unit - blk.unit_begin[pj];
-        const int grp = local / pr.rank_slices, slice = local % pr.rank_slices;
-        switch (pr.vap_cols) {
-          case 16: rank_unit<16>(pr, grp, slice, red, qbuf, flag, etid); break;
-          case 32: rank_unit<32>(pr, grp, slice, red, qbuf, flag, etid); break;
-          default: rank_unit<64>(pr, grp, slice, red, qbuf, flag, etid); break;
-        }
+        fine = finish_unit(blk.proj[pj], unit - blk.unit_begin[pj], qbuf, flag, abort_flag, etid);
       }
     }
     got = is_main ? 1 : 0;
@@ -678,7 +662,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
 
 // c_stages > 0 means INT8 storage: the W0 ring holds 8 KB tiles of codes and c_stages converted tiles follow it
 inline int dec_ring_bytes(int w_stages, int c_stages, int x_stages, int tn) {
-  return w_stages * (c_stages > 0 ? RAW_TILE_BYTES : W_TILE_BYTES) + c_stages * W_TILE_BYTES + x_stages * tn * 128;
+  return kVatStages * VAT_SLOT_BYTES + w_stages * (c_stages > 0 ? RAW_TILE_BYTES : W_TILE_BYTES) + c_stages * W_TILE_BYTES +
+         x_stages * tn * 128;
 }
 inline int dec_smem_bytes(int w_stages, int c_stages, int x_stages, int tn) {
   return 1024 + dec_ring_bytes(w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
@@ -804,16 +789,14 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   const int resident_ctas = resident_cache[splits] * splits;
   const int main_ctas = m_total * splits;
   if (n > 1 && main_ctas > resident_ctas) return kBlockNotFused;
-  // Launch a full wave: the CTAs beyond the W0-streaming ones only take rank-path units.  A unit is a group of
-  // 4 tokens (2 for ranks above 32) over one K slice; slices multiply the units until the wave is busy (at most 8).
+  // Launch a full wave: the CTAs beyond the W0-streaming ones only take finishing units of the rank path (groups
+  // of 8 tokens).
   const int grid_total = main_ctas > resident_ctas ? main_ctas : resident_ctas;
 
   DBlock blk{};
   DMaps maps{};
   blk.n_proj = n;
   blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
-  int groups_total = 0;
-  for (int i = 0; i < n; ++i) groups_total += ((int)T + rank_group_tokens(items[i].a->vap_cols) - 1) / rank_group_tokens(items[i].a->vap_cols);
   int cta = 0, unit = 0;
   for (int i = 0; i < n; ++i) {
     const essa_adapter* a = items[i].a;
@@ -833,18 +816,28 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     p.y = items[i].y;
     p.ldy = a->d_out;
     p.scale = int8 ? a->w0_scale : nullptr;
-    p.x = items[i].x;
-    p.VAp = a->VAp;
-    p.vap_cols = a->vap_cols;
-    const int gtok = rank_group_tokens(a->vap_cols);
-    p.rank_groups = ((int)T + gtok - 1) / gtok;
-    int slices = blk.rank_ctas / groups_total;
-    if (slices > 8) slices = 8;
-    if (slices > a->d_in / 512) slices = a->d_in / 512;  // at least 64 row blocks per slice
-    if (slices < 1) slices = 1;
-    p.rank_slices = slices;
-    p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)i * 8 * kDecodeMaxTokens * kRankPadMax;
-    p.grp_count = ctx->dec_grp + i * (kDecodeMaxTokens / 2);
+    p.r_pad = a->r_pad;
+    p.rank_groups = ((int)T + kFinishTokens - 1) / kFinishTokens;
+    // slices of the down-projection: the K blocks of a split are dealt to the first row tiles, p_c each, at most
+    // kMaxPSlices slots per projection
+    {
+      const int nkb_max = (p.main_kb + splits - 1) / splits;
+      int owners = kMaxPSlices / splits;  // per split
+      if (owners > p.m_tiles) owners = p.m_tiles;
+      if (owners > 16) owners = 16;
+      if (owners < 1) owners = 1;
+      p.p_c = (nkb_max + owners - 1) / owners;
+      p.p_per_split = (nkb_max + p.p_c - 1) / p.p_c;
+      int delivered = 0;
+      for (int sp = 0; sp < splits; ++sp) {
+        const int nkb_s = p.main_kb / splits + (sp < p.main_kb % splits ? 1 : 0);
+        delivered += (nkb_s + p.p_c - 1) / p.p_c;
+      }
+      p.p_count = ctx->dec_pcnt + i;
+      ctx->dec_pepoch[i] += (uint32_t)delivered;
+      p.p_target = ctx->dec_pepoch[i];
+    }
+    p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)i * kMaxPSlices * kDecodeMaxTokens * kRankPadMax;
     p.seg = seg;
     p.P = P;
     p.sigma = sigma;
@@ -861,7 +854,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     blk.cta_begin[i] = cta;
     blk.unit_begin[i] = unit;
     cta += p.m_tiles * splits;
-    unit += p.rank_groups * p.rank_slices;
+    unit += p.rank_groups;
 
     maps.tm[i][0] = int8 ? a->tm_W0q : a->tm_W0[0];  // 64-row boxes of bf16 W0 / 128-row boxes of codes
     int32_t st = make_tensor_map_2d(ctx, &maps.tm[i][1], 0, items[i].x, (uint64_t)T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
@@ -872,6 +865,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     if (st != ESSA_OK) return st;
     maps.tm[i][3] = a->tm_UBp[0][0];  // 64-row boxes of the U_B slabs
     maps.tm[i][4] = a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0];
+    maps.tm[i][5] = a->tm_VAt;
   }
   for (int i = n; i <= kMaxBlockProj; ++i) { blk.cta_begin[i] = cta; blk.unit_begin[i] = unit; }
 

@@ -126,6 +126,11 @@ __device__ __forceinline__ float ld_cg_f32(const float* addr) {
   asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(addr) : "memory");
   return v;
 }
+__device__ __forceinline__ float4 ld_cg_f32x4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void st_cg_zero_v4(float* addr) {
   asm volatile("st.global.cg.v4.f32 [%0], {%1, %1, %1, %1};" ::"l"(addr), "f"(0.f) : "memory");
 }

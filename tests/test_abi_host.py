@@ -77,7 +77,9 @@ def test_plan_is_consistent(lib, name):
             assert p["splits"] in (1, 2, 4, 8) and p["splits"] <= n // 64 and p["grid"] <= {1: 148, 2: 148, 4: 132, 8: 120}[p["splits"]]
             assert p["grid"] == p["tiles"] * p["splits"] and p["scratch_bytes"] == 0
             # bf16 storage: 16 KB W0 tiles; INT8 storage: 8 KB tiles of codes plus three converted tiles
-            rings = p["stages"] * (64 * 128 if dtype else 128 * 128) + (3 * 128 * 128 if dtype else 0) + p["x_stages"] * p["block_n"] * 128
+            # ... and two 8 KB tiles of V_A^T for the down-projection slices
+            rings = (2 * 64 * 128 + p["stages"] * (64 * 128 if dtype else 128 * 128) + (3 * 128 * 128 if dtype else 0)
+                     + p["x_stages"] * p["block_n"] * 128)
             assert 1 <= p["stages"] <= 16 and 1 <= p["x_stages"] <= 6
             assert 1024 + rings + 8192 <= 227 * 1024
             per = -(-(-(-p["block_n"] // p["splits"])) // 16) * 16
