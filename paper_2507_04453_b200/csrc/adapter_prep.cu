@@ -12,14 +12,6 @@ __global__ void build_vat_kernel(const __nv_bfloat16* __restrict__ V_A, int n, i
   for (int j = 0; j < kRankPadMax; ++j) VAt[(size_t)j * n + c] = (j < r) ? V_A[(size_t)c * r + j] : __float2bfloat16(0.f);
 }
 
-// VAp[c][j] = V_A[c][j] for j < r, 0 up to the padded width (rows are read in 16-byte chunks by the decode kernel).
-__global__ void build_vap_kernel(const __nv_bfloat16* __restrict__ V_A, int n, int r, int cols, __nv_bfloat16* __restrict__ VAp) {
-  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (size_t)n * cols) return;
-  const int c = (int)(idx / cols), j = (int)(idx % cols);
-  VAp[idx] = (j < r) ? V_A[(size_t)c * r + j] : __float2bfloat16(0.f);
-}
-
 // UBp[e][o][j]: bf16 W0 -> one slab, U_B[o][j] zero-padded to 64 columns.
 // INT8 W0 -> two slabs holding g = U_B[o][j] / scale[o] split as hi = bf16(g), lo = bf16(g - hi), because the
 // kernel multiplies the whole accumulator (base + rank term) by scale[o] once at the end.
@@ -81,9 +73,7 @@ int32_t launch_adapter_prep(essa_ctx* ctx, essa_adapter* a, const __nv_bfloat16*
   const int tot = a->d_out * kRankPadMax;
   build_ubp_kernel<<<(tot + 255) / 256, 256, 0, stream>>>(a->U_B, a->w0_scale, a->d_out, a->rank, a->ext_blocks, a->UBp);
   build_core_kernel<<<(kRankPadMax * kRankPadMax + 255) / 256, 256, 0, stream>>>(U_A, V_B, a->rank, a->M);
-  const size_t vtot = (size_t)a->d_in * a->vap_cols;
-  build_vap_kernel<<<(unsigned)((vtot + 255) / 256), 256, 0, stream>>>(a->V_A, a->d_in, a->rank, a->vap_cols, a->VAp);
-  ctx->launches += 4;
+  ctx->launches += 3;
   return check_cuda(ctx, cudaGetLastError(), "adapter prep launch");
 }
 

@@ -264,7 +264,6 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   a->d_in = d->d_in; a->d_out = d->d_out; a->rank = d->rank; a->w0_dtype = d->w0_dtype;
   a->r_pad = ((d->rank + 15) / 16) * 16;
   a->ext_blocks = int8 ? 2 : 1;
-  a->vap_cols = a->r_pad <= 16 ? 16 : a->r_pad <= 32 ? 32 : 64;
   const size_t n = d->d_in, m = d->d_out, r = d->rank;
   // INT8 weights stay stored as codes (1 byte per weight).  The decode kernel converts them to bf16 in shared
   // memory; a prefill call dequantises them once into the context's scratch before its GEMM.  Either way the fp16
@@ -279,7 +278,6 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   alloc((void**)&a->UBp, (size_t)a->ext_blocks * m * kRankPadMax * 2);
   alloc((void**)&a->U_B, m * r * 2);
   alloc((void**)&a->V_A, n * r * 2);
-  alloc((void**)&a->VAp, n * (size_t)a->vap_cols * 2);
   alloc((void**)&a->M, (size_t)kRankPadMax * kRankPadMax * 4);
   alloc((void**)&dUA, r * r * 2);
   alloc((void**)&dVB, r * r * 2);
@@ -326,7 +324,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
 int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* a) {
   if (!ctx || !a) return ESSA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->VAp, a->M};
+  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->M};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   delete a;

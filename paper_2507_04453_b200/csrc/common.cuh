@@ -59,12 +59,10 @@ struct essa_adapter {
   void* W0 = nullptr;            // [d_out][d_in] bf16 (bf16 storage only)
   int8_t* W0q = nullptr;         // [d_out][d_in] int8 codes as given (INT8 storage only)
   __half* w0_scale = nullptr;    // [d_out] fp16 (INT8)
-  __nv_bfloat16* VAt = nullptr;  // [64][d_in]: V_A^T, rows >= rank are zero (K-major B operand of the down-projection)
+  __nv_bfloat16* VAt = nullptr;  // [64][d_in]: V_A^T, rows >= rank are zero (K-major operand of the down-projection)
   __nv_bfloat16* UBp = nullptr;  // [ext][d_out][64]: U_B zero-padded to 64 columns; INT8: (U_B/scale) split hi, lo
   __nv_bfloat16* U_B = nullptr;  // [d_out][rank] as given (CUDA-core path)
   __nv_bfloat16* V_A = nullptr;  // [d_in][rank] as given (CUDA-core path)
-  __nv_bfloat16* VAp = nullptr;  // [d_in][vap_cols]: V_A zero-padded to 16 / 32 / 64 columns (16-byte row chunks)
-  int vap_cols = 0;
   float* M = nullptr;            // [64][64] fp32: M = V_B^T U_A zero-padded
   int ext_blocks = 1;            // rank-path K-slabs appended to the base contraction (1 bf16, 2 INT8)
   CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256 (bf16 storage only)
