@@ -32,7 +32,7 @@
 // Slice owners never wait for another CTA before they deliver, the finishing CTAs wait only for the owners, and
 // both are low-numbered CTAs of the first wave, so every wait ends; all are bounded all the same.  Warp roles (192 threads): warp 0 = TMA
 // producer of both rings, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue; INT8 storage
-// adds warps 6..7, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
+// adds warps 6..9, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
 // on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster barriers, frees its TMEM and exits.
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -46,8 +46,8 @@ constexpr int kDecThreads = 192;
 constexpr int kDecSmemBudget = 227 * 1024;
 constexpr int W_TILE_BYTES = DEC_M * DEC_K * 2;  // 16 KB
 constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 6;
-constexpr int kInt8ConvStages = 3;  // converted tiles between the two converting warps and the tensor core
-constexpr int kDecThreadsInt8 = 256;             // + warps 6..7: INT8 -> bf16 converters
+constexpr int kInt8ConvStages = 4;  // converted tiles between the converting warps and the tensor core
+constexpr int kDecThreadsInt8 = 320;             // + warps 6..9: INT8 -> bf16 converters
 constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored INT8 codes
 constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
 static_assert(kFinishTokens == 8, "finish_unit loads four tokens per thread as one float4");
@@ -473,7 +473,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   }
 
   // ------------------------------------------------------------------ INT8 -> bf16 conversion (INT8 storage only)
-  // Items of the converted ring are handed out to warps 6..7 by a ticket counter in shared memory, so the two
+  // Items of the converted ring are handed out to warps 6..9 by a ticket counter in shared memory, so the
   // warps work on different tiles at once.  A warp converts a whole tile:
   // raw tile = 128 rows of 64 codes, row r at byte 64 r; converted tile = the K-major 128-byte-swizzled operand
   // layout, row r at byte 128 r, 16-byte chunk c at position c ^ (r & 7).  Lane l takes the 16-code chunks
@@ -522,13 +522,13 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       if (i >= nkb) continue;
       const int sr = i % SW;
       while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}  // complete: acquire for every lane
-      const uint8_t* raw = smem_w + sr * RAW_TILE_BYTES;
-      uint8_t* out = smem_c + sc * W_TILE_BYTES;
+      const uint32_t raw = smem_u32(smem_w + sr * RAW_TILE_BYTES);
+      const uint32_t out = smem_u32(smem_c + sc * W_TILE_BYTES);
 #pragma unroll 2
       for (int c0 = 0; c0 < RAW_TILE_BYTES / 16; c0 += 64) {
         uint4 w[2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) w[h] = *reinterpret_cast<const uint4*>(raw + (c0 + 32 * h + lane) * 16);
+        for (int h = 0; h < 2; ++h) w[h] = lds_v4(raw + (uint32_t)((c0 + 32 * h + lane) * 16));
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const int chunk = c0 + 32 * h + lane;
@@ -538,9 +538,9 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
           int8x4_to_bf16x4(w[h].y, o0.z, o0.w);
           int8x4_to_bf16x4(w[h].z, o1.x, o1.y);
           int8x4_to_bf16x4(w[h].w, o1.z, o1.w);
-          uint8_t* orow = out + r * 128;
-          *reinterpret_cast<uint4*>(orow + (((2 * part) ^ (r & 7)) << 4)) = o0;
-          *reinterpret_cast<uint4*>(orow + (((2 * part + 1) ^ (r & 7)) << 4)) = o1;
+          const uint32_t orow = out + (uint32_t)(r * 128);
+          sts_v4(orow + (uint32_t)(((2 * part) ^ (r & 7)) << 4), o0);
+          sts_v4(orow + (uint32_t)(((2 * part + 1) ^ (r & 7)) << 4), o1);
         }
       }
       fence_proxy_async_smem();

@@ -76,9 +76,9 @@ def test_plan_is_consistent(lib, name):
             assert p["block_n"] == -(-T // 16) * 16 and p["tiles"] == -(-m // 128)
             assert p["splits"] in (1, 2, 4, 8) and p["splits"] <= n // 64 and p["grid"] <= {1: 148, 2: 148, 4: 132, 8: 120}[p["splits"]]
             assert p["grid"] == p["tiles"] * p["splits"] and p["scratch_bytes"] == 0
-            # bf16 storage: 16 KB W0 tiles; INT8 storage: 8 KB tiles of codes plus three converted tiles
+            # bf16 storage: 16 KB W0 tiles; INT8 storage: 8 KB tiles of codes plus four converted tiles
             # ... and two 8 KB tiles of V_A^T for the down-projection slices
-            rings = (2 * 64 * 128 + p["stages"] * (64 * 128 if dtype else 128 * 128) + (3 * 128 * 128 if dtype else 0)
+            rings = (2 * 64 * 128 + p["stages"] * (64 * 128 if dtype else 128 * 128) + (4 * 128 * 128 if dtype else 0)
                      + p["x_stages"] * p["block_n"] * 128)
             assert 1 <= p["stages"] <= 16 and 1 <= p["x_stages"] <= 6
             assert 1024 + rings + 8192 <= 227 * 1024
