@@ -214,17 +214,17 @@ __device__ __forceinline__ bool finish_unit(const DParams& p, int grp, float* qb
 // deterministic), scale, round to bf16, store; four tokens per pass so that their loads overlap.
 // recv layout: [slot][per][128 channels] fp32; each thread owns 4 consecutive channels.
 template <int NS>
-__device__ __forceinline__ void sum_store(const float* mine, int per, int j0, int j_end, const float (&sc)[4],
+__device__ __forceinline__ void sum_store(uint32_t mine /*shared-space address*/, int per, int j0, int j_end, const float (&sc)[4],
                                           __nv_bfloat16* yrow0, int ldy) {
   for (int j = j0; j < j_end; j += 16) {
     float4 acc[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int jj = min(j + 4 * u, j_end - 1);  // clamped rows are loaded twice and stored once
-      acc[u] = *reinterpret_cast<const float4*>(mine + (size_t)jj * DEC_M);
+      acc[u] = lds_v4f(mine + (uint32_t)(jj * DEC_M * 4));
 #pragma unroll
       for (int r = 1; r < NS; ++r) {
-        const float4 v = *reinterpret_cast<const float4*>(mine + ((size_t)r * per + jj) * DEC_M);
+        const float4 v = lds_v4f(mine + (uint32_t)((r * per + jj) * DEC_M * 4));
         acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
       }
     }
@@ -642,7 +642,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
 #pragma unroll
         for (int i = 0; i < 4; ++i) sc[i] = __half2float(__ldg(p.scale + ch0 + i));
       }
-      const float* mine = recv + 4 * lane;
+      const uint32_t mine = smem_u32(recv + 4 * lane);
       __nv_bfloat16* yrow0 = p.y + (size_t)t0 * p.ldy + ch0;
       const int ldy = p.ldy;
       switch (p.splits) {
