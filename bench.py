@@ -33,7 +33,7 @@ METRIC = "candidate-tokens/sec through q/k/v/o SVD-LoRA projections"
 UNIT = "candidate-tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), keyed by config; None = not captured.
-NCU_TRAFFIC_BYTES = {"2": 172.2e6, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch
+NCU_TRAFFIC_BYTES = {"2": None, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch; 2: kernel changed since the capture
 
 
 def load_peaks():
@@ -230,6 +230,8 @@ def run_ours(args, cfg):
     ctx = binding.Context(local_rank)
     if args.pair_tiles >= 0:
         ctx.set_option(binding.ESSA_OPT_PAIR_TILES, args.pair_tiles)
+    if args.fuse_down >= 0:
+        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, args.fuse_down)
     adapters = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
     offsets = wl.make_segments(cfg)
     T = int(offsets[-1])
@@ -391,6 +393,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--pair-tiles", type=int, default=-1, help="override ESSA_OPT_PAIR_TILES (0 / 1)")
+    ap.add_argument("--fuse-down", type=int, default=-1, help="override ESSA_OPT_FUSE_DOWN (0 / 1)")
     ap.add_argument("--single-calls", action="store_true",
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")

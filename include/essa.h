@@ -74,8 +74,12 @@ const char* essa_last_error(essa_ctx* ctx);
 int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
 /* Scheduling options of a context.
  *   ESSA_OPT_PAIR_TILES (0 / 1): run the base + up step of prefill-sized calls (T >= 512, 256-channel tiles) on
- *   256-token x 256-channel tiles shared by pairs of CTAs (tcgen05 cta_group::2) instead of 128 x 256 tiles per CTA. */
+ *   256-token x 256-channel tiles shared by pairs of CTAs (tcgen05 cta_group::2) instead of 128 x 256 tiles per CTA.
+ *   ESSA_OPT_FUSE_DOWN (0 / 1): on those pair tiles also compute the down-projection and the rank core inside the
+ *   same launch (the tiles of the first channel column produce u for their token rows, the others wait for it),
+ *   instead of a separate rank-down launch that reads x a second time.  Both default to 1. */
 #define ESSA_OPT_PAIR_TILES 1
+#define ESSA_OPT_FUSE_DOWN 2
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

@@ -26,6 +26,7 @@ ESSA_ERR_NO_DEVICE = -6
 ESSA_W0_BF16 = 0
 ESSA_W0_INT8_PERCHANNEL = 1
 ESSA_OPT_PAIR_TILES = 1
+ESSA_OPT_FUSE_DOWN = 2
 
 EXPORTED_SYMBOLS = (
     "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",
@@ -194,7 +195,7 @@ class Context:
         self._check(self.lib.essa_reserve(self.handle, max_tokens, max_d_in, max_d_out))
 
     def set_option(self, option: int, value: int):
-        """essa_set_option (ESSA_OPT_PAIR_TILES = 1)."""
+        """essa_set_option (ESSA_OPT_PAIR_TILES = 1, ESSA_OPT_FUSE_DOWN = 2)."""
         self._check(self.lib.essa_set_option(self.handle, option, value))
 
     def reserve_dequant(self, max_d_in: int, max_d_out: int):

@@ -176,6 +176,7 @@ int32_t essa_destroy(essa_ctx* ctx) {
   free_scratch(ctx->stage_off);
   free_scratch(ctx->stage_sigma);
   free_scratch(ctx->w_deq);
+  free_scratch(ctx->pair_ready);
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->dec_u) cudaFree(ctx->dec_u);
@@ -203,6 +204,8 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
     for (uint32_t& e : ctx->dec_epoch) e = 0;
     for (uint32_t& e : ctx->dec_pepoch) e = 0;
+    if (ctx->pair_ready.ptr) cudaMemset(ctx->pair_ready.ptr, 0, ctx->pair_ready.bytes);
+    ctx->pair_epoch = 0;
   }
   return ESSA_OK;
 }
@@ -211,6 +214,7 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx) return ESSA_ERR_INVALID_ARG;
   switch (option) {
     case ESSA_OPT_PAIR_TILES: ctx->pair_tiles = value != 0; return ESSA_OK;
+    case ESSA_OPT_FUSE_DOWN: ctx->fuse_down = value != 0; return ESSA_OK;
     default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
   }
 }
@@ -307,6 +311,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
     }
     if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q, 1, a->W0q, m, n, n, 128, 64, 0);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
+    if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAtH, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad / 2, 64, 128);
   }
   // The temporaries (and, with host sources, the caller's buffers) are only needed until the copies and the
   // preparation kernels have run.

@@ -32,6 +32,9 @@ struct essa_ctx {
   int32_t* d_status = nullptr;  // device status word
   int64_t launches = 0;         // kernels of this library enqueued through this context
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
+  bool fuse_down = true;        // ... which also compute the down-projection (no rank-down launch)
+  essa::Scratch pair_ready;     // [token tiles][2] uint32: epoch of the last call that published u for (token tile, CTA rank)
+  uint32_t pair_epoch = 0;      // epoch of the latest fused call (grows by one per call)
   // decode schedule: rank-path vector u of one call, [kDecodeMaxTokens][64] bf16, and the count of rows
   // published so far (monotonic across calls; dec_epoch is the host's copy of where the next call starts)
   void* dec_u = nullptr;
@@ -68,6 +71,7 @@ struct essa_adapter {
   CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256 (bf16 storage only)
   CUtensorMap tm_UBp[3][2];
   CUtensorMap tm_VAt;
+  CUtensorMap tm_VAtH;           // the same with boxes of r_pad / 2 rows (one CTA's half in the pair kernel)
   CUtensorMap tm_W0q;            // INT8 storage: the codes, 128-row x 64-byte boxes, unswizzled
 };
 
@@ -112,9 +116,22 @@ int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const 
 void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,
                      essa_plan* out);
 // proj_tc2.cu
+// `down` != nullptr: the launch also computes u (fused down-projection) instead of reading the rank-down launch's.
+struct PairDown {
+  int r_pad, r;
+  const CUtensorMap* tmV;  // V_A^T with boxes of r_pad / 2 rows x 64 columns
+  const int32_t* seg;
+  int P;
+  const float* sigma;
+  int ld_sigma, sA_col, sB_col;
+  const float* M;
+  __nv_bfloat16* u;
+  uint32_t* u_ready;
+  uint32_t u_target;
+};
 int32_t launch_base_up_pair(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2,
                             const CUtensorMap& tmB2a, const CUtensorMap& tmB2b, int T, int d_out, int main_kb, int ext_kb,
-                            int ext_ksteps, __nv_bfloat16* y, const __half* scale, cudaStream_t stream);
+                            int ext_ksteps, __nv_bfloat16* y, const __half* scale, const PairDown* down, cudaStream_t stream);
 // proj_decode.cu
 struct BlockItem {
   const essa_adapter* a;

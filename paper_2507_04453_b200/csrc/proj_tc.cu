@@ -551,6 +551,33 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     if (st != ESSA_OK) return st;
   }
 
+  // ---- fused: the pair-tile launch computes u itself (no rank-down launch, x is read once)
+  // (measured: it pays while every pair takes at most one first-column tile, i.e. up to 74 x 256 tokens; with more
+  // token tiles those tiles, which cannot overlap their epilogue with the next tile, cost more than the launch saved)
+  const bool fused = use_pairs && ctx->fuse_down && (g.T + 255) / 256 <= (ctx->sm_count > 0 ? ctx->sm_count : 148) / 2;
+  PairDown pd{};
+  if (fused) {
+    const int pair_m_tiles = (int)((g.T + 255) / 256);
+    void* before = ctx->pair_ready.ptr;
+    st = ensure_scratch(ctx, ctx->pair_ready, (size_t)pair_m_tiles * 2 * sizeof(uint32_t), true, stream);
+    if (st != ESSA_OK) return st;
+    if (ctx->pair_ready.ptr != before) ctx->pair_epoch = 0;  // a new (zeroed) counter array
+    ctx->pair_epoch += 1;
+    pd.r_pad = a->r_pad;
+    pd.r = a->rank;
+    pd.tmV = &a->tm_VAtH;
+    pd.seg = g.seg_offsets;
+    pd.P = g.P;
+    pd.sigma = g.sigma;
+    pd.ld_sigma = g.ld_sigma;
+    pd.sA_col = g.sA_col;
+    pd.sB_col = g.sB_col;
+    pd.M = a->M;
+    pd.u = u;
+    pd.u_ready = static_cast<uint32_t*>(ctx->pair_ready.ptr);
+    pd.u_target = ctx->pair_epoch;
+  }
+
   // ---- launch 1: rank-down
   KParams kp{};
   kp.T = (int)g.T;
@@ -573,14 +600,16 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   kp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
   kp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
   kp.status = ctx->d_status;
-  switch (a->r_pad) {
-    case 16: st = launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-    case 32: st = launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-    case 48: st = launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-    case 64: st = launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-    default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
+  if (!fused) {
+    switch (a->r_pad) {
+      case 16: st = launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+      case 32: st = launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+      case 48: st = launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+      case 64: st = launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
+      default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
+    }
+    if (st != ESSA_OK) return st;
   }
-  if (st != ESSA_OK) return st;
   if (ev) cudaEventRecord(ev[1], stream);
 
   // ---- launch 2: base contraction + up-projection
@@ -602,7 +631,8 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   if (use_pairs) {
     const CUtensorMap& tmW128 = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? tm_wdeq : a->tm_W0[1];
     st = launch_base_up_pair(ctx, tm_x, tmW128, tm_u, a->tm_UBp[1][0], a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0], (int)g.T,
-                             a->d_out, a->d_in / BLOCK_K, a->ext_blocks, a->r_pad / UMMA_K, g.y, mp.scale, stream);
+                             a->d_out, a->d_in / BLOCK_K, a->ext_blocks, a->r_pad / UMMA_K, g.y, mp.scale, fused ? &pd : nullptr,
+                             stream);
     if (ev) cudaEventRecord(ev[2], stream);
     return st;
   }

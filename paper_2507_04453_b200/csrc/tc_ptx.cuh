@@ -191,6 +191,9 @@ __device__ __forceinline__ void red_release_add_u32(uint32_t* addr, uint32_t v) 
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
 }
 // Order async-proxy (TMA) reads of global memory after this thread's generic-proxy view of it.
+__device__ __forceinline__ void st_release_u32(uint32_t* addr, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 // Make generic-proxy shared-memory writes visible to the async proxy (tcgen05.mma operand reads, TMA).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -162,6 +162,39 @@ def test_scaled_configs_full_outputs(torch, ctx, name):
     case.close()
 
 
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("2", 1024, 256, 16, 4, 700),    # T = 2800: 11 token tiles, ragged last tile
+                                               ("2", 1024, 256, 33, 8, 300),    # padded rank 48
+                                               ("5b", 2048, 512, 64, 16, 128)])  # INT8 storage, rank 64, five stages
+def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, L):
+    """Prefill-sized call on 256-channel tiles: the pair-tile launch that also computes u (default) and the
+    two-launch schedule (ESSA_OPT_FUSE_DOWN = 0) both match the oracle; the fused one is deterministic."""
+    from paper_2507_04453_b200 import binding
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg, projections=[0])
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    plan = binding.plan_projection(dm, dm, r, 1 if cfg.w0_dtype == "int8" else 0, case.T)
+    assert plan["block_n"] == 256 and plan["splits"] == 1 and case.T >= 512  # the shape the pair tiles take
+    x = case.tokens(0)
+    want = case.oracle_projection(0, x)
+    try:
+        outs, counts = {}, {}
+        for fuse in (1, 0):
+            ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, fuse)
+            n0 = ctx.gpu_launches
+            got = case.gpu_projection(0, x, "tc")
+            counts[fuse] = ctx.gpu_launches - n0
+            assert np.isfinite(got).all()
+            assert orc.relative_error(got, want) <= tol, (cfg.name, fuse)
+            outs[fuse] = got
+        assert counts[0] - counts[1] == 1  # the rank-down launch is gone
+        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 1)
+        again = case.gpu_projection(0, x, "tc")
+        assert np.array_equal(again, outs[1])
+    finally:
+        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 1)
+    case.close()
+
+
 @pytest.mark.parametrize("rank", [1, 3, 8, 17, 33, 48, 64])
 def test_rank_padding(torch, ctx, rank):
     cfg = wl.scaled_config("1", d_model=256, d_kv=256, rank=rank, P=5, seg_len=37)
