@@ -33,7 +33,7 @@ METRIC = "candidate-tokens/sec through q/k/v/o SVD-LoRA projections"
 UNIT = "candidate-tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), keyed by config; None = not captured.
-NCU_TRAFFIC_BYTES = {"2": None, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch; 2: kernel changed since the capture
+NCU_TRAFFIC_BYTES = {"2": 299.3e6, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch
 
 
 def load_peaks():

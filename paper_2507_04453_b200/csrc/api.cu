@@ -214,7 +214,10 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx) return ESSA_ERR_INVALID_ARG;
   switch (option) {
     case ESSA_OPT_PAIR_TILES: ctx->pair_tiles = value != 0; return ESSA_OK;
-    case ESSA_OPT_FUSE_DOWN: ctx->fuse_down = value != 0; return ESSA_OK;
+    case ESSA_OPT_FUSE_DOWN:
+      if (value < 0 || value > 2) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_FUSE_DOWN takes 0, 1 or 2");
+      ctx->fuse_down = value;
+      return ESSA_OK;
     default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
   }
 }

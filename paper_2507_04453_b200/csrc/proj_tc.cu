@@ -551,10 +551,14 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     if (st != ESSA_OK) return st;
   }
 
-  // ---- fused: the pair-tile launch computes u itself (no rank-down launch, x is read once)
-  // (measured: it pays while every pair takes at most one first-column tile, i.e. up to 74 x 256 tokens; with more
-  // token tiles those tiles, which cannot overlap their epilogue with the next tile, cost more than the launch saved)
-  const bool fused = use_pairs && ctx->fuse_down && (g.T + 255) / 256 <= (ctx->sm_count > 0 ? ctx->sm_count : 148) / 2;
+  // ---- fused: the pair-tile launch computes u itself (no rank-down launch)
+  // (measured: it pays when the first-column tiles, one per 256 tokens, keep most pairs busy in the first round and
+  // no pair takes two of them: with fewer token tiles the other pairs idle until u appears, with more the
+  // first-column tiles, which cannot overlap their epilogue with the next tile, cost more than the launch saved)
+  const int n_pairs_dev = (ctx->sm_count > 0 ? ctx->sm_count : 148) / 2;
+  const int64_t pair_rows = (g.T + 255) / 256;
+  const bool fused = use_pairs && (ctx->fuse_down == 2 ||
+                                   (ctx->fuse_down == 1 && pair_rows <= n_pairs_dev && 4 * pair_rows >= 3 * n_pairs_dev));
   PairDown pd{};
   if (fused) {
     const int pair_m_tiles = (int)((g.T + 255) / 256);

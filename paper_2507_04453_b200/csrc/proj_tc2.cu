@@ -14,7 +14,7 @@
 // u = sB_k .* (M (sA_k .* p)) for their token rows, store it (bf16) and release-increment a per-(token tile, CTA
 // rank) counter; every producer thread acquires that counter (bounded) before it loads a tile's u slab.  Tiles of
 // the first column wait only for themselves, all other tiles only for first-column tiles, which precede them in
-// every pair's list, so the waits end.  This removes the separate rank-down launch and its second pass over x.
+// every pair's list, so the waits end.  This removes the separate rank-down launch.
 //
 // Warp roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator (+ MMA issuer in the leader),
 // warps 2..5 = epilogue.  Barriers: `full` lives in the leader (one arrive.expect_tx for the bytes of both CTAs;

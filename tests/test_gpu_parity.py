@@ -166,7 +166,7 @@ def test_scaled_configs_full_outputs(torch, ctx, name):
                                                ("2", 1024, 256, 33, 8, 300),    # padded rank 48
                                                ("5b", 2048, 512, 64, 16, 128)])  # INT8 storage, rank 64, five stages
 def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, L):
-    """Prefill-sized call on 256-channel tiles: the pair-tile launch that also computes u (default) and the
+    """Prefill-sized call on 256-channel tiles: the pair-tile launch that also computes u (ESSA_OPT_FUSE_DOWN = 2) and the
     two-launch schedule (ESSA_OPT_FUSE_DOWN = 0) both match the oracle; the fused one is deterministic."""
     from paper_2507_04453_b200 import binding
     cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
@@ -178,7 +178,7 @@ def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, 
     want = case.oracle_projection(0, x)
     try:
         outs, counts = {}, {}
-        for fuse in (1, 0):
+        for fuse in (2, 0):  # 2 = fused at any token count (1, the default, fuses only where it pays)
             ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, fuse)
             n0 = ctx.gpu_launches
             got = case.gpu_projection(0, x, "tc")
@@ -186,10 +186,10 @@ def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, 
             assert np.isfinite(got).all()
             assert orc.relative_error(got, want) <= tol, (cfg.name, fuse)
             outs[fuse] = got
-        assert counts[0] - counts[1] == 1  # the rank-down launch is gone
-        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 1)
+        assert counts[0] - counts[2] == 1  # the rank-down launch is gone
+        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 2)
         again = case.gpu_projection(0, x, "tc")
-        assert np.array_equal(again, outs[1])
+        assert np.array_equal(again, outs[2])
     finally:
         ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 1)
     case.close()
