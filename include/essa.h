@@ -167,7 +167,10 @@ int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_
 /* The same operation with HOST buffers: x, seg_offsets, sigma are copied to the device, the
  * projection runs, y is copied back, and the call returns after `stream` has been synchronised.
  * seg_offsets are validated on the host (ESSA_ERR_INVALID_ARG if not monotone from 0 to T).
- * Pinned host memory makes the copies asynchronous with respect to each other; pageable works. */
+ * Calls of 4096 tokens or more are cut into up to eight chunks of whole candidates (candidates are independent)
+ * that run as a three-stage pipeline: copies in on one internal stream, projections on `stream`, copies out on
+ * another, so both copy directions and the compute overlap.  Pinned host memory is what makes the copies
+ * asynchronous; pageable memory works, serially. */
 int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* adapter, const void* x_host, int64_t T,
                                    const int32_t* seg_offsets_host, int32_t P, const float* sigma_host,
                                    int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y_host,

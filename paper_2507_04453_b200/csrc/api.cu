@@ -178,6 +178,9 @@ int32_t essa_destroy(essa_ctx* ctx) {
   free_scratch(ctx->w_deq);
   free_scratch(ctx->pair_ready);
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->host_events) cudaEventDestroy(e);
+  if (ctx->host_h2d) cudaStreamDestroy(ctx->host_h2d);
+  if (ctx->host_d2h) cudaStreamDestroy(ctx->host_d2h);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->dec_u) cudaFree(ctx->dec_u);
   if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
@@ -448,18 +451,90 @@ int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* a, const v
   int32_t st;
   if ((st = ensure_scratch(ctx, ctx->stage_x, xb, false, stream)) != ESSA_OK) return st;
   if ((st = ensure_scratch(ctx, ctx->stage_y, yb, false, stream)) != ESSA_OK) return st;
-  if ((st = ensure_scratch(ctx, ctx->stage_off, ob, false, stream)) != ESSA_OK) return st;
   if ((st = ensure_scratch(ctx, ctx->stage_sigma, sb, false, stream)) != ESSA_OK) return st;
-  cudaError_t e = cudaMemcpyAsync(ctx->stage_x.ptr, x_host, xb, cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, seg_host, ob, cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, stream);
+
+  // Chunks of whole candidates, at least kMinChunkTokens tokens each and at most kMaxChunks of them: candidates are
+  // independent, so a chunk is a call of its own on a slice of x, y, the offsets and the table.
+  constexpr int64_t kMinChunkTokens = 2048;
+  constexpr int kMaxChunks = 8;
+  std::vector<int32_t> first;  // first candidate of each chunk, then P
+  first.push_back(0);
+  if (T >= 2 * kMinChunkTokens) {
+    int64_t target = T / kMaxChunks;
+    if (target < kMinChunkTokens) target = kMinChunkTokens;
+    for (int32_t k = 1; k < P; ++k)
+      if ((int64_t)seg_host[k] - seg_host[first.back()] >= target && T - seg_host[k] >= kMinChunkTokens) first.push_back(k);
+  }
+  first.push_back(P);
+  const int n_chunks = (int)first.size() - 1;
+  if ((st = ensure_scratch(ctx, ctx->stage_off, ob + (size_t)n_chunks * 4, false, stream)) != ESSA_OK) return st;
+
+  if (n_chunks == 1) {
+    cudaError_t e = cudaMemcpyAsync(ctx->stage_x.ptr, x_host, xb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, seg_host, ob, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
+    st = essa_apply_projection(ctx, a, ctx->stage_x.ptr, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
+                               static_cast<const float*>(ctx->stage_sigma.ptr), ld_sigma, sA_col, sB_col, ctx->stage_y.ptr,
+                               stream_v);
+    if (st != ESSA_OK) return st;
+    e = cudaMemcpyAsync(y_host, ctx->stage_y.ptr, yb, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    return check_cuda(ctx, e, "apply_projection_host: D2H");
+  }
+
+  // Three-stage pipeline over the chunks: host -> device copies on one stream, the projections on `stream`, device
+  // -> host copies on a third, chained by events, so that a chunk's copies overlap its neighbours' compute and the
+  // two copy directions overlap each other (with pinned host memory).
+  if (!ctx->host_h2d && cudaStreamCreateWithFlags(&ctx->host_h2d, cudaStreamNonBlocking) != cudaSuccess)
+    return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaStreamCreate");
+  if (!ctx->host_d2h && cudaStreamCreateWithFlags(&ctx->host_d2h, cudaStreamNonBlocking) != cudaSuccess)
+    return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaStreamCreate");
+  while (ctx->host_events.size() < (size_t)(2 * kMaxChunks + 1)) {
+    cudaEvent_t ev;
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess)
+      return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaEventCreate");
+    ctx->host_events.push_back(ev);
+  }
+  // per-chunk offsets, rebased to start at 0: chunk c occupies entries [first[c] + c, first[c + 1] + c] of one array
+  std::vector<int32_t> off((size_t)P + n_chunks);
+  for (int c = 0; c < n_chunks; ++c)
+    for (int32_t k = first[c]; k <= first[c + 1]; ++k) off[(size_t)k + c] = seg_host[k] - seg_host[first[c]];
+  cudaError_t e = cudaEventRecord(ctx->host_events[2 * kMaxChunks], stream);  // earlier work on `stream` may still read the staging buffers
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_h2d, ctx->host_events[2 * kMaxChunks], 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, off.data(), off.size() * 4, cudaMemcpyHostToDevice, ctx->host_h2d);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, ctx->host_h2d);
   if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
-  st = essa_apply_projection(ctx, a, ctx->stage_x.ptr, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
-                             static_cast<const float*>(ctx->stage_sigma.ptr), ld_sigma, sA_col, sB_col, ctx->stage_y.ptr,
-                             stream_v);
-  if (st != ESSA_OK) return st;
-  e = cudaMemcpyAsync(y_host, ctx->stage_y.ptr, yb, cudaMemcpyDeviceToHost, stream);
+  const uint8_t* xh = static_cast<const uint8_t*>(x_host);
+  uint8_t* yh = static_cast<uint8_t*>(y_host);
+  uint8_t* xd = static_cast<uint8_t*>(ctx->stage_x.ptr);
+  uint8_t* yd = static_cast<uint8_t*>(ctx->stage_y.ptr);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int64_t t0 = seg_host[first[c]], t1 = seg_host[first[c + 1]];
+    const size_t xo = (size_t)t0 * a->d_in * 2, yo = (size_t)t0 * a->d_out * 2;
+    e = cudaMemcpyAsync(xd + xo, xh + xo, (size_t)(t1 - t0) * a->d_in * 2, cudaMemcpyHostToDevice, ctx->host_h2d);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->host_events[2 * c], ctx->host_h2d);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->host_events[2 * c], 0);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
+    if (t1 > t0) {
+      st = essa_apply_projection(ctx, a, xd + xo, t1 - t0, static_cast<const int32_t*>(ctx->stage_off.ptr) + first[c] + c,
+                                 first[c + 1] - first[c], static_cast<const float*>(ctx->stage_sigma.ptr) + (size_t)first[c] * ld_sigma,
+                                 ld_sigma, sA_col, sB_col, yd + yo, stream_v);
+      if (st != ESSA_OK) {
+        cudaStreamSynchronize(ctx->host_h2d);
+        cudaStreamSynchronize(stream);
+        cudaStreamSynchronize(ctx->host_d2h);
+        return st;
+      }
+    }
+    e = cudaEventRecord(ctx->host_events[2 * c + 1], stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_d2h, ctx->host_events[2 * c + 1], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(yh + yo, yd + yo, (size_t)(t1 - t0) * a->d_out * 2, cudaMemcpyDeviceToHost, ctx->host_d2h);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: D2H");
+  }
+  e = cudaStreamSynchronize(ctx->host_d2h);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->host_h2d);
   return check_cuda(ctx, e, "apply_projection_host: D2H");
 }
 

@@ -51,6 +51,9 @@ struct essa_ctx {
   essa::Scratch simt_buf;     // [T_cap][64] fp32: rank-path vector of the CUDA-core cross-check path
   essa::Scratch stage_x, stage_y, stage_off, stage_sigma;  // device staging of the host-buffer entry point
   essa::Scratch w_deq;        // [d_out][d_in] bf16: INT8 W0 of the current prefill call, dequantised (unscaled) per call
+  // host-buffer entry point: copy streams and per-chunk events of its three-stage pipeline (created on first use)
+  cudaStream_t host_h2d = nullptr, host_d2h = nullptr;
+  std::vector<cudaEvent_t> host_events;
   void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
   // essa_profile_begin/end: three events per recorded call
   bool prof_on = false;

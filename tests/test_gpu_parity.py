@@ -284,6 +284,37 @@ def test_host_buffer_entry_point(torch, ctx):
     case.close()
 
 
+def test_host_buffer_entry_point_pipelined_chunks(torch, ctx):
+    """A call of several thousand tokens is cut into chunks of whole candidates that pipeline copies and compute:
+    ragged segments (some empty), pinned and pageable host memory, all against the oracle and equal to each
+    other up to the last bf16 bit; later calls re-use the staging buffers."""
+    cfg = wl.scaled_config("4", d_model=512, d_kv=128, rank=32, P=40, seg_len=300)  # ragged lengths, T of several thousand
+    case = Case(torch, ctx, cfg, projections=[0])
+    off = case.offsets.copy()
+    off[5] = off[4]            # an empty candidate inside a chunk
+    off[21:23] = off[20]       # ... and two at what would be a chunk boundary
+    assert case.T >= 3 * 2048 and np.all(np.diff(off) >= 0)
+    x = case.tokens(0)
+    sA, sB = cfg.sigma_cols(0)
+    ad = case.adapters[0]
+    want = orc.apply_projection(oracle_weight(ad), ad.U_A, ad.V_A, ad.U_B, ad.V_B, x, off, case.sigma32, sA, sB, ad.rank)
+    xh = torch.from_numpy(x).to(torch.bfloat16)
+    outs = []
+    for pinned in (True, False, True):
+        xin = xh.pin_memory() if pinned else xh.clone()
+        yh = torch.zeros((case.T, ad.d_out), dtype=torch.bfloat16)
+        yh = yh.pin_memory() if pinned else yh
+        ctx.apply_projection_host(case.handles[0], xin, torch.from_numpy(off), torch.from_numpy(case.sigma32), sA, sB, yh)
+        got = yh.float().numpy()
+        assert np.isfinite(got).all()
+        assert orc.relative_error(got, want) <= TOL_BF16
+        outs.append(got)
+    for other in outs[1:]:  # (chunks of this size take the split-K schedule, whose fp32 add order varies: last-bit differences)
+        assert np.max(np.abs(outs[0] - other) / np.maximum(1.0, np.abs(outs[0]))) <= 2.0 ** -7
+    assert ctx.get_status() == 0
+    case.close()
+
+
 def test_argument_validation(torch, ctx):
     from paper_2507_04453_b200.binding import EssaError
     cfg = wl.scaled_config("1", d_model=128, d_kv=128, rank=8, P=2, seg_len=4)
