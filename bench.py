@@ -306,7 +306,7 @@ def run_ours(args, cfg):
     ms_per_step = ms / args.steps
     value = world * T * args.steps / (ms * 1e-3)
 
-    # ---- end to end through the host-buffer entry point (H2D of x/offsets/sigma and D2H of y inside the call)
+    # ---- end to end through the host-buffer entry points (H2D of x/offsets/sigma and D2H of y inside the call)
     xh = [x.pin_memory() for x in xs_host]
     yh = [torch.empty((T, a.d_out), dtype=torch.bfloat16).pin_memory() for a in adapters]
     off_h = torch.from_numpy(offsets).pin_memory()
@@ -316,9 +316,12 @@ def run_ours(args, cfg):
         ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, out=sigma, k_begin=k_begin)
         sig_h.copy_(sigma, non_blocking=True)
         stream.synchronize()
-        for i, h in enumerate(handles):
-            sA, sB = cfg.sigma_cols(i)
-            ctx.apply_projection_host(h, xh[i], off_h, sig_h, sA, sB, yh[i])
+        if args.single_calls:
+            for i, h in enumerate(handles):
+                sA, sB = cfg.sigma_cols(i)
+                ctx.apply_projection_host(h, xh[i], off_h, sig_h, sA, sB, yh[i])
+        else:  # the block's projections in one host call: offsets and the table travel once
+            ctx.apply_block_host(handles, xh, off_h, sig_h, [cfg.sigma_cols(i) for i in range(len(handles))], yh)
 
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     for _ in range(2):
@@ -333,7 +336,7 @@ def run_ours(args, cfg):
         t = torch.tensor([e2e_ms], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
-    h2d = sum(x.numel() * 2 for x in xh) + len(handles) * (off_h.numel() * 4 + sig_h.numel() * 4)
+    h2d = sum(x.numel() * 2 for x in xh) + (len(handles) if args.single_calls else 1) * (off_h.numel() * 4 + sig_h.numel() * 4)
     d2h = sum(y.numel() * 2 for y in yh) + sig_h.numel() * 4
     e2e = {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}

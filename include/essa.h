@@ -175,6 +175,13 @@ int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* adapter, c
                                    const int32_t* seg_offsets_host, int32_t P, const float* sigma_host,
                                    int32_t ld_sigma, int32_t sA_col, int32_t sB_col, void* y_host,
                                    void* stream);
+/* essa_apply_block with HOST buffers (Algorithm 1, line 7, for the projections of a block): items_host[i].x and
+ * .y are host pointers, everything else as in essa_apply_projection_host.  At decode sizes the whole block is
+ * copied in, runs as one essa_apply_block call and is copied out; larger blocks run the three-stage pipeline over
+ * all (projection, chunk) units, so one projection's copy-out overlaps the next one's copy-in. */
+int32_t essa_apply_block_host(essa_ctx* ctx, const essa_block_item* items_host, int32_t n_items, int64_t T,
+                              const int32_t* seg_offsets_host, int32_t P, const float* sigma_host, int32_t ld_sigma,
+                              void* stream);
 
 /* (No counterpart in the paper: an engineering variant of essa_apply_projection.)
  * The same operation, same arguments and same result as essa_apply_projection, for callers that must not

@@ -34,7 +34,7 @@ EXPORTED_SYMBOLS = (
     "essa_sample_population_range", "essa_apply_projection", "essa_apply_projection_host",
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
-    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_set_option",
+    "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
 )
 
 
@@ -92,6 +92,7 @@ def load_library() -> C.CDLL:
         "essa_reserve_dequant": (i32, [vp, i32, i32]),
         "essa_set_option": (i32, [vp, i32, i32]),
         "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
+        "essa_apply_block_host": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -312,6 +313,21 @@ class Context:
                                                  sigma_host.stride(0), sA_col, sB_col, y_host.data_ptr(), _stream(stream))
         self._check(st)
         return y_host
+
+    def apply_block_host(self, adapters, xs_host, seg_offsets_host, sigma_host, cols, ys_host, stream=None):
+        """essa_apply_block_host: apply_block with host tensors (bf16 x per projection, int32 offsets, fp32 sigma) and
+        host bf16 outputs."""
+        T = xs_host[0].shape[0]
+        P = seg_offsets_host.numel() - 1
+        n = len(adapters)
+        arr = (BlockItem * n)()
+        for i in range(n):
+            arr[i] = BlockItem(adapters[i].handle, xs_host[i].data_ptr() if T else None, cols[i][0], cols[i][1],
+                               ys_host[i].data_ptr() if T else None)
+        st = self.lib.essa_apply_block_host(self.handle, arr, n, T, seg_offsets_host.data_ptr(), P, sigma_host.data_ptr(),
+                                            sigma_host.stride(0), _stream(stream))
+        self._check(st)
+        return ys_host
 
     def profile_begin(self, max_calls: int):
         """essa_profile_begin: record per-kernel CUDA events inside the following apply_projection calls."""

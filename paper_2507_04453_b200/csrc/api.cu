@@ -434,23 +434,31 @@ int32_t essa_apply_projection_simt(essa_ctx* ctx, const essa_adapter* a, const v
   return launch_projection_simt(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 
-int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* a, const void* x_host, int64_t T,
-                                   const int32_t* seg_host, int32_t P, const float* sigma_host, int32_t ld_sigma,
-                                   int32_t sA_col, int32_t sB_col, void* y_host, void* stream_v) {
+// Host-buffer calls: n projections over the same tokens, segments and table; items[i].x / .y are HOST pointers.
+static int32_t host_pipeline(essa_ctx* ctx, const essa_block_item* items, int32_t n, int64_t T, const int32_t* seg_host,
+                             int32_t P, const float* sigma_host, int32_t ld_sigma, void* stream_v, const char* who) {
   if (!ctx) return ESSA_ERR_INVALID_ARG;
-  if (!a) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: adapter is NULL");
-  if (T < 0 || P < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: negative T or P");
+  if (!items || n < 1 || n > ESSA_MAX_BLOCK_ITEMS) return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": 1 .. ESSA_MAX_BLOCK_ITEMS items expected");
+  if (T < 0 || P < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": negative T or P");
+  for (int32_t i = 0; i < n; ++i)
+    if (!items[i].adapter) return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": adapter is NULL");
   if (T == 0) return ESSA_OK;
-  if (!x_host || !seg_host || !sigma_host || !y_host || P == 0)
-    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: NULL buffer or no candidates");
+  if (!seg_host || !sigma_host || P == 0) return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": NULL buffer or no candidates");
+  for (int32_t i = 0; i < n; ++i)
+    if (!items[i].x || !items[i].y) return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": NULL buffer or no candidates");
   if (essa_validate_segments(seg_host, P, T) != ESSA_OK)
-    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_projection_host: seg_offsets must rise from 0 to T");
+    return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": seg_offsets must rise from 0 to T");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  const size_t xb = (size_t)T * a->d_in * 2, yb = (size_t)T * a->d_out * 2, ob = (size_t)(P + 1) * 4,
-               sb = (size_t)P * ld_sigma * 4;
+  // staging: the items' x (and y) one after the other, each 256-byte aligned
+  size_t x_off[ESSA_MAX_BLOCK_ITEMS + 1] = {0}, y_off[ESSA_MAX_BLOCK_ITEMS + 1] = {0};
+  for (int32_t i = 0; i < n; ++i) {
+    x_off[i + 1] = x_off[i] + (((size_t)T * items[i].adapter->d_in * 2 + 255) & ~(size_t)255);
+    y_off[i + 1] = y_off[i] + (((size_t)T * items[i].adapter->d_out * 2 + 255) & ~(size_t)255);
+  }
+  const size_t ob = (size_t)(P + 1) * 4, sb = (size_t)P * ld_sigma * 4;
   int32_t st;
-  if ((st = ensure_scratch(ctx, ctx->stage_x, xb, false, stream)) != ESSA_OK) return st;
-  if ((st = ensure_scratch(ctx, ctx->stage_y, yb, false, stream)) != ESSA_OK) return st;
+  if ((st = ensure_scratch(ctx, ctx->stage_x, x_off[n], false, stream)) != ESSA_OK) return st;
+  if ((st = ensure_scratch(ctx, ctx->stage_y, y_off[n], false, stream)) != ESSA_OK) return st;
   if ((st = ensure_scratch(ctx, ctx->stage_sigma, sb, false, stream)) != ESSA_OK) return st;
 
   // Chunks of whole candidates, at least kMinChunkTokens tokens each and at most kMaxChunks of them: candidates are
@@ -468,74 +476,96 @@ int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* a, const v
   first.push_back(P);
   const int n_chunks = (int)first.size() - 1;
   if ((st = ensure_scratch(ctx, ctx->stage_off, ob + (size_t)n_chunks * 4, false, stream)) != ESSA_OK) return st;
+  uint8_t* xd = static_cast<uint8_t*>(ctx->stage_x.ptr);
+  uint8_t* yd = static_cast<uint8_t*>(ctx->stage_y.ptr);
 
   if (n_chunks == 1) {
-    cudaError_t e = cudaMemcpyAsync(ctx->stage_x.ptr, x_host, xb, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, seg_host, ob, cudaMemcpyHostToDevice, stream);
+    // small call (decode sizes among them): everything in, one device call for the block, everything out
+    cudaError_t e = cudaMemcpyAsync(ctx->stage_off.ptr, seg_host, ob, cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, stream);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
-    st = essa_apply_projection(ctx, a, ctx->stage_x.ptr, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
-                               static_cast<const float*>(ctx->stage_sigma.ptr), ld_sigma, sA_col, sB_col, ctx->stage_y.ptr,
-                               stream_v);
+    essa_block_item dev[ESSA_MAX_BLOCK_ITEMS];
+    for (int32_t i = 0; i < n && e == cudaSuccess; ++i) {
+      e = cudaMemcpyAsync(xd + x_off[i], items[i].x, (size_t)T * items[i].adapter->d_in * 2, cudaMemcpyHostToDevice, stream);
+      dev[i] = essa_block_item{items[i].adapter, xd + x_off[i], items[i].sA_col, items[i].sB_col, yd + y_off[i]};
+    }
+    if (e != cudaSuccess) return check_cuda(ctx, e, "host call: H2D");
+    st = essa_apply_block(ctx, dev, n, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
+                          static_cast<const float*>(ctx->stage_sigma.ptr), ld_sigma, stream_v);
     if (st != ESSA_OK) return st;
-    e = cudaMemcpyAsync(y_host, ctx->stage_y.ptr, yb, cudaMemcpyDeviceToHost, stream);
+    for (int32_t i = 0; i < n && e == cudaSuccess; ++i)
+      e = cudaMemcpyAsync(items[i].y, yd + y_off[i], (size_t)T * items[i].adapter->d_out * 2, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-    return check_cuda(ctx, e, "apply_projection_host: D2H");
+    return check_cuda(ctx, e, "host call: D2H");
   }
 
-  // Three-stage pipeline over the chunks: host -> device copies on one stream, the projections on `stream`, device
-  // -> host copies on a third, chained by events, so that a chunk's copies overlap its neighbours' compute and the
-  // two copy directions overlap each other (with pinned host memory).
+  // Three-stage pipeline over (projection, chunk) units: host -> device copies on one stream, the projections on
+  // `stream`, device -> host copies on a third, chained by events, so that a unit's copies overlap its neighbours'
+  // compute and the two copy directions overlap each other (with pinned host memory).
   if (!ctx->host_h2d && cudaStreamCreateWithFlags(&ctx->host_h2d, cudaStreamNonBlocking) != cudaSuccess)
-    return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaStreamCreate");
+    return check_cuda(ctx, cudaGetLastError(), "host call: cudaStreamCreate");
   if (!ctx->host_d2h && cudaStreamCreateWithFlags(&ctx->host_d2h, cudaStreamNonBlocking) != cudaSuccess)
-    return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaStreamCreate");
-  while (ctx->host_events.size() < (size_t)(2 * kMaxChunks + 1)) {
+    return check_cuda(ctx, cudaGetLastError(), "host call: cudaStreamCreate");
+  const size_t n_events = (size_t)2 * kMaxChunks * ESSA_MAX_BLOCK_ITEMS + 1;
+  while (ctx->host_events.size() < n_events) {
     cudaEvent_t ev;
     if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess)
-      return check_cuda(ctx, cudaGetLastError(), "apply_projection_host: cudaEventCreate");
+      return check_cuda(ctx, cudaGetLastError(), "host call: cudaEventCreate");
     ctx->host_events.push_back(ev);
   }
   // per-chunk offsets, rebased to start at 0: chunk c occupies entries [first[c] + c, first[c + 1] + c] of one array
   std::vector<int32_t> off((size_t)P + n_chunks);
   for (int c = 0; c < n_chunks; ++c)
     for (int32_t k = first[c]; k <= first[c + 1]; ++k) off[(size_t)k + c] = seg_host[k] - seg_host[first[c]];
-  cudaError_t e = cudaEventRecord(ctx->host_events[2 * kMaxChunks], stream);  // earlier work on `stream` may still read the staging buffers
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_h2d, ctx->host_events[2 * kMaxChunks], 0);
+  cudaError_t e = cudaEventRecord(ctx->host_events[n_events - 1], stream);  // earlier work on `stream` may still read the staging buffers
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_h2d, ctx->host_events[n_events - 1], 0);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_off.ptr, off.data(), off.size() * 4, cudaMemcpyHostToDevice, ctx->host_h2d);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, ctx->host_h2d);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
-  const uint8_t* xh = static_cast<const uint8_t*>(x_host);
-  uint8_t* yh = static_cast<uint8_t*>(y_host);
-  uint8_t* xd = static_cast<uint8_t*>(ctx->stage_x.ptr);
-  uint8_t* yd = static_cast<uint8_t*>(ctx->stage_y.ptr);
-  for (int c = 0; c < n_chunks; ++c) {
-    const int64_t t0 = seg_host[first[c]], t1 = seg_host[first[c + 1]];
-    const size_t xo = (size_t)t0 * a->d_in * 2, yo = (size_t)t0 * a->d_out * 2;
-    e = cudaMemcpyAsync(xd + xo, xh + xo, (size_t)(t1 - t0) * a->d_in * 2, cudaMemcpyHostToDevice, ctx->host_h2d);
-    if (e == cudaSuccess) e = cudaEventRecord(ctx->host_events[2 * c], ctx->host_h2d);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->host_events[2 * c], 0);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: H2D");
-    if (t1 > t0) {
-      st = essa_apply_projection(ctx, a, xd + xo, t1 - t0, static_cast<const int32_t*>(ctx->stage_off.ptr) + first[c] + c,
-                                 first[c + 1] - first[c], static_cast<const float*>(ctx->stage_sigma.ptr) + (size_t)first[c] * ld_sigma,
-                                 ld_sigma, sA_col, sB_col, yd + yo, stream_v);
-      if (st != ESSA_OK) {
-        cudaStreamSynchronize(ctx->host_h2d);
-        cudaStreamSynchronize(stream);
-        cudaStreamSynchronize(ctx->host_d2h);
-        return st;
+  if (e != cudaSuccess) return check_cuda(ctx, e, "host call: H2D");
+  auto drain = [&]() {
+    cudaStreamSynchronize(ctx->host_h2d);
+    cudaStreamSynchronize(stream);
+    cudaStreamSynchronize(ctx->host_d2h);
+  };
+  int unit = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const essa_adapter* a = items[i].adapter;
+    const uint8_t* xh = static_cast<const uint8_t*>(items[i].x);
+    uint8_t* yh = static_cast<uint8_t*>(items[i].y);
+    for (int c = 0; c < n_chunks; ++c, ++unit) {
+      const int64_t t0 = seg_host[first[c]], t1 = seg_host[first[c + 1]];
+      const size_t xo = (size_t)t0 * a->d_in * 2, yo = (size_t)t0 * a->d_out * 2;
+      e = cudaMemcpyAsync(xd + x_off[i] + xo, xh + xo, (size_t)(t1 - t0) * a->d_in * 2, cudaMemcpyHostToDevice, ctx->host_h2d);
+      if (e == cudaSuccess) e = cudaEventRecord(ctx->host_events[2 * unit], ctx->host_h2d);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->host_events[2 * unit], 0);
+      if (e != cudaSuccess) { drain(); return check_cuda(ctx, e, "host call: H2D"); }
+      if (t1 > t0) {
+        st = essa_apply_projection(ctx, a, xd + x_off[i] + xo, t1 - t0, static_cast<const int32_t*>(ctx->stage_off.ptr) + first[c] + c,
+                                   first[c + 1] - first[c], static_cast<const float*>(ctx->stage_sigma.ptr) + (size_t)first[c] * ld_sigma,
+                                   ld_sigma, items[i].sA_col, items[i].sB_col, yd + y_off[i] + yo, stream_v);
+        if (st != ESSA_OK) { drain(); return st; }
       }
+      e = cudaEventRecord(ctx->host_events[2 * unit + 1], stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_d2h, ctx->host_events[2 * unit + 1], 0);
+      if (e == cudaSuccess) e = cudaMemcpyAsync(yh + yo, yd + y_off[i] + yo, (size_t)(t1 - t0) * a->d_out * 2, cudaMemcpyDeviceToHost, ctx->host_d2h);
+      if (e != cudaSuccess) { drain(); return check_cuda(ctx, e, "host call: D2H"); }
     }
-    e = cudaEventRecord(ctx->host_events[2 * c + 1], stream);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->host_d2h, ctx->host_events[2 * c + 1], 0);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(yh + yo, yd + yo, (size_t)(t1 - t0) * a->d_out * 2, cudaMemcpyDeviceToHost, ctx->host_d2h);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "apply_projection_host: D2H");
   }
   e = cudaStreamSynchronize(ctx->host_d2h);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->host_h2d);
-  return check_cuda(ctx, e, "apply_projection_host: D2H");
+  return check_cuda(ctx, e, "host call: D2H");
+}
+
+int32_t essa_apply_projection_host(essa_ctx* ctx, const essa_adapter* a, const void* x_host, int64_t T,
+                                   const int32_t* seg_host, int32_t P, const float* sigma_host, int32_t ld_sigma,
+                                   int32_t sA_col, int32_t sB_col, void* y_host, void* stream_v) {
+  const essa_block_item item{a, x_host, sA_col, sB_col, y_host};
+  return host_pipeline(ctx, &item, 1, T, seg_host, P, sigma_host, ld_sigma, stream_v, "apply_projection_host");
+}
+
+int32_t essa_apply_block_host(essa_ctx* ctx, const essa_block_item* items_host, int32_t n_items, int64_t T,
+                              const int32_t* seg_host, int32_t P, const float* sigma_host, int32_t ld_sigma, void* stream_v) {
+  return host_pipeline(ctx, items_host, n_items, T, seg_host, P, sigma_host, ld_sigma, stream_v, "apply_block_host");
 }
 
 int32_t essa_plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count,

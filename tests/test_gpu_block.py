@@ -95,3 +95,26 @@ def test_block_full_size(torch, ctx, name, max_cands):
         ref = ctx.apply_projection_simt(case.handles[i], xs[i], case.d_offsets, case.d_sigma, *cfg.sigma_cols(i))
         assert orc.relative_error(ys[i].float().cpu().numpy(), ref.float().cpu().numpy().astype(np.float64)) <= tol
     case.close()
+
+
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 1024, 192, 16, 200, 1),     # decode sizes: one device call for the block
+                                               ("4", 512, 128, 32, 24, 300)])    # ragged prefill: pipelined (projection, chunk) units
+def test_block_host_entry_point(torch, ctx, base, dm, dkv, r, P, L):
+    """essa_apply_block_host: host buffers in, host buffers out, against the oracle for every projection."""
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    n = len(cfg.projections)
+    xs = [case.tokens(i) for i in range(n)]
+    xh = [torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in xs]
+    yh = [torch.zeros((case.T, case.adapters[i].d_out), dtype=torch.bfloat16).pin_memory() for i in range(n)]
+    cols = [cfg.sigma_cols(i) for i in range(n)]
+    hs = [case.handles[i] for i in range(n)]
+    for _ in range(2):  # the second call re-uses the staging buffers
+        ctx.apply_block_host(hs, xh, torch.from_numpy(case.offsets), torch.from_numpy(case.sigma32), cols, yh)
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    for i in range(n):
+        got = yh[i].float().numpy()
+        assert np.isfinite(got).all()
+        assert orc.relative_error(got, case.oracle_projection(i, xs[i])) <= tol, (cfg.name, cfg.projections[i])
+    assert ctx.get_status() == 0
+    case.close()
