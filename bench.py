@@ -284,7 +284,14 @@ def run_ours(args, cfg):
     barrier()
     sampler = ClockSampler(torch, local_rank)
     launches0 = ctx.gpu_launches
-    ctx.profile_begin(args.steps * len(handles))
+    # Per-launch durations for the roofline come from CUDA events that the library records around every launch.
+    # At prefill sizes they are recorded inside the timed steps (three event records per call are ~1 % of a step).
+    # At decode sizes they would be a fifth of a step, and an event between two kernels also defeats the dependent
+    # launch that lets the decode kernel's set-up overlap the population draw, so there the timed steps run without
+    # them and the same K steps run once more, right after, with them.
+    events_inside = T > 256
+    if events_inside:
+        ctx.profile_begin(args.steps * len(handles))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
     e0.record(stream)
@@ -292,9 +299,14 @@ def run_ours(args, cfg):
         step()
     e1.record(stream)
     barrier()
+    launches = ctx.gpu_launches - launches0
+    if not events_inside:
+        ctx.profile_begin(args.steps * len(handles))
+        for _ in range(args.steps):
+            step()
+        barrier()
     clocks = sampler.stop()
     prof = ctx.profile_end()
-    launches = ctx.gpu_launches - launches0
     ms = e0.elapsed_time(e1)
     if dist is not None:
         t = torch.tensor([ms], device="cuda")
@@ -356,7 +368,7 @@ def run_ours(args, cfg):
         achieved, peak, unit = per_launch / main_s / 1e9, peaks["hbm_gbs"], "GB/s"
     roofline = {"bound": model["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
                 "traffic": None if (decode and not block_call) or args.candidates > 0 or args.pair_tiles == 0
-                           else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc_kernel<BLOCK_N, EPI_STORE> (base + up)",
+                           else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc2_kernel / essa_tc_kernel (base + up; on pair tiles with the down-projection inside when fused)",
                 "peak_source": f"{peak_src} ({('burst bf16' if decode else 'sustained bf16') if unit == 'TFLOP/s' else 'copy'})",
                 "avg_launch_us": main_s * 1e6, "launches_timed": prof["calls"],
                 "rank_down_avg_us": prof["rank_down_ms"] * 1e3 / calls,
@@ -374,6 +386,8 @@ def run_ours(args, cfg):
                                                      "every step streams W0 from HBM",
                            "calls_per_step": "essa_sample_population + 1 x essa_apply_block" if block_call
                                              else f"essa_sample_population + {len(handles)} x essa_apply_projection",
+                           "kernel_timing": "CUDA events around every launch, inside the timed steps" if events_inside
+                                            else "CUDA events around every launch in a second pass of the same steps (not inside the timed steps)",
                            "parallelism": f"dp{world} (candidate-sharded, no data-path collective)"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
         print(json.dumps(line), flush=True)

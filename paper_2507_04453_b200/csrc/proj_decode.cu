@@ -363,6 +363,10 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = is_main ? *tmem_slot : 0u;
+  // Everything up to here (barriers, TMEM, the first tiles of the frozen W0) depends on no earlier kernel and, with
+  // a programmatic dependent launch, overlaps the kernel before this one in the stream (typically the population
+  // draw); x, the singular values, the scratch buffers and y are touched only after this point.
+  grid_dep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer: one thread feeds both rings,
@@ -875,13 +879,15 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see grid_dep_wait in the kernel
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   ctx->launches += 1;
   const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, maps, blk)
                              : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, maps, blk);

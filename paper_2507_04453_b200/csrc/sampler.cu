@@ -2,6 +2,7 @@
 // (Section 3, "Evolutionary optimization": x^(k) ~ N(m_t, sigma_t^2 C_t), regenerable from a seed;
 //  Algorithm 1, line 5).  Philox4x32-10 (Salmon et al., SC'11) + Box-Muller, all in this file.
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace essa {
 namespace {
@@ -44,6 +45,7 @@ __device__ __forceinline__ void normals_block(uint2 key, uint32_t j, uint32_t k,
 // Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
 __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, const float* __restrict__ Dvec, int d,
                                    uint2 key, int k_begin, int k_count, float* __restrict__ sigma_out) {
+  grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
   const int nb = (d + 3) >> 2;
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (idx >= (long long)k_count * nb) return;
@@ -74,6 +76,7 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
                                                                       int k_begin, int k_count,
                                                                       float* __restrict__ sigma_out) {
   extern __shared__ __align__(16) double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
+  grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
   const int nb = (d + 3) >> 2, d4 = nb * 4;
   const int kk0 = blockIdx.x * kCand;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -191,6 +191,11 @@ __device__ __forceinline__ void red_release_add_u32(uint32_t* addr, uint32_t v) 
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
 }
 // Order async-proxy (TMA) reads of global memory after this thread's generic-proxy view of it.
+// Programmatic dependent launch.  grid_dep_wait: block until the grids this launch depends on have completed and
+// their writes are visible (a no-op for a launch without the attribute).  grid_dep_launch: let a dependent launch
+// of the next kernel in the stream start now; whatever it reads from this kernel it reads after its own wait.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void st_release_u32(uint32_t* addr, uint32_t v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
 }
