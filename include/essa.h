@@ -134,6 +134,27 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
                                      const float* Dvec, int32_t d, uint64_t seed, int32_t k_begin,
                                      int32_t k_count, float* sigma_out, void* stream);
 
+/* Top-alpha selection (Section 3, "LoRA + SVD parameterization": only the top-alpha fraction of the singular
+ * values of each factor is exposed to the optimizer; the sensitivity study's caption fixes the rounding:
+ * rank 8 with alpha = 0.1 rounds down to zero trainable values).  With alpha = alpha_num / alpha_den and a table
+ * whose n_factors slices of `rank` columns follow one another, writes the columns of the
+ * floor(alpha * rank) leading entries of every slice to index_out (host, ascending; may be NULL to ask for the
+ * count only) and their number to *count_out.  Integer arithmetic: no rounding of alpha itself. */
+int32_t essa_top_alpha_index(int32_t n_factors, int32_t rank, int32_t alpha_num, int32_t alpha_den, int32_t* index_out,
+                             int32_t* count_out);
+/* Draw a population when only d_t of the d coordinates are optimised (top-alpha selection):
+ *   sigma_out[k][c] = frozen[c] for every column c, then for i < d_t
+ *   sigma_out[k][index[i]] = mean_t[i] + step * sum_j Bfactor_t[i][j] * Dvec_t[j] * z_k[j],
+ * with z_k the d_t-dimensional standard-normal vector of candidate k_begin + k from the shared stream (blocks of
+ * four coordinates of the OPTIMISED vector, as in essa_sample_population).  d_t = 0 gives k_count copies of frozen.
+ *   frozen [d] fp32 dev (the values the other coordinates keep, e.g. the singular values after SFT);
+ *   index [d_t] int32 dev, distinct columns in [0, d) (entries outside the range are skipped);
+ *   mean_t [d_t], Bfactor_t [d_t][d_t] or NULL, Dvec_t [d_t] or NULL: the search distribution over the optimised
+ *   coordinates; sigma_out [k_count][d] fp32 dev (written). */
+int32_t essa_sample_population_masked(essa_ctx* ctx, const float* frozen, const int32_t* index, const float* mean_t,
+                                      float step, const float* Bfactor_t, const float* Dvec_t, int32_t d, int32_t d_t,
+                                      uint64_t seed, int32_t k_begin, int32_t k_count, float* sigma_out, void* stream);
+
 /* Population-batched adapted projection (Algorithm 1 line 7 applied to every candidate's tokens).
  *   x           [T][d_in] bf16 dev: all candidates' tokens stacked; token t belongs to the candidate
  *               k with seg_offsets[k] <= t < seg_offsets[k+1];

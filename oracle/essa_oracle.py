@@ -117,6 +117,29 @@ def sample_population(mean, step: float, Bfactor, Dvec, seed: int, P: int, k_beg
     return mean[None, :] + float(step) * w
 
 
+def top_alpha_index(n_factors: int, rank: int, alpha) -> np.ndarray:
+    """Columns of the optimised singular values when only the top-alpha fraction of each factor's `rank` values is
+    exposed to the optimizer (Section 3, "LoRA + SVD parameterization"); the count per factor is alpha * rank
+    rounded DOWN (the caption of the rank / population / alpha sensitivity figure: rank 8 with alpha = 0.1 leaves
+    zero trainable values).  The table holds the factors' slices one after the other, leading values first."""
+    from fractions import Fraction
+    per = int(Fraction(str(alpha)) * rank // 1)
+    return np.array([f * rank + j for f in range(n_factors) for j in range(per)], dtype=np.int64)
+
+
+def sample_population_masked(frozen, index, mean_t, step: float, Bfactor_t, Dvec_t, seed: int, P: int,
+                             k_begin: int = 0) -> np.ndarray:
+    """sigma[P, d] (fp64) when only the coordinates `index` are optimised: those columns are a draw from
+    N(mean_t, step^2 C_t) taken from the shared stream in the optimised vector's own numbering, every other column
+    keeps its frozen value (Section 3: the rest of the singular values stay as they were after SFT)."""
+    frozen = np.asarray(frozen, dtype=np.float64)
+    sigma = np.tile(frozen[None, :], (P, 1))
+    index = np.asarray(index, dtype=np.int64)
+    if index.size:
+        sigma[:, index] = sample_population(mean_t, step, Bfactor_t, Dvec_t, seed, P, k_begin)
+    return sigma
+
+
 # ---------------------------------------------------------------------------
 # Projection.
 # ---------------------------------------------------------------------------

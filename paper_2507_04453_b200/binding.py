@@ -35,7 +35,25 @@ EXPORTED_SYMBOLS = (
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
     "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
+    "essa_top_alpha_index", "essa_sample_population_masked",
 )
+
+
+def top_alpha_index(n_factors: int, rank: int, alpha) -> list:
+    """essa_top_alpha_index: columns of the floor(alpha * rank) leading entries of each of n_factors slices of `rank`
+    columns.  alpha may be a float, a string or a Fraction; it is turned into an exact ratio of integers first."""
+    from fractions import Fraction
+    fr = alpha if isinstance(alpha, Fraction) else Fraction(str(alpha))
+    lib = load_library()
+    cnt = C.c_int32(0)
+    st = lib.essa_top_alpha_index(n_factors, rank, fr.numerator, fr.denominator, None, C.byref(cnt))
+    if st != ESSA_OK:
+        raise EssaError(st, "top_alpha_index: bad arguments")
+    out = (C.c_int32 * max(cnt.value, 1))()
+    st = lib.essa_top_alpha_index(n_factors, rank, fr.numerator, fr.denominator, out, C.byref(cnt))
+    if st != ESSA_OK:
+        raise EssaError(st, "top_alpha_index: bad arguments")
+    return [int(out[i]) for i in range(cnt.value)]
 
 
 class EssaError(RuntimeError):
@@ -97,6 +115,8 @@ def load_library() -> C.CDLL:
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
         "essa_sample_population_range": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, vp]),
+        "essa_top_alpha_index": (i32, [i32, i32, i32, i32, vp, vp]),
+        "essa_sample_population_masked": (i32, [vp, vp, vp, vp, f32, vp, vp, i32, i32, u64, i32, i32, vp, vp]),
         "essa_apply_projection": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_apply_projection_host": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_apply_projection_simt": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
@@ -245,6 +265,21 @@ class Context:
         else:
             st = self.lib.essa_sample_population_range(self.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec),
                                                        d, seed, k_begin, P, out.data_ptr(), _stream(stream))
+        self._check(st)
+        return out
+
+    def sample_population_masked(self, frozen, index, mean_t, step: float, Bfactor_t, Dvec_t, seed: int, P: int,
+                                 out=None, k_begin: int = 0, stream=None):
+        """essa_sample_population_masked: sigma[P, d] with the columns `index` (int32, device) drawn around mean_t
+        and every other column equal to frozen."""
+        torch = self.torch
+        d = frozen.numel()
+        d_t = 0 if index is None else index.numel()
+        if out is None:
+            out = torch.empty((P, d), dtype=torch.float32, device=self.device)
+        st = self.lib.essa_sample_population_masked(self.handle, frozen.data_ptr(), _ptr(index) if d_t else None,
+                                                    _ptr(mean_t) if d_t else None, step, _ptr(Bfactor_t), _ptr(Dvec_t),
+                                                    d, d_t, seed, k_begin, P, out.data_ptr(), _stream(stream))
         self._check(st)
         return out
 

@@ -356,7 +356,7 @@ int32_t essa_sample_population(essa_ctx* ctx, const float* mean, float step, con
                                int32_t d, uint64_t seed, int32_t P, float* sigma_out, void* stream) {
   const int32_t st = validate_sampler(ctx, mean, d, 0, P, sigma_out);
   if (st != ESSA_OK) return st;
-  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, 0, P, sigma_out, static_cast<cudaStream_t>(stream));
+  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, 0, P, nullptr, d, sigma_out, static_cast<cudaStream_t>(stream));
 }
 
 int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float step, const float* Bfactor,
@@ -364,8 +364,34 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
                                      float* sigma_out, void* stream) {
   const int32_t st = validate_sampler(ctx, mean, d, k_begin, k_count, sigma_out);
   if (st != ESSA_OK) return st;
-  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, k_begin, k_count, sigma_out,
+  return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, k_begin, k_count, nullptr, d, sigma_out,
                         static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_top_alpha_index(int32_t n_factors, int32_t rank, int32_t alpha_num, int32_t alpha_den, int32_t* index_out,
+                             int32_t* count_out) {
+  if (n_factors < 0 || rank < 1 || alpha_den < 1 || alpha_num < 0 || alpha_num > alpha_den || !count_out) return ESSA_ERR_INVALID_ARG;
+  const int32_t per = (int32_t)(((int64_t)alpha_num * rank) / alpha_den);  // floor(alpha * rank), exactly
+  *count_out = n_factors * per;
+  if (index_out)
+    for (int32_t f = 0; f < n_factors; ++f)
+      for (int32_t j = 0; j < per; ++j) index_out[(size_t)f * per + j] = f * rank + j;
+  return ESSA_OK;
+}
+
+int32_t essa_sample_population_masked(essa_ctx* ctx, const float* frozen, const int32_t* index, const float* mean_t, float step,
+                                      const float* Bfactor_t, const float* Dvec_t, int32_t d, int32_t d_t, uint64_t seed,
+                                      int32_t k_begin, int32_t k_count, float* sigma_out, void* stream_v) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (d < 1 || d_t < 0 || d_t > d || k_begin < 0 || k_count < 0)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population_masked: need 0 <= d_t <= d, d >= 1, k_begin >= 0, k_count >= 0");
+  if (k_count == 0) return ESSA_OK;
+  if (!frozen || !sigma_out || (d_t > 0 && (!index || !mean_t)))
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_population_masked: NULL buffer");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  const int32_t st = launch_fill_rows(ctx, frozen, d, k_count, sigma_out, stream);
+  if (st != ESSA_OK || d_t == 0) return st;
+  return launch_sampler(ctx, mean_t, step, Bfactor_t, Dvec_t, d_t, seed, k_begin, k_count, index, d, sigma_out, stream);
 }
 
 int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* x, int64_t T, const int32_t* seg,

@@ -44,7 +44,8 @@ __device__ __forceinline__ void normals_block(uint2 key, uint32_t j, uint32_t k,
 
 // Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
 __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, const float* __restrict__ Dvec, int d,
-                                   uint2 key, int k_begin, int k_count, float* __restrict__ sigma_out) {
+                                   uint2 key, int k_begin, int k_count, const int32_t* __restrict__ index, int ld_out,
+                                   float* __restrict__ sigma_out) {
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
   const int nb = (d + 3) >> 2;
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
@@ -57,7 +58,8 @@ __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, c
     const int i = 4 * j + e;
     if (i < d) {
       const double w = Dvec ? (double)Dvec[i] * zz[e] : zz[e];
-      sigma_out[(size_t)kk * d + i] = (float)((double)mean[i] + (double)step * w);
+      const int col = index ? index[i] : i;  // top-alpha: coordinate i of the optimised vector sits in column index[i]
+      if (col >= 0 && col < ld_out) sigma_out[(size_t)kk * ld_out + col] = (float)((double)mean[i] + (double)step * w);
     }
   }
 }
@@ -74,6 +76,7 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
                                                                       const float* __restrict__ Bfactor,
                                                                       const float* __restrict__ Dvec, int d, uint2 key,
                                                                       int k_begin, int k_count,
+                                                                      const int32_t* __restrict__ index, int ld_out,
                                                                       float* __restrict__ sigma_out) {
   extern __shared__ __align__(16) double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
@@ -148,9 +151,12 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
   }
   if (live && q == 0) {
     const double mi = (double)mean[i];
+    const int col = index ? index[i] : i;
+    if (col >= 0 && col < ld_out) {
 #pragma unroll
-    for (int c = 0; c < kCand; ++c)
-      if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * d + i] = (float)(mi + (double)step * acc[c]);
+      for (int c = 0; c < kCand; ++c)
+        if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * ld_out + col] = (float)(mi + (double)step * acc[c]);
+    }
   }
 }
 
@@ -174,19 +180,35 @@ __global__ void segment_map_kernel(const int32_t* __restrict__ off, int P, int T
 
 inline uint2 key_of(uint64_t seed) { return make_uint2((uint32_t)(seed & 0xffffffffull), (uint32_t)(seed >> 32)); }
 
+// Rows of the table = frozen values everywhere (top-alpha: the coordinates the optimiser does not see).
+__global__ void fill_rows_kernel(const float* __restrict__ frozen, int d, int k_count, float* __restrict__ sigma_out) {
+  const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (idx < (long long)k_count * d) sigma_out[idx] = frozen[idx % d];
+}
+
 }  // namespace
 
+int32_t launch_fill_rows(essa_ctx* ctx, const float* frozen, int32_t d, int32_t k_count, float* sigma_out, cudaStream_t stream) {
+  const long long total = (long long)k_count * d;
+  if (total == 0) return ESSA_OK;
+  fill_rows_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(frozen, d, k_count, sigma_out);
+  ctx->launches += 1;
+  return check_cuda(ctx, cudaGetLastError(), "fill_rows launch");
+}
+
+// index != NULL: coordinate i of the sampled vector is written to column index[i] of rows of ld_out floats.
 int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
-                       uint64_t seed, int32_t k_begin, int32_t k_count, float* sigma_out, cudaStream_t stream) {
-  if (k_count == 0) return ESSA_OK;
+                       uint64_t seed, int32_t k_begin, int32_t k_count, const int32_t* index, int32_t ld_out, float* sigma_out,
+                       cudaStream_t stream) {
+  if (k_count == 0 || d == 0) return ESSA_OK;
   const int nb = (d + 3) / 4;
   if (Bfactor == nullptr) {
     const long long total = (long long)k_count * nb;
     const int threads = 256;
     const long long blocks = (total + threads - 1) / threads;
     if (blocks > 0x7fffffffLL) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: P*d too large");
-    sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count,
-                                                                 sigma_out);
+    sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count, index,
+                                                                 ld_out, sigma_out);
   } else {
     if (d > 4096) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 4096 with a full covariance factor");
     const size_t smem = (size_t)kCand * nb * 4 * sizeof(double);
@@ -197,7 +219,7 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
       if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(sample_full_kernel)");
     }
     dim3 grid((k_count + kCand - 1) / kCand, (d + kRows - 1) / kRows);
-    kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin, k_count,
+    kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin, k_count, index, ld_out,
                                                     sigma_out);
   }
   ctx->launches += 1;

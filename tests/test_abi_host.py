@@ -126,3 +126,15 @@ def test_workload_generator_is_deterministic_and_exact():
     v = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -9], dtype=np.float32)
     assert list(wl.round_to_bf16(v)) == [1.0, 1.0 + 2.0 ** -6, 1.0]
     assert abs(np.linalg.norm(a.V_A.astype(np.float64).T @ a.V_A.astype(np.float64) - np.eye(8))) < 0.05
+
+
+def test_top_alpha_index_host(lib):
+    """essa_top_alpha_index against the paper's stated rounding and the oracle's own count."""
+    from oracle import essa_oracle as orc
+    assert binding.top_alpha_index(8, 8, 0.1) == []                      # rank 8, alpha 0.1: zero trainable values
+    assert binding.top_alpha_index(1, 100, 0.29) == list(range(29))      # exact decimal arithmetic
+    for n_f, r, alpha in [(3, 4, 0.5), (2, 16, 0.3), (8, 16, 1.0), (4, 64, 0.75), (2, 7, "1/3")]:
+        want = orc.top_alpha_index(n_f, r, alpha if alpha != "1/3" else "1/3")
+        assert binding.top_alpha_index(n_f, r, alpha) == [int(v) for v in want]
+    with pytest.raises(binding.EssaError):
+        binding.top_alpha_index(2, 8, 1.5)

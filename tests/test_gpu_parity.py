@@ -98,6 +98,34 @@ def test_sampler_general_cases(torch, ctx):
     assert out.shape == (0, 4)
 
 
+def test_masked_sampler_matches_oracle(torch, ctx):
+    """Top-alpha selection: only some columns of the table are drawn, the rest keep their frozen values."""
+    from paper_2507_04453_b200 import binding
+    rng = np.random.default_rng(21)
+    for n_f, r, alpha, P, full, k_begin in [(8, 16, 0.5, 64, True, 0), (8, 16, 0.25, 33, False, 5), (8, 8, 0.1, 4, True, 0),
+                                            (2, 64, 1.0, 16, True, 0), (6, 33, "1/3", 9, True, 3)]:
+        d = n_f * r
+        idx = orc.top_alpha_index(n_f, r, alpha)
+        assert binding.top_alpha_index(n_f, r, alpha) == [int(v) for v in idx]
+        dt = idx.size
+        frozen = rng.standard_normal(d).astype(np.float32)
+        mean_t = rng.standard_normal(dt).astype(np.float32)
+        Dv = rng.uniform(0.5, 1.5, dt).astype(np.float32)
+        Bf = (rng.standard_normal((dt, dt)) / np.sqrt(max(dt, 1))).astype(np.float32) if full and dt else None
+        seed = (7 << 32) + 13
+        want = orc.sample_population_masked(frozen, idx, mean_t, np.float32(0.32), Bf, Dv, seed, P, k_begin)
+        got = ctx.sample_population_masked(to_dev(torch, frozen), to_dev(torch, idx.astype(np.int32)) if dt else None,
+                                           to_dev(torch, mean_t) if dt else None, 0.32,
+                                           None if Bf is None else to_dev(torch, Bf), to_dev(torch, Dv) if dt else None,
+                                           seed, P, k_begin=k_begin)
+        torch.cuda.synchronize()
+        got = got.cpu().numpy()
+        assert got.shape == (P, d)
+        assert sigma_error(got, want) <= TOL_SIGMA, (n_f, r, alpha)
+        rest = np.setdiff1d(np.arange(d), idx)
+        assert np.array_equal(got[:, rest], np.tile(frozen[rest], (P, 1)))  # frozen columns are bit-exact copies
+
+
 def test_sampler_range_regenerates_any_member(torch, ctx):
     rng = np.random.default_rng(13)
     d, P = 128, 64

@@ -313,3 +313,45 @@ def test_relative_error_metric():
     got = want + np.array([[0.1, 0.0], [0.0, 0.0]])
     rms = math.sqrt(21 / 4)
     assert abs(orc.relative_error(got, want) - 0.1 / rms) < 1e-15
+
+
+# ------------------------------------------------------------------ top-alpha selection (Section 3; sensitivity-figure caption)
+def test_top_alpha_rounds_down_as_the_paper_states():
+    # the paper's own example: rank 8 with alpha = 0.1 leaves zero trainable singular values
+    assert orc.top_alpha_index(8, 8, 0.1).size == 0
+    # decimal fractions are taken exactly: 0.29 * 100 is 29, not floor(28.999999999999996)
+    assert orc.top_alpha_index(1, 100, 0.29).size == 29
+    # alpha = 1: every coordinate, in order; alpha = 0.5 of rank 4 on three factors: the two leading ones of each slice
+    assert np.array_equal(orc.top_alpha_index(3, 4, 1.0), np.arange(12))
+    assert np.array_equal(orc.top_alpha_index(3, 4, 0.5), np.array([0, 1, 4, 5, 8, 9]))
+    assert np.array_equal(orc.top_alpha_index(2, 16, 0.3), np.array([0, 1, 2, 3, 16, 17, 18, 19]))  # floor(4.8) = 4
+
+
+def test_masked_population_special_cases():
+    rng = np.random.default_rng(5)
+    d, P, seed = 24, 7, (3 << 32) + 11
+    frozen = rng.standard_normal(d)
+    # nothing optimised: every candidate is the frozen vector
+    assert np.array_equal(orc.sample_population_masked(frozen, [], None, 0.3, None, None, seed, P), np.tile(frozen, (P, 1)))
+    # everything optimised: the unmasked draw, whatever `frozen` holds
+    mean = rng.standard_normal(d)
+    Bf = rng.standard_normal((d, d)) / 5
+    Dv = rng.uniform(0.5, 1.5, d)
+    full = orc.sample_population(mean, 0.3, Bf, Dv, seed, P)
+    assert np.array_equal(orc.sample_population_masked(frozen, np.arange(d), mean, 0.3, Bf, Dv, seed, P), full)
+    # a proper subset: the optimised columns are the draw of the SMALL problem (its own stream numbering), scattered;
+    # the others are untouched; a permuted index scatters the same draw to the permuted columns
+    idx = orc.top_alpha_index(3, 8, 0.5)          # 12 of 24 columns
+    dt = idx.size
+    small = orc.sample_population(mean[:dt], 0.3, Bf[:dt, :dt], Dv[:dt], seed, P, k_begin=2)
+    got = orc.sample_population_masked(frozen, idx, mean[:dt], 0.3, Bf[:dt, :dt], Dv[:dt], seed, P, k_begin=2)
+    assert np.array_equal(got[:, idx], small)
+    rest = np.setdiff1d(np.arange(d), idx)
+    assert np.array_equal(got[:, rest], np.tile(frozen[rest], (P, 1)))
+    perm = idx[::-1].copy()
+    got_p = orc.sample_population_masked(frozen, perm, mean[:dt], 0.3, Bf[:dt, :dt], Dv[:dt], seed, P, k_begin=2)
+    assert np.array_equal(got_p[:, perm], small)
+    # moments of the optimised columns (diagonal case): mean m_i, standard deviation step * D_i
+    many = orc.sample_population_masked(frozen, idx, mean[:dt], 0.5, None, Dv[:dt], 9, 20000)
+    assert np.allclose(many[:, idx].mean(axis=0), mean[:dt], atol=0.03)
+    assert np.allclose(many[:, idx].std(axis=0), 0.5 * Dv[:dt], rtol=0.03)
