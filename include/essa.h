@@ -134,6 +134,17 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
                                      const float* Dvec, int32_t d, uint64_t seed, int32_t k_begin,
                                      int32_t k_count, float* sigma_out, void* stream);
 
+/* Candidate reconstruction for hand-off to an external inference engine (Algorithm 1, line 7, as the paper's
+ * workers do it: A'_k = U_A diag(sA_k) V_A^T, B'_k = U_B diag(sB_k) V_B^T, the engine then runs W0 + B'_k A'_k).
+ * The projection entry points above never form these matrices; this call does, for candidates
+ * k_begin .. k_begin + k_count - 1 of the table (row k of sigma is candidate k):
+ *   A_out [k_count][rank][d_in] bf16 dev, B_out [k_count][d_out][rank] bf16 dev (either may be NULL to skip it);
+ *   sigma [>= k_begin + k_count][ld_sigma] fp32 dev; sA_col / sB_col as in essa_apply_projection.
+ * fp32 accumulation, one rounding to bf16.  k_count <= 65535 per call. */
+int32_t essa_export_candidates(essa_ctx* ctx, const essa_adapter* adapter, const float* sigma, int32_t ld_sigma,
+                               int32_t sA_col, int32_t sB_col, int32_t k_begin, int32_t k_count, void* A_out, void* B_out,
+                               void* stream);
+
 /* Top-alpha selection (Section 3, "LoRA + SVD parameterization": only the top-alpha fraction of the singular
  * values of each factor is exposed to the optimizer; the sensitivity study's caption fixes the rounding:
  * rank 8 with alpha = 0.1 rounds down to zero trainable values).  With alpha = alpha_num / alpha_den and a table

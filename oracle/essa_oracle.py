@@ -157,12 +157,18 @@ def dequantize_int8(q, scale) -> np.ndarray:
     return np.asarray(q).astype(np.float64) * np.asarray(scale).astype(np.float64)[:, None]
 
 
-def reconstruct_delta_w(U_A, V_A, U_B, V_B, sA, sB) -> np.ndarray:
-    """Dense update of one candidate, as Algorithm 1 line 7 writes it:
-    A' = U_A diag(sA) V_A^T (r x n), B' = U_B diag(sB) V_B^T (m x r), DeltaW = B' A' (m x n)."""
+def reconstruct_factors(U_A, V_A, U_B, V_B, sA, sB):
+    """The two LoRA factors of one candidate, as Algorithm 1 line 7 writes them:
+    A' = U_A diag(sA) V_A^T (r x n), B' = U_B diag(sB) V_B^T (m x r)."""
     U_A, V_A, U_B, V_B = (np.asarray(a, dtype=np.float64) for a in (U_A, V_A, U_B, V_B))
     A_prime = U_A @ np.diag(np.asarray(sA, dtype=np.float64)) @ V_A.T
     B_prime = U_B @ np.diag(np.asarray(sB, dtype=np.float64)) @ V_B.T
+    return A_prime, B_prime
+
+
+def reconstruct_delta_w(U_A, V_A, U_B, V_B, sA, sB) -> np.ndarray:
+    """Dense update of one candidate, as Algorithm 1 line 7 writes it: DeltaW = B' A' (m x n)."""
+    A_prime, B_prime = reconstruct_factors(U_A, V_A, U_B, V_B, sA, sB)
     return B_prime @ A_prime
 
 

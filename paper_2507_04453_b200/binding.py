@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
     "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
-    "essa_top_alpha_index", "essa_sample_population_masked",
+    "essa_top_alpha_index", "essa_sample_population_masked", "essa_export_candidates",
 )
 
 
@@ -116,6 +116,7 @@ def load_library() -> C.CDLL:
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
         "essa_sample_population_range": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, vp]),
         "essa_top_alpha_index": (i32, [i32, i32, i32, i32, vp, vp]),
+        "essa_export_candidates": (i32, [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]),
         "essa_sample_population_masked": (i32, [vp, vp, vp, vp, f32, vp, vp, i32, i32, u64, i32, i32, vp, vp]),
         "essa_apply_projection": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
         "essa_apply_projection_host": (i32, [vp, vp, vp, i64, vp, i32, vp, i32, i32, i32, vp, vp]),
@@ -282,6 +283,18 @@ class Context:
                                                     d, d_t, seed, k_begin, P, out.data_ptr(), _stream(stream))
         self._check(st)
         return out
+
+    def export_candidates(self, adapter, sigma, sA_col: int, sB_col: int, k_begin: int, k_count: int, want_a=True,
+                          want_b=True, stream=None):
+        """essa_export_candidates: (A'[k_count, rank, d_in], B'[k_count, d_out, rank]) bf16 on the device."""
+        torch = self.torch
+        A = torch.empty((k_count, adapter.rank, adapter.d_in), dtype=torch.bfloat16, device=self.device) if want_a else None
+        B = torch.empty((k_count, adapter.d_out, adapter.rank), dtype=torch.bfloat16, device=self.device) if want_b else None
+        st = self.lib.essa_export_candidates(self.handle, adapter.handle, sigma.data_ptr(), sigma.stride(0), sA_col, sB_col,
+                                             k_begin, k_count, _ptr(A) if k_count else None, _ptr(B) if k_count else None,
+                                             _stream(stream))
+        self._check(st)
+        return A, B
 
     # -- projection
     def _proj(self, fn, adapter, x, seg_offsets, sigma, sA_col, sB_col, out, stream):

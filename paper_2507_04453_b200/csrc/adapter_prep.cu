@@ -58,7 +58,116 @@ __global__ void widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* _
   reinterpret_cast<uint4*>(out + i)[1] = o1;
 }
 
+// Candidate reconstruction (Algorithm 1, line 7: A' = U_A diag(sA_k) V_A^T, B' = U_B diag(sB_k) V_B^T), for export to
+// an engine that wants the dense LoRA factors.  CUDA cores: 2 r^2 (n + m) FLOP per candidate against 2 r (n + m)
+// bytes written, i.e. r FLOP per byte; RP = rank rounded up to 16 keeps the per-thread vectors in registers.
+// A'[i][c] = sum_j U_A[i][j] sA[j] V_A[c][j]: one thread per input feature c, blockIdx.y = candidate; a thread scales
+// its row of V_A once and takes the r dot products with the rows of U_A (shared memory, broadcast reads); the stores
+// of a warp are consecutive in c.
+template <int RP>
+__global__ void __launch_bounds__(128) export_a_kernel(const __nv_bfloat16* __restrict__ U_A, const __nv_bfloat16* __restrict__ V_A,
+                                                      int n, int r, const float* __restrict__ sigma, int ld_sigma, int sA_col,
+                                                      int k_begin, __nv_bfloat16* __restrict__ A_out) {
+  __shared__ __align__(16) float ua[RP * RP];
+  __shared__ float sa[RP];
+  const int kk = blockIdx.y;
+  for (int idx = threadIdx.x; idx < RP * RP; idx += blockDim.x) {
+    const int i = idx / RP, j = idx % RP;
+    ua[idx] = (i < r && j < r) ? __bfloat162float(U_A[i * r + j]) : 0.f;
+  }
+  if (threadIdx.x < RP) sa[threadIdx.x] = threadIdx.x < r ? sigma[(size_t)(k_begin + kk) * ld_sigma + sA_col + threadIdx.x] : 0.f;
+  __syncthreads();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= n) return;
+  float w[RP];
+#pragma unroll
+  for (int j = 0; j < RP; ++j) w[j] = j < r ? sa[j] * __bfloat162float(V_A[(size_t)c * r + j]) : 0.f;
+  __nv_bfloat16* out = A_out + (size_t)kk * r * n + c;
+  for (int i = 0; i < r; ++i) {
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < RP; j += 4) {  // one 16-byte broadcast read per four multiply-adds
+      const float4 u4 = *reinterpret_cast<const float4*>(ua + i * RP + j);
+      acc = fmaf(u4.x, w[j], acc);
+      acc = fmaf(u4.y, w[j + 1], acc);
+      acc = fmaf(u4.z, w[j + 2], acc);
+      acc = fmaf(u4.w, w[j + 3], acc);
+    }
+    out[(size_t)i * n] = __float2bfloat16(acc);
+  }
+}
+
+// B'[o][j] = sum_i U_B[o][i] sB[i] V_B[j][i]: one thread per output channel o, blockIdx.y = candidate.  The 128 rows
+// of a block are one contiguous piece of the output: they are staged in shared memory and stored 16 bytes at a time.
+template <int RP>
+__global__ void __launch_bounds__(128) export_b_kernel(const __nv_bfloat16* __restrict__ U_B, const __nv_bfloat16* __restrict__ V_B,
+                                                      int m, int r, const float* __restrict__ sigma, int ld_sigma, int sB_col,
+                                                      int k_begin, __nv_bfloat16* __restrict__ B_out) {
+  __shared__ __align__(16) float vb[RP * RP];
+  __shared__ float sb[RP];
+  __shared__ __align__(16) __nv_bfloat16 tile[128 * RP];  // [row][r], packed
+  const int kk = blockIdx.y;
+  for (int idx = threadIdx.x; idx < RP * RP; idx += blockDim.x) {
+    const int j = idx / RP, i = idx % RP;
+    vb[idx] = (i < r && j < r) ? __bfloat162float(V_B[j * r + i]) : 0.f;
+  }
+  if (threadIdx.x < RP) sb[threadIdx.x] = threadIdx.x < r ? sigma[(size_t)(k_begin + kk) * ld_sigma + sB_col + threadIdx.x] : 0.f;
+  __syncthreads();
+  const int o0 = blockIdx.x * 128;
+  const int o = o0 + threadIdx.x;
+  if (o < m) {
+    float w[RP];
+#pragma unroll
+    for (int i = 0; i < RP; ++i) w[i] = i < r ? sb[i] * __bfloat162float(U_B[(size_t)o * r + i]) : 0.f;
+    for (int j = 0; j < r; ++j) {
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < RP; i += 4) {
+        const float4 v4 = *reinterpret_cast<const float4*>(vb + j * RP + i);
+        acc = fmaf(v4.x, w[i], acc);
+        acc = fmaf(v4.y, w[i + 1], acc);
+        acc = fmaf(v4.z, w[i + 2], acc);
+        acc = fmaf(v4.w, w[i + 3], acc);
+      }
+      tile[threadIdx.x * r + j] = __float2bfloat16(acc);
+    }
+  }
+  __syncthreads();
+  const int rows = min(128, m - o0);
+  const size_t bytes = (size_t)rows * r * 2;  // m is a multiple of 8: a multiple of 16 bytes, and the piece starts 16-byte aligned
+  uint4* dst = reinterpret_cast<uint4*>(B_out + ((size_t)kk * m + o0) * r);
+  const uint4* src = reinterpret_cast<const uint4*>(tile);
+  for (size_t v = threadIdx.x; v < bytes / 16; v += blockDim.x) dst[v] = src[v];
+}
+
 }  // namespace
+
+int32_t launch_export_candidates(essa_ctx* ctx, const essa_adapter* a, const float* sigma, int32_t ld_sigma, int32_t sA_col,
+                                 int32_t sB_col, int32_t k_begin, int32_t k_count, __nv_bfloat16* A_out, __nv_bfloat16* B_out,
+                                 cudaStream_t stream) {
+  if (k_count == 0) return ESSA_OK;
+  if (A_out) {
+    dim3 grid((unsigned)((a->d_in + 127) / 128), (unsigned)k_count);
+    switch (a->r_pad) {
+      case 16: export_a_kernel<16><<<grid, 128, 0, stream>>>(a->U_A, a->V_A, a->d_in, a->rank, sigma, ld_sigma, sA_col, k_begin, A_out); break;
+      case 32: export_a_kernel<32><<<grid, 128, 0, stream>>>(a->U_A, a->V_A, a->d_in, a->rank, sigma, ld_sigma, sA_col, k_begin, A_out); break;
+      case 48: export_a_kernel<48><<<grid, 128, 0, stream>>>(a->U_A, a->V_A, a->d_in, a->rank, sigma, ld_sigma, sA_col, k_begin, A_out); break;
+      default: export_a_kernel<64><<<grid, 128, 0, stream>>>(a->U_A, a->V_A, a->d_in, a->rank, sigma, ld_sigma, sA_col, k_begin, A_out); break;
+    }
+    ctx->launches += 1;
+  }
+  if (B_out) {
+    dim3 grid((unsigned)((a->d_out + 127) / 128), (unsigned)k_count);
+    switch (a->r_pad) {
+      case 16: export_b_kernel<16><<<grid, 128, 0, stream>>>(a->U_B, a->V_B, a->d_out, a->rank, sigma, ld_sigma, sB_col, k_begin, B_out); break;
+      case 32: export_b_kernel<32><<<grid, 128, 0, stream>>>(a->U_B, a->V_B, a->d_out, a->rank, sigma, ld_sigma, sB_col, k_begin, B_out); break;
+      case 48: export_b_kernel<48><<<grid, 128, 0, stream>>>(a->U_B, a->V_B, a->d_out, a->rank, sigma, ld_sigma, sB_col, k_begin, B_out); break;
+      default: export_b_kernel<64><<<grid, 128, 0, stream>>>(a->U_B, a->V_B, a->d_out, a->rank, sigma, ld_sigma, sB_col, k_begin, B_out); break;
+    }
+    ctx->launches += 1;
+  }
+  return check_cuda(ctx, cudaGetLastError(), "export_candidates launch");
+}
 
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream) {
   const size_t threads = (count + 15) / 16;

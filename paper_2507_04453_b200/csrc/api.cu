@@ -279,7 +279,6 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   // memory; a prefill call dequantises them once into the context's scratch before its GEMM.  Either way the fp16
   // per-channel scale is applied to the fp32 accumulator, so the dequantisation is exact.
   const size_t w0_bytes = m * n * 2;
-  __nv_bfloat16 *dUA = nullptr, *dVB = nullptr;
   cudaError_t e = cudaSuccess;
   auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
   if (!int8) alloc(&a->W0, w0_bytes);
@@ -289,8 +288,8 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   alloc((void**)&a->U_B, m * r * 2);
   alloc((void**)&a->V_A, n * r * 2);
   alloc((void**)&a->M, (size_t)kRankPadMax * kRankPadMax * 4);
-  alloc((void**)&dUA, r * r * 2);
-  alloc((void**)&dVB, r * r * 2);
+  alloc((void**)&a->U_A, r * r * 2);
+  alloc((void**)&a->V_B, r * r * 2);
   int32_t st = ESSA_OK;
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -304,9 +303,9 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   if (int8) copy(a->w0_scale, d->w0_scale, m * 2);
   copy(a->U_B, d->U_B, m * r * 2);
   copy(a->V_A, d->V_A, n * r * 2);
-  copy(dUA, d->U_A, r * r * 2);
-  copy(dVB, d->V_B, r * r * 2);
-  if (st == ESSA_OK) st = launch_adapter_prep(ctx, a, dUA, dVB, stream);
+  copy(a->U_A, d->U_A, r * r * 2);
+  copy(a->V_B, d->V_B, r * r * 2);
+  if (st == ESSA_OK) st = launch_adapter_prep(ctx, a, a->U_A, a->V_B, stream);
   if (st == ESSA_OK) {
     const uint32_t rows[3] = {64, 128, 256};
     for (int i = 0; i < 3 && st == ESSA_OK; ++i) {
@@ -319,11 +318,8 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAtH, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad / 2, 64, 128);
   }
-  // The temporaries (and, with host sources, the caller's buffers) are only needed until the copies and the
-  // preparation kernels have run.
+  // With host sources the caller's buffers are only needed until the copies have run.
   if (cudaStreamSynchronize(stream) != cudaSuccess && st == ESSA_OK) st = check_cuda(ctx, cudaGetLastError(), "load_adapter: sync");
-  if (dUA) cudaFree(dUA);
-  if (dVB) cudaFree(dVB);
   if (st != ESSA_OK) {
     essa_free_adapter(ctx, a);
     return st;
@@ -335,7 +331,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
 int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* a) {
   if (!ctx || !a) return ESSA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->M};
+  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->U_A, a->V_B, a->M};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   delete a;
@@ -366,6 +362,20 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
   if (st != ESSA_OK) return st;
   return launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, k_begin, k_count, nullptr, d, sigma_out,
                         static_cast<cudaStream_t>(stream));
+}
+
+int32_t essa_export_candidates(essa_ctx* ctx, const essa_adapter* a, const float* sigma, int32_t ld_sigma, int32_t sA_col,
+                               int32_t sB_col, int32_t k_begin, int32_t k_count, void* A_out, void* B_out, void* stream) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!a) return fail(ctx, ESSA_ERR_INVALID_ARG, "export_candidates: adapter is NULL");
+  if (k_begin < 0 || k_count < 0) return fail(ctx, ESSA_ERR_INVALID_ARG, "export_candidates: negative candidate range");
+  if (k_count == 0) return ESSA_OK;
+  if (!sigma || (!A_out && !B_out)) return fail(ctx, ESSA_ERR_INVALID_ARG, "export_candidates: NULL buffer");
+  if (sA_col < 0 || sB_col < 0 || sA_col + a->rank > ld_sigma || sB_col + a->rank > ld_sigma)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "export_candidates: sigma columns outside the row");
+  if (k_count > 65535) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "export_candidates: more than 65535 candidates in one call");
+  return launch_export_candidates(ctx, a, sigma, ld_sigma, sA_col, sB_col, k_begin, k_count, static_cast<__nv_bfloat16*>(A_out),
+                                  static_cast<__nv_bfloat16*>(B_out), static_cast<cudaStream_t>(stream));
 }
 
 int32_t essa_top_alpha_index(int32_t n_factors, int32_t rank, int32_t alpha_num, int32_t alpha_den, int32_t* index_out,

@@ -70,6 +70,8 @@ struct essa_adapter {
   __nv_bfloat16* UBp = nullptr;  // [ext][d_out][64]: U_B zero-padded to 64 columns; INT8: (U_B/scale) split hi, lo
   __nv_bfloat16* U_B = nullptr;  // [d_out][rank] as given (CUDA-core path)
   __nv_bfloat16* V_A = nullptr;  // [d_in][rank] as given (CUDA-core path)
+  __nv_bfloat16* U_A = nullptr;  // [rank][rank] as given (candidate export)
+  __nv_bfloat16* V_B = nullptr;  // [rank][rank] as given (candidate export)
   float* M = nullptr;            // [64][64] fp32: M = V_B^T U_A zero-padded
   int ext_blocks = 1;            // rank-path K-slabs appended to the base contraction (1 bf16, 2 INT8)
   CUtensorMap tm_W0[3];          // box rows 64 / 128 / 256 (bf16 storage only)
@@ -104,6 +106,10 @@ int32_t launch_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P,
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream);
 int32_t launch_adapter_prep(essa_ctx* ctx, essa_adapter* a, const __nv_bfloat16* U_A, const __nv_bfloat16* V_B,
                             cudaStream_t stream);
+// Reconstructed factors of candidates k_begin .. k_begin + k_count - 1: A_out [k][rank][d_in], B_out [k][d_out][rank] bf16.
+int32_t launch_export_candidates(essa_ctx* ctx, const essa_adapter* a, const float* sigma, int32_t ld_sigma, int32_t sA_col,
+                                 int32_t sB_col, int32_t k_begin, int32_t k_count, __nv_bfloat16* A_out, __nv_bfloat16* B_out,
+                                 cudaStream_t stream);
 
 struct ProjArgs {
   const __nv_bfloat16* x;

@@ -343,6 +343,38 @@ def test_host_buffer_entry_point_pipelined_chunks(torch, ctx):
     case.close()
 
 
+@pytest.mark.parametrize("base,dm,dkv,r,P", [("2", 512, 128, 16, 9), ("4", 640, 128, 33, 5), ("5b", 512, 192, 64, 3)])
+def test_exported_candidates_match_oracle(torch, ctx, base, dm, dkv, r, P):
+    """essa_export_candidates: A'_k and B'_k of a range of candidates against the oracle's reconstruction, and the
+    product B'_k A'_k x against the library's own projection of the same candidate (the two routes to W' x)."""
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=40)
+    case = Case(torch, ctx, cfg, projections=[1])
+    ad = case.adapters[1]
+    sA, sB = cfg.sigma_cols(1)
+    k0, kc = 1, P - 1
+    A, B = ctx.export_candidates(case.handles[1], case.d_sigma, sA, sB, k0, kc)
+    torch.cuda.synchronize()
+    assert A.shape == (kc, ad.rank, ad.d_in) and B.shape == (kc, ad.d_out, ad.rank)
+    A, B = A.float().cpu().numpy(), B.float().cpu().numpy()
+    for kk in range(kc):
+        srow = case.sigma32[k0 + kk].astype(np.float64)
+        wa, wb = orc.reconstruct_factors(ad.U_A, ad.V_A, ad.U_B, ad.V_B, srow[sA:sA + ad.rank], srow[sB:sB + ad.rank])
+        assert orc.relative_error(A[kk], wa) <= 2.0 ** -8, (cfg.name, kk)   # one bf16 rounding of an fp32 sum
+        assert orc.relative_error(B[kk], wb) <= 2.0 ** -8, (cfg.name, kk)
+    # only one of the two outputs
+    A_only, none = ctx.export_candidates(case.handles[1], case.d_sigma, sA, sB, 0, 2, want_b=False)
+    assert none is None and A_only.shape[0] == 2
+    # the exported factors reproduce the library's projection of that candidate's tokens
+    x = case.tokens(1)
+    y = case.gpu_projection(1, x)
+    lo, hi = int(case.offsets[k0]), int(case.offsets[k0 + 1])
+    W0 = oracle_weight(ad)
+    via_export = x[lo:hi].astype(np.float64) @ (W0 + B[0].astype(np.float64) @ A[0].astype(np.float64)).T
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    assert orc.relative_error(y[lo:hi], via_export) <= tol
+    case.close()
+
+
 def test_argument_validation(torch, ctx):
     from paper_2507_04453_b200.binding import EssaError
     cfg = wl.scaled_config("1", d_model=128, d_kv=128, rank=8, P=2, seg_len=4)

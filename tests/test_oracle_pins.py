@@ -355,3 +355,27 @@ def test_masked_population_special_cases():
     many = orc.sample_population_masked(frozen, idx, mean[:dt], 0.5, None, Dv[:dt], 9, 20000)
     assert np.allclose(many[:, idx].mean(axis=0), mean[:dt], atol=0.03)
     assert np.allclose(many[:, idx].std(axis=0), 0.5 * Dv[:dt], rtol=0.03)
+
+
+# ------------------------------------------------------------------ candidate reconstruction (Algorithm 1, line 7)
+def test_reconstructed_factors_round_trip_the_svd():
+    """With the singular values the thin SVD of a LoRA factor produced, the reconstruction is that factor again
+    (library SVD as the independent routine); scaling one singular value scales exactly its rank-one term."""
+    rng = np.random.default_rng(17)
+    m, n, r = 24, 40, 6
+    A = rng.standard_normal((r, n))
+    Bm = rng.standard_normal((m, r))
+    UA, SA, VAt = np.linalg.svd(A, full_matrices=False)    # A = UA diag(SA) VAt, UA r x r, VAt r x n
+    UB, SB, VBt = np.linalg.svd(Bm, full_matrices=False)   # B = UB diag(SB) VBt, UB m x r, VBt r x r
+    A2, B2 = orc.reconstruct_factors(UA, VAt.T, UB, VBt.T, SA, SB)
+    assert np.allclose(A2, A, atol=1e-12) and np.allclose(B2, Bm, atol=1e-12)
+    assert np.allclose(orc.reconstruct_delta_w(UA, VAt.T, UB, VBt.T, SA, SB), Bm @ A, atol=1e-11)
+    s2 = SA.copy(); s2[2] *= 3.0
+    A3, _ = orc.reconstruct_factors(UA, VAt.T, UB, VBt.T, s2, SB)
+    assert np.allclose(A3 - A, 2.0 * SA[2] * np.outer(UA[:, 2], VAt[2, :]), atol=1e-12)
+    # element by element, scalar loops
+    A4 = np.zeros((r, n))
+    for i in range(r):
+        for c in range(n):
+            A4[i, c] = sum(UA[i, j] * SA[j] * VAt[j, c] for j in range(r))
+    assert np.allclose(A4, A2, atol=1e-12)
