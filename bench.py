@@ -33,7 +33,7 @@ METRIC = "candidate-tokens/sec through q/k/v/o SVD-LoRA projections"
 UNIT = "candidate-tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), keyed by config; None = not captured.
-NCU_TRAFFIC_BYTES = {"2": 299.3e6, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch
+NCU_TRAFFIC_BYTES = {"2": 184.4e6, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch
 
 
 def load_peaks():
@@ -367,8 +367,8 @@ def run_ours(args, cfg):
         per_launch = model["bytes_main"] / per_call
         achieved, peak, unit = per_launch / main_s / 1e9, peaks["hbm_gbs"], "GB/s"
     roofline = {"bound": model["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": None if (decode and not block_call) or args.candidates > 0 or args.pair_tiles == 0
-                           else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc2_kernel / essa_tc_kernel (base + up; on pair tiles with the down-projection inside when fused)",
+                "traffic": None if (decode and not block_call) or args.candidates > 0 or args.pair_tiles == 0 or args.fuse_down > 0
+                           else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc2_kernel / essa_tc_kernel (base + up; --fuse-down 1|2 puts the down-projection inside the pair-tile launch)",
                 "peak_source": f"{peak_src} ({('burst bf16' if decode else 'sustained bf16') if unit == 'TFLOP/s' else 'copy'})",
                 "avg_launch_us": main_s * 1e6, "launches_timed": prof["calls"],
                 "rank_down_avg_us": prof["rank_down_ms"] * 1e3 / calls,

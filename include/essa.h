@@ -77,8 +77,10 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   256-token x 256-channel tiles shared by pairs of CTAs (tcgen05 cta_group::2) instead of 128 x 256 tiles per CTA.
  *   ESSA_OPT_FUSE_DOWN (0 / 1 / 2): on those pair tiles also compute the down-projection and the rank core inside
  *   the same launch (the tiles of the first channel column produce u for their token rows, the others wait for it),
- *   instead of a separate rank-down launch: 0 never, 1 when the token count is in the
- *   range where it pays (about 14 K to 19 K tokens on 148 SMs), 2 whenever pair tiles are used.  Both default to 1. */
+ *   instead of a separate rank-down launch: 0 never (the default: the two-launch
+ *   schedule measured within 0-3 % of it and has no waits between CTAs), 1 when the token count is in the range
+ *   where it measured faster (about 14 K to 19 K tokens on 148 SMs), 2 whenever pair tiles are used.
+ *   ESSA_OPT_PAIR_TILES defaults to 1. */
 #define ESSA_OPT_PAIR_TILES 1
 #define ESSA_OPT_FUSE_DOWN 2
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);

@@ -32,8 +32,8 @@ struct essa_ctx {
   int32_t* d_status = nullptr;  // device status word
   int64_t launches = 0;         // kernels of this library enqueued through this context
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
-  int fuse_down = 1;            // ... which also compute the down-projection (no rank-down launch): 0 never, 1 when
-                                // it pays, 2 whenever pair tiles are used
+  int fuse_down = 0;            // ... which also compute the down-projection (no rank-down launch): 0 never (default),
+                                // 1 in the token range where it measured faster, 2 whenever pair tiles are used
   essa::Scratch pair_ready;     // [token tiles][2] uint32: epoch of the last call that published u for (token tile, CTA rank)
   uint32_t pair_epoch = 0;      // epoch of the latest fused call (grows by one per call)
   // decode schedule: rank-path vector u of one call, [kDecodeMaxTokens][64] bf16, and the count of rows

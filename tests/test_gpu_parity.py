@@ -206,7 +206,7 @@ def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, 
     want = case.oracle_projection(0, x)
     try:
         outs, counts = {}, {}
-        for fuse in (2, 0):  # 2 = fused at any token count (1, the default, fuses only where it pays)
+        for fuse in (2, 0):  # 2 = fused at any token count, 0 = the default two-launch schedule
             ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, fuse)
             n0 = ctx.gpu_launches
             got = case.gpu_projection(0, x, "tc")
@@ -219,7 +219,7 @@ def test_pair_tiles_with_fused_down_projection(torch, ctx, base, dm, dkv, r, P, 
         again = case.gpu_projection(0, x, "tc")
         assert np.array_equal(again, outs[2])
     finally:
-        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 1)
+        ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, 0)
     case.close()
 
 
