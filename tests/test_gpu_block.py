@@ -98,7 +98,9 @@ def test_block_full_size(torch, ctx, name, max_cands):
 
 
 @pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 1024, 192, 16, 200, 1),     # decode sizes: one device call for the block
-                                               ("4", 512, 128, 32, 24, 300)])    # ragged prefill: pipelined (projection, chunk) units
+                                               ("5a", 1024, 256, 64, 96, 1),     # ... INT8 storage
+                                               ("4", 512, 128, 32, 24, 300),     # ragged prefill: pipelined (projection, chunk) units
+                                               ("5b", 512, 128, 64, 20, 256)])   # ... INT8 storage: every chunk dequantises W0 again
 def test_block_host_entry_point(torch, ctx, base, dm, dkv, r, P, L):
     """essa_apply_block_host: host buffers in, host buffers out, against the oracle for every projection."""
     cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
