@@ -3,20 +3,27 @@
 
 One step = one pass of the whole hot path over one synthetic batch: draw the population's singular values
 (essa_sample_population) and run the q, k, v, o adapted projections for every candidate's tokens
-(4 x essa_apply_projection).  Metric: candidate-tokens/s (a candidate-token = one token of one candidate
-through all projections of the block).
+(essa_apply_block at decode sizes, 4 x essa_apply_projection otherwise).  Metric: candidate-tokens/s (a
+candidate-token = one token of one candidate through all projections of the block).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
 
-N > 1 is launched with torch.distributed.run (one rank per GPU).  Candidates are independent, so ranks take
-disjoint candidate ranges of an N-times larger population with no data-path collective (weak scaling).
-Rank 0 prints ONE JSON line.
+Without --config the run times the five benchmark workloads (2, 3, 4, 5a, 5b) one after the other in one
+process and prints ONE JSON line: its top-level fields describe the largest single-GPU bf16 workload (config 4)
+and config.per_config holds the same measurements for each of the five.  With --config C only that workload runs.
+
+N > 1: one rank per GPU (the launcher's RANK / LOCAL_RANK / WORLD_SIZE are used when present; otherwise this
+script re-executes itself under torch.distributed.run with N local ranks).  Candidates are independent, so ranks
+take disjoint candidate ranges of an N-times larger population with no data-path collective (weak scaling).
+Rank 0 prints the line.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import subprocess
 import sys
 import threading
 import time
@@ -32,8 +39,34 @@ from paper_2507_04453_b200 import workloads as wl
 METRIC = "candidate-tokens/sec through q/k/v/o SVD-LoRA projections"
 UNIT = "candidate-tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), keyed by config; None = not captured.
-NCU_TRAFFIC_BYTES = {"2": 184.4e6, "3": 67.9e6, "5a": 171.4e6}  # configs 3, 5a: the block launch
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}  # chip figures, printed beside the measured ones
+ALL_CONFIGS = ("2", "3", "4", "5a", "5b")
+HEADLINE = "4"
+L2_BYTES = 126e6
+CSRC = os.path.join(ROOT, "paper_2507_04453_b200", "csrc")
+# DRAM bytes (read + write) per launch of the dominant kernel from the ncu captures summarised under profiles/,
+# with the SHA-256 (first 16 hex digits) of the kernel's source file at capture time: a kernel that has changed
+# since reports "traffic": null until it is captured again.
+NCU_TRAFFIC = {
+    "2": {"bytes": 184.4e6, "source": "proj_tc2.cu", "sha16": "", "profile": "profiles/essa_tc2_kernel_cfg2_prefill.md"},
+    "3": {"bytes": 67.9e6, "source": "proj_decode.cu", "sha16": "", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
+    "5a": {"bytes": 171.4e6, "source": "proj_decode.cu", "sha16": "", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
+}
+
+
+def source_sha16(name):
+    try:
+        with open(os.path.join(CSRC, name), "rb") as f:
+            return hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+
+
+def ncu_traffic(config_key):
+    rec = NCU_TRAFFIC.get(config_key)
+    if rec is None or not rec["sha16"] or source_sha16(rec["source"]) != rec["sha16"]:
+        return None
+    return rec["bytes"]
 
 
 def load_peaks():
@@ -56,20 +89,28 @@ def projection_work(n, m, r, T, P, w_bytes):
     return flops_call, bytes_call, flops_main, bytes_main
 
 
-def block_roofline(cfg, T, peaks, sustained=True):
-    tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * 1e12
-    bw = peaks["hbm_gbs"] * 1e9
+def block_model(cfg, T):
+    """Algorithmic work of the block's projection calls, each bounded by whichever of its FLOPs and bytes is slower
+    at NOMINAL peak ratios (the bound does not depend on which measured peak is used: the configurations are far
+    from the ridge except 3 and 5a, which are HBM-bound by bytes / copy bandwidth vs FLOPs / burst peak)."""
     w = 1 if cfg.w0_dtype == "int8" else 2
-    t_total, fl, by, fl_main, by_main = 0.0, 0.0, 0.0, 0.0, 0.0
-    bound_votes = {"tensor": 0.0, "hbm": 0.0}
+    rows = []
     for _, n, m in cfg.projections:
-        f, b, fm, bm = projection_work(n, m, cfg.rank, T, cfg.P, w)
+        rows.append(projection_work(n, m, cfg.rank, T, cfg.P, w))
+    return rows
+
+
+def block_roofline(cfg, T, tflops, gbs):
+    tf, bw = tflops * 1e12, gbs * 1e9
+    t_total, fl, by, fl_main, by_main = 0.0, 0.0, 0.0, 0.0, 0.0
+    votes = {"tensor": 0.0, "hbm": 0.0}
+    for f, b, fm, bm in block_model(cfg, T):
         t = max(f / tf, b / bw)
-        bound_votes["tensor" if f / tf >= b / bw else "hbm"] += t
+        votes["tensor" if f / tf >= b / bw else "hbm"] += t
         t_total += t
         fl += f; by += b; fl_main += fm; by_main += bm
-    bound = max(bound_votes, key=bound_votes.get)
-    return {"time_s": t_total, "flops": fl, "bytes": by, "flops_main": fl_main, "bytes_main": by_main, "bound": bound}
+    return {"time_s": t_total, "flops": fl, "bytes": by, "flops_main": fl_main, "bytes_main": by_main,
+            "bound": max(votes, key=votes.get)}
 
 
 # ---------------------------------------------------------------------------------------------- clocks
@@ -98,20 +139,23 @@ class ClockSampler:
             self.nv = None
             self.err = repr(e)
 
-    def _run(self):
+    def _sample(self):
         nv = self.nv
+        try:
+            self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+            self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+        except Exception:
+            pass
+
+    def _run(self):
         while not self._stop.is_set():
-            try:
-                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
-                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
-                    else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
-            except Exception:
-                pass
-            time.sleep(0.004)
+            self._sample()
+            time.sleep(0.002)
 
     def start(self):
         if self.nv is not None:
@@ -146,26 +190,44 @@ def oracle_candidates_pass(cfg, adapters, weights, offsets, sigma, xs, cands):
                              candidates=cands)
 
 
-def oracle_setup(cfg):
+def oracle_setup(cfg, max_candidates=None):
+    """Oracle inputs.  Only the tokens of the first max_candidates candidates are generated as fp64 (the timed sample
+    never touches the others, and the full fp64 activations of the largest workloads would not fit host memory)."""
     from oracle import essa_oracle as orc
     adapters = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
     offsets = wl.make_segments(cfg)
     T = int(offsets[-1])
     cma = wl.make_cma_state(cfg, adapters)
     weights = [a.W0.astype(np.float64) if a.w0_dtype == "bf16" else orc.dequantize_int8(a.W0_q, a.W0_scale) for a in adapters]
-    xs = [wl.make_tokens(cfg, i, T).astype(np.float64) for i in range(len(adapters))]
-    return adapters, weights, offsets, T, cma, xs
+    kmax = cfg.P if max_candidates is None else min(cfg.P, max_candidates)
+    t_need = int(offsets[kmax])
+    xs = []
+    for i in range(len(adapters)):
+        x = wl.make_tokens(cfg, i, T)
+        xs.append(np.ascontiguousarray(x[:t_need]).astype(np.float64))
+        del x
+    return adapters, weights, offsets, T, cma, xs, kmax
 
 
-def time_oracle_sample(cfg, budget_s=15.0, prepared=None):
+def warm_blas():
+    """A few fp64 products before timing: the first BLAS calls of a process pay for thread start-up."""
+    a = np.ones((512, 512))
+    for _ in range(3):
+        a = (a @ a) * 1e-3
+
+
+def time_oracle_sample(cfg, budget_s=15.0, max_candidates=32):
     """cpu_baseline: the oracle timed on a bounded sample (whole candidates, in order) of the workload."""
     from oracle import essa_oracle as orc
-    adapters, weights, offsets, T, cma, xs = prepared or oracle_setup(cfg)
+    adapters, weights, offsets, T, cma, xs, kmax = oracle_setup(cfg, max_candidates)
+    warm_blas()
+    oracle_candidates_pass(cfg, adapters, weights, offsets, orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, 1),
+                           xs, [0])  # untimed warm-up pass on one candidate
     t0 = time.perf_counter()
     sigma = orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, cfg.P)
     t_sample = time.perf_counter() - t0
     done_tokens, done_c, elapsed = 0, 0, t_sample
-    for k in range(cfg.P):
+    for k in range(kmax):
         t0 = time.perf_counter()
         oracle_candidates_pass(cfg, adapters, weights, offsets, sigma, xs, [k])
         elapsed += time.perf_counter() - t0
@@ -175,7 +237,8 @@ def time_oracle_sample(cfg, budget_s=15.0, prepared=None):
             break
     return {"value": done_tokens / elapsed, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"first {done_c} of {cfg.P} candidates ({done_tokens} of {T} tokens), all {len(adapters)} projections, "
-                      f"all channels, plus the full population draw; {elapsed:.1f} s"}
+                      f"all channels, plus the full population draw; {elapsed:.1f} s after one untimed warm-up candidate; "
+                      "numpy fp64 with BLAS matrix products"}
 
 
 def run_reference(args, cfg):
@@ -184,14 +247,15 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    prepared = oracle_setup(cfg)
-    adapters, weights, offsets, T, cma, xs = prepared
+    adapters, weights, offsets, T, cma, xs, kmax = oracle_setup(cfg, 32)
+    warm_blas()
     sigma = orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, cfg.P)
+    oracle_candidates_pass(cfg, adapters, weights, offsets, sigma, xs, [0])
     t0 = time.perf_counter()
     oracle_candidates_pass(cfg, adapters, weights, offsets, sigma, xs, [0])
     t1 = max(time.perf_counter() - t0, 1e-4)
     total_steps = args.steps + args.warmup
-    c = int(max(1, min(cfg.P, 100.0 / (total_steps * t1))))  # whole run within a couple of minutes
+    c = int(max(1, min(kmax, 100.0 / (total_steps * t1))))  # whole run within a couple of minutes
     cands = list(range(c))
     tokens = int(offsets[c] - offsets[0])
     for _ in range(args.warmup):
@@ -202,7 +266,8 @@ def run_reference(args, cfg):
         oracle_candidates_pass(cfg, adapters, weights, offsets, sigma, xs, cands)
     dt = time.perf_counter() - t0
     value = tokens * args.steps / dt
-    sample = f"each step: full population draw + first {c} of {cfg.P} candidates ({tokens} of {T} tokens), all projections, all channels"
+    sample = (f"each step: full population draw + first {c} of {cfg.P} candidates ({tokens} of {T} tokens), all projections, "
+              "all channels; numpy fp64 with BLAS matrix products")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -213,19 +278,11 @@ def run_reference(args, cfg):
 
 
 # ---------------------------------------------------------------------------------------------- GPU arm
-def run_ours(args, cfg):
-    import torch
-    from paper_2507_04453_b200 import binding
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    peaks, peak_src = load_peaks()
+def measure_config(key, cfg, args, env):
+    """All measurements of one workload on this rank's GPU; returns the per-config record (max over ranks applied)."""
+    torch, binding, dist = env["torch"], env["binding"], env["dist"]
+    world, rank, local_rank = env["world"], env["rank"], env["local_rank"]
+    peaks, peak_src = env["peaks"], env["peak_src"]
 
     ctx = binding.Context(local_rank)
     if args.pair_tiles >= 0:
@@ -240,28 +297,31 @@ def run_ours(args, cfg):
     # device copies of the block's adapters that each step streams its W0 from HBM, as a forward pass over many
     # layers does.
     w_bytes = sum(a.d_in * a.d_out * (1 if cfg.w0_dtype == 'int8' else 2) for a in adapters)  # as stored
-    L2_BYTES = 126e6
     copies = 1 if w_bytes > 2 * L2_BYTES else int(np.ceil(2 * L2_BYTES / w_bytes)) + 1
     handle_sets = [[ctx.load_adapter(a) for a in adapters] for _ in range(copies)]
     handles = handle_sets[0]
-    dev = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(a))).cuda()
-    xs_host = [torch.from_numpy(wl.make_tokens(cfg, i, T)).to(torch.bfloat16) for i in range(len(adapters))]
+    del adapters[:]  # the host copies of the weights are not needed any more
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    xs_host = []
+    for i in range(len(handles)):
+        xs_host.append(torch.from_numpy(wl.make_tokens(cfg, i, T)).to(torch.bfloat16))
     xs = [x.cuda() for x in xs_host]
-    ys = [torch.empty((T, a.d_out), dtype=torch.bfloat16, device="cuda") for a in adapters]
+    ys = [torch.empty((T, h.d_out), dtype=torch.bfloat16, device="cuda") for h in handles]
     d_off = dev(offsets)
     d_mean = dev(cma.mean)
     d_B = None if cma.Bfactor is None else dev(cma.Bfactor)
     d_D = None if cma.Dvec is None else dev(cma.Dvec)
     sigma = torch.empty((cfg.P, cfg.d), dtype=torch.float32, device="cuda")
     k_begin = rank * cfg.P  # weak scaling: rank g evaluates candidates [g*P, (g+1)*P) of an N*P population
-    ctx.reserve(T, max(a.d_in for a in adapters), max(a.d_out for a in adapters))
+    ctx.reserve(T, max(h.d_in for h in handles), max(h.d_out for h in handles))
     if cfg.w0_dtype == "int8":
-        ctx.reserve_dequant(max(a.d_in for a in adapters), max(a.d_out for a in adapters))
+        ctx.reserve_dequant(max(h.d_in for h in handles), max(h.d_out for h in handles))
     stream = torch.cuda.current_stream()
 
     step_no = [0]
-    cols = [cfg.sigma_cols(i) for i in range(len(adapters))]
-    block_call = T <= 256 and len(adapters) > 1 and not args.single_calls
+    cols = [cfg.sigma_cols(i) for i in range(len(handles))]
+    decode = T <= 256  # one-launch decode schedule (essa_plan.decode)
+    block_call = decode and len(handles) > 1 and not args.single_calls
 
     def step():
         hs = handle_sets[step_no[0] % copies]
@@ -279,7 +339,16 @@ def run_ours(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    def max_over_ranks(v):
+        if dist is None:
+            return v
+        t = torch.tensor([v], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    steps = args.steps
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         step()
     barrier()
     sampler = ClockSampler(torch, local_rank)
@@ -289,38 +358,70 @@ def run_ours(args, cfg):
     # At decode sizes they would be a fifth of a step, and an event between two kernels also defeats the dependent
     # launch that lets the decode kernel's set-up overlap the population draw, so there the timed steps run without
     # them and the same K steps run once more, right after, with them.
-    events_inside = T > 256
+    events_inside = not decode
     if events_inside:
-        ctx.profile_begin(args.steps * len(handles))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ctx.profile_begin(steps * len(handles))
+    # The K timed steps are bracketed by one pair of events (the mean); events between groups of steps (every step
+    # at prefill sizes, every `group` steps at decode sizes, where a step is tens of microseconds) give the spread.
+    group = 1 if not decode else max(1, min(10, steps // 5))
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps // group + 2)]
     sampler.start()
-    e0.record(stream)
-    for _ in range(args.steps):
+    t_host0 = time.perf_counter()
+    marks[0].record(stream)
+    n_marks = 1
+    for s in range(steps):
         step()
-    e1.record(stream)
+        if (s + 1) % group == 0 or s + 1 == steps:
+            marks[n_marks].record(stream)
+            n_marks += 1
+    host_issue_ms = (time.perf_counter() - t_host0) * 1e3  # wall clock of issuing the K steps without synchronising
     barrier()
     launches = ctx.gpu_launches - launches0
+    clocks = sampler.stop()
     if not events_inside:
-        ctx.profile_begin(args.steps * len(handles))
-        for _ in range(args.steps):
+        ctx.profile_begin(steps * len(handles))
+        for _ in range(steps):
             step()
         barrier()
-    clocks = sampler.stop()
     prof = ctx.profile_end()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(marks[0].elapsed_time(marks[n_marks - 1]))
+    per_group = []
+    for g in range(1, n_marks):
+        n_in = group if g * group <= steps else steps - (g - 1) * group
+        per_group.append(marks[g - 1].elapsed_time(marks[g]) / max(n_in, 1))
     status = ctx.get_status()
     if status != 0:
-        raise RuntimeError(f"device status {status} after the timed region")
-    ms_per_step = ms / args.steps
-    value = world * T * args.steps / (ms * 1e-3)
+        raise RuntimeError(f"device status {status} after the timed region of config {key}")
+    ms_per_step = ms / steps
+    value = world * T * steps / (ms * 1e-3)
+
+    # ---- L2-warm regime (decode configurations): the same steps on ONE copy of the weights, which then stay in L2
+    warm_ms = None
+    if copies > 1:
+        hs0 = handle_sets[0]
+
+        def step_warm():
+            ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, out=sigma, k_begin=k_begin)
+            if block_call:
+                ctx.apply_block(hs0, xs, d_off, sigma, cols, outs=ys)
+            else:
+                for i, h in enumerate(hs0):
+                    ctx.apply_projection(h, xs[i], d_off, sigma, cols[i][0], cols[i][1], out=ys[i])
+        for _ in range(3):
+            step_warm()
+        barrier()
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0.record(stream)
+        for _ in range(steps):
+            step_warm()
+        w1.record(stream)
+        barrier()
+        warm_ms = max_over_ranks(w0.elapsed_time(w1)) / steps
 
     # ---- end to end through the host-buffer entry points (H2D of x/offsets/sigma and D2H of y inside the call)
     xh = [x.pin_memory() for x in xs_host]
-    yh = [torch.empty((T, a.d_out), dtype=torch.bfloat16).pin_memory() for a in adapters]
+    del xs_host
+    yh = [torch.empty((T, h.d_out), dtype=torch.bfloat16).pin_memory() for h in handles]
     off_h = torch.from_numpy(offsets).pin_memory()
     sig_h = torch.empty((cfg.P, cfg.d), dtype=torch.float32).pin_memory()
 
@@ -333,9 +434,9 @@ def run_ours(args, cfg):
                 sA, sB = cfg.sigma_cols(i)
                 ctx.apply_projection_host(h, xh[i], off_h, sig_h, sA, sB, yh[i])
         else:  # the block's projections in one host call: offsets and the table travel once
-            ctx.apply_block_host(handles, xh, off_h, sig_h, [cfg.sigma_cols(i) for i in range(len(handles))], yh)
+            ctx.apply_block_host(handles, xh, off_h, sig_h, cols, yh)
 
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_steps = max(1, min(steps, args.e2e_steps))
     for _ in range(2):
         step_e2e()
     barrier()
@@ -343,70 +444,138 @@ def run_ours(args, cfg):
     for _ in range(e2e_steps):
         step_e2e()
     torch.cuda.synchronize()
-    e2e_ms = (time.perf_counter() - t0) * 1e3
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
     h2d = sum(x.numel() * 2 for x in xh) + (len(handles) if args.single_calls else 1) * (off_h.numel() * 4 + sig_h.numel() * 4)
     d2h = sum(y.numel() * 2 for y in yh) + sig_h.numel() * 4
     e2e = {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
 
-    # ---- roofline of the dominant kernel (base contraction + up-projection), timed live by the library's events
-    decode = T <= 256  # one-launch decode schedule (essa_plan.decode)
-    # a kernel inside a long, power-capped step is held against the sustained tensor peak, a short one against the burst peak
-    model = block_roofline(cfg, T, peaks, sustained=not decode)
+    # ---- roofline of the dominant kernel (base contraction + up-projection), timed live by the library's events.
+    # Tensor peak: the sustained figure only if this workload's own clock samples show the power cap, else burst.
+    capped = "sw_power_cap" in clocks.get("reasons", [])
+    tf_key = "bf16_tflops_sustained" if capped else "bf16_tflops"
+    model = block_roofline(cfg, T, peaks[tf_key], peaks["hbm_gbs"])
+    nominal = block_roofline(cfg, T, NOMINAL_PEAKS["bf16_tflops"], NOMINAL_PEAKS["hbm_gbs"])
     calls = max(prof["calls"], 1)
     main_s = prof["base_up_ms"] * 1e-3 / calls  # average launch duration
     per_call = 1 if block_call else len(handles)  # a block call is one launch for all projections
     if model["bound"] == "tensor":
         per_launch = model["flops_main"] / per_call
-        achieved, peak, unit = per_launch / main_s / 1e12, peaks["bf16_tflops" if decode else "bf16_tflops_sustained"], "TFLOP/s"
+        achieved, peak, peak_nom, unit = per_launch / main_s / 1e12, peaks[tf_key], NOMINAL_PEAKS["bf16_tflops"], "TFLOP/s"
+        peak_kind = "sustained bf16 (sw_power_cap sampled during the timed steps)" if capped else "burst bf16 (no power cap sampled)"
     else:
         per_launch = model["bytes_main"] / per_call
-        achieved, peak, unit = per_launch / main_s / 1e9, peaks["hbm_gbs"], "GB/s"
+        achieved, peak, peak_nom, unit = per_launch / main_s / 1e9, peaks["hbm_gbs"], NOMINAL_PEAKS["hbm_gbs"], "GB/s"
+        peak_kind = "copy bandwidth"
+    traffic = None
+    if not ((decode and not block_call) or args.candidates > 0 or args.pair_tiles == 0 or args.fuse_down > 0):
+        traffic = ncu_traffic(key)
+    if decode:
+        kernel = "essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)"
+    else:
+        kernel = "essa_tc2_kernel / essa_tc_kernel (base contraction + up-projection)"
     roofline = {"bound": model["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": None if (decode and not block_call) or args.candidates > 0 or args.pair_tiles == 0 or args.fuse_down > 0
-                           else NCU_TRAFFIC_BYTES.get(args.config), "kernel": ("essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)") if decode else "essa_tc2_kernel / essa_tc_kernel (base + up; --fuse-down 1|2 puts the down-projection inside the pair-tile launch)",
-                "peak_source": f"{peak_src} ({('burst bf16' if decode else 'sustained bf16') if unit == 'TFLOP/s' else 'copy'})",
-                "avg_launch_us": main_s * 1e6, "launches_timed": prof["calls"],
+                "traffic": traffic, "kernel": kernel, "peak_kind": peak_kind, "peak_source": f"{peak_src} ({peak_kind})",
+                "peak_nominal": peak_nom, "frac_of_nominal": achieved / peak_nom,
+                "algorithmic_per_launch": per_launch, "avg_launch_us": main_s * 1e6, "launches_timed": prof["calls"],
                 "rank_down_avg_us": prof["rank_down_ms"] * 1e3 / calls,
-                "block_roofline_us": model["time_s"] * 1e6, "block_frac": model["time_s"] * 1e3 / ms_per_step}
+                "block_roofline_us": model["time_s"] * 1e6, "block_frac": model["time_s"] * 1e3 / ms_per_step,
+                "block_roofline_us_nominal": nominal["time_s"] * 1e6,
+                "block_frac_of_nominal": nominal["time_s"] * 1e3 / ms_per_step}
 
-    if rank == 0:
-        cpu = time_oracle_sample(cfg, budget_s=args.cpu_budget) if world == 1 and not args.no_cpu_baseline else None
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16" if cfg.w0_dtype == "bf16" else "bf16 (int8 weights)", "data": "synthetic",
-                "config": {"workload": cfg.name, "tokens_per_gpu_step": T, "candidates_per_gpu": cfg.P, "rank": cfg.rank,
-                           "projections": [f"{nm}:{n}->{m}" for nm, n, m in cfg.projections],
-                           "l2": "inputs larger than L2 (x, W0 and y of the projections exceed 126 MB per step)"
-                                 if copies == 1 else f"weights rotate through {copies} device copies ({copies * w_bytes / 1e6:.0f} MB > 2 x L2): "
-                                                     "every step streams W0 from HBM",
-                           "calls_per_step": "essa_sample_population + 1 x essa_apply_block" if block_call
-                                             else f"essa_sample_population + {len(handles)} x essa_apply_projection",
-                           "kernel_timing": "CUDA events around every launch, inside the timed steps" if events_inside
-                                            else "CUDA events around every launch in a second pass of the same steps (not inside the timed steps)",
-                           "parallelism": f"dp{world} (candidate-sharded, no data-path collective)"},
-                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
-        print(json.dumps(line), flush=True)
+    rec = {"workload": cfg.name, "tokens_per_gpu_step": T, "candidates_per_gpu": cfg.P, "rank": cfg.rank,
+           "dtype": "bf16" if cfg.w0_dtype == "bf16" else "bf16 (int8 weights)",
+           "projections": [f"{nm}:{n}->{m}" for nm, n, m in cfg.projections],
+           "value": value, "steps": steps, "warmup": warmup,
+           "ms_per_step": ms_per_step, "ms_per_step_median": float(np.median(per_group)), "ms_per_step_min": float(np.min(per_group)),
+           "timing_group": group, "ms_per_step_l2_warm": warm_ms, "host_issue_ms_per_step": host_issue_ms / steps,
+           "l2": "inputs larger than L2 (x, W0 and y of the projections exceed 126 MB per step)"
+                 if copies == 1 else f"weights rotate through {copies} device copies ({copies * w_bytes / 1e6:.0f} MB > 2 x L2): "
+                                     "every step streams W0 from HBM (ms_per_step_l2_warm: one copy, W0 served from L2)",
+           "calls_per_step": "essa_sample_population + 1 x essa_apply_block" if block_call
+                             else f"essa_sample_population + {len(handles)} x essa_apply_projection",
+           "kernel_timing": "CUDA events around every launch, inside the timed steps" if events_inside
+                            else "CUDA events around every launch in a second pass of the same steps (not inside the timed steps)",
+           "roofline": roofline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
     for hs in handle_sets:
         for h in hs:
             h.free()
     ctx.close()
+    del xs, ys, xh, yh
+    torch.cuda.empty_cache()
+    return rec
+
+
+def run_ours(args):
+    import torch
+    from paper_2507_04453_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}")
+    if not torch.cuda.is_available():
+        raise SystemExit(f"bench.py: rank {rank} has no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks, peak_src = load_peaks()
+    env = {"torch": torch, "binding": binding, "dist": dist, "world": world, "rank": rank, "local_rank": local_rank,
+           "peaks": peaks, "peak_src": peak_src}
+
+    keys = [args.config] if args.config else list(ALL_CONFIGS)
+    head_key = args.config if args.config else HEADLINE
+    per_config = {}
+    for key in keys:
+        cfg = wl.CONFIGS[key]
+        if args.candidates > 0:
+            import dataclasses
+            cfg = dataclasses.replace(cfg, P=args.candidates, name=f"{cfg.name}-P{args.candidates}")
+        per_config[key] = measure_config(key, cfg, args, env)
+    head = per_config[head_key]
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            cpu = time_oracle_sample(wl.CONFIGS[head_key], budget_s=args.cpu_budget)
+        config = {k: head[k] for k in ("workload", "tokens_per_gpu_step", "candidates_per_gpu", "rank", "projections", "l2",
+                                       "calls_per_step", "kernel_timing")}
+        config["parallelism"] = f"dp{world} (candidate-sharded, no data-path collective)"
+        config["headline"] = ("largest single-GPU bf16 workload of the five" if not args.config else "--config given")
+        config["peaks"] = {"source": peak_src, "bf16_tflops_burst": peaks["bf16_tflops"],
+                           "bf16_tflops_sustained": peaks["bf16_tflops_sustained"], "hbm_gbs": peaks["hbm_gbs"],
+                           "nominal_bf16_tflops": NOMINAL_PEAKS["bf16_tflops"], "nominal_hbm_gbs": NOMINAL_PEAKS["hbm_gbs"]}
+        config["per_config"] = per_config
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": head["steps"],
+                "warmup": head["warmup"], "ms_per_step": head["ms_per_step"], "ms_per_step_median": head["ms_per_step_median"],
+                "ms_per_step_min": head["ms_per_step_min"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": head["dtype"], "data": "synthetic", "config": config, "roofline": head["roofline"],
+                "cpu_baseline": cpu, "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"]}
+        print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def spawn_ranks(args):
+    """--gpus N without a launcher: re-execute this script under torch.distributed.run with N local ranks."""
+    port = 29500 + (os.getpid() % 2000)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="2", choices=list(wl.CONFIGS))
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--config", default=None, choices=list(wl.CONFIGS),
+                    help="one workload only (default: 2, 3, 4, 5a, 5b in turn, config 4 as the headline)")
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--pair-tiles", type=int, default=-1, help="override ESSA_OPT_PAIR_TILES (0 / 1)")
@@ -415,14 +584,14 @@ def main():
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")
     args = ap.parse_args()
-    cfg = wl.CONFIGS[args.config]
-    if args.candidates > 0:
-        import dataclasses
-        cfg = dataclasses.replace(cfg, P=args.candidates, name=f"{cfg.name}-P{args.candidates}")
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
     if args.impl == "reference":
-        run_reference(args, cfg)
-    else:
-        run_ours(args, cfg)
+        run_reference(args, wl.CONFIGS[args.config or HEADLINE])
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)
+    run_ours(args)
 
 
 if __name__ == "__main__":
