@@ -323,14 +323,20 @@ def measure_config(key, cfg, args, env):
     decode = T <= 256  # one-launch decode schedule (essa_plan.decode)
     block_call = decode and len(handles) > 1 and not args.single_calls
 
+    # Decode steps are tens of microseconds: their two calls are marshalled once (binding.PreparedSample /
+    # PreparedBlock: the same C entry points, argument tuples built ahead of time) so that the host keeps ahead.
+    stream_handle = stream.cuda_stream
+    prep_sample = ctx.prepare_sample(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, sigma, k_begin)
+    prep_blocks = [ctx.prepare_block(hs, xs, d_off, sigma, cols, ys) for hs in handle_sets] if block_call else None
+
     def step():
-        hs = handle_sets[step_no[0] % copies]
+        c = step_no[0] % copies
         step_no[0] += 1
-        ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, out=sigma, k_begin=k_begin)
+        prep_sample.run(stream_handle)
         if block_call:  # decode sizes: the block's projections share tokens, segments and the table -> one call
-            ctx.apply_block(hs, xs, d_off, sigma, cols, outs=ys)
+            prep_blocks[c].run(stream_handle)
         else:
-            for i, h in enumerate(hs):
+            for i, h in enumerate(handle_sets[c]):
                 ctx.apply_projection(h, xs[i], d_off, sigma, cols[i][0], cols[i][1], out=ys[i])
 
     def barrier():

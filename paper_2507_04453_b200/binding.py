@@ -177,6 +177,49 @@ class AdapterHandle:
             self.handle = None
 
 
+class PreparedBlock:
+    """essa_apply_block with its arguments marshalled ahead of time (see Context.prepare_block)."""
+
+    def __init__(self, ctx, adapters, xs, seg_offsets, sigma, cols, outs):
+        n = len(adapters)
+        T = xs[0].shape[0]
+        self.keep = (list(adapters), list(xs), seg_offsets, sigma, list(outs))
+        self.arr = (BlockItem * n)()
+        for i in range(n):
+            self.arr[i] = BlockItem(adapters[i].handle, xs[i].data_ptr() if T else None, cols[i][0], cols[i][1],
+                                    outs[i].data_ptr() if T else None)
+        self.ctx = ctx
+        self.fn = ctx.lib.essa_apply_block
+        self.args = (ctx.handle, self.arr, n, T, seg_offsets.data_ptr(), seg_offsets.numel() - 1, sigma.data_ptr(),
+                     sigma.stride(0) if sigma.dim() == 2 else sigma.numel())
+
+    def run(self, stream_handle):
+        """stream_handle: the integer cudaStream_t (torch's ``stream.cuda_stream``; 0 / None = default stream)."""
+        st = self.fn(*self.args, stream_handle or None)
+        if st != ESSA_OK:
+            self.ctx._check(st)
+
+
+class PreparedSample:
+    """essa_sample_population(_range) with its arguments marshalled ahead of time (see Context.prepare_sample)."""
+
+    def __init__(self, ctx, mean, step, Bfactor, Dvec, seed, P, out, k_begin):
+        self.keep = (mean, Bfactor, Dvec, out)
+        self.ctx = ctx
+        d = mean.numel()
+        if k_begin == 0:
+            self.fn = ctx.lib.essa_sample_population
+            self.args = (ctx.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec), d, seed, P, out.data_ptr())
+        else:
+            self.fn = ctx.lib.essa_sample_population_range
+            self.args = (ctx.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec), d, seed, k_begin, P, out.data_ptr())
+
+    def run(self, stream_handle):
+        st = self.fn(*self.args, stream_handle or None)
+        if st != ESSA_OK:
+            self.ctx._check(st)
+
+
 class Context:
     """Owns one essa_ctx on a CUDA device."""
 
@@ -332,6 +375,16 @@ class Context:
                                        sigma.stride(0) if sigma.dim() == 2 else sigma.numel(), _stream(stream))
         self._check(st)
         return outs
+
+    def prepare_block(self, adapters, xs, seg_offsets, sigma, cols, outs):
+        """The arguments of one essa_apply_block call marshalled once; ``run(stream)`` then issues the call with a
+        single foreign-function call (at decode sizes the Python-side marshalling of a step is otherwise comparable
+        to the step's device time).  The tensors must stay alive and in place while the object is used."""
+        return PreparedBlock(self, adapters, xs, seg_offsets, sigma, cols, outs)
+
+    def prepare_sample(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, out, k_begin: int = 0):
+        """The arguments of one essa_sample_population(_range) call marshalled once; ``run(stream)`` issues it."""
+        return PreparedSample(self, mean, step, Bfactor, Dvec, seed, P, out, k_begin)
 
     def apply_projection_static(self, adapter, x, seg_offsets, sigma, sA_col: int, sB_col: int, out, stream=None):
         """essa_apply_projection_static: same result as apply_projection without any device allocation.

@@ -42,6 +42,22 @@ int32_t ensure_scratch(essa_ctx* ctx, Scratch& s, size_t bytes, bool zero, cudaS
   return ESSA_OK;
 }
 
+// Device-side ordering of calls that share the context's scratch: see essa_ctx::last_stream.
+void order_stream(essa_ctx* ctx, cudaStream_t stream) {
+  if (ctx->last_stream_valid && ctx->last_stream != stream) {
+    if (!ctx->order_event && cudaEventCreateWithFlags(&ctx->order_event, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      ctx->order_event = nullptr;
+    }
+    // (a stream the caller has destroyed in the meantime has no work left to wait for: errors are dropped)
+    if (ctx->order_event && cudaEventRecord(ctx->order_event, ctx->last_stream) == cudaSuccess)
+      cudaStreamWaitEvent(stream, ctx->order_event, 0);
+    cudaGetLastError();
+  }
+  ctx->last_stream = stream;
+  ctx->last_stream_valid = true;
+}
+
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -178,6 +194,7 @@ int32_t essa_destroy(essa_ctx* ctx) {
   free_scratch(ctx->w_deq);
   free_scratch(ctx->pair_ready);
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
+  if (ctx->order_event) cudaEventDestroy(ctx->order_event);
   for (cudaEvent_t e : ctx->host_events) cudaEventDestroy(e);
   if (ctx->host_h2d) cudaStreamDestroy(ctx->host_h2d);
   if (ctx->host_d2h) cudaStreamDestroy(ctx->host_d2h);
@@ -318,8 +335,10 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAtH, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad / 2, 64, 128);
   }
-  // With host sources the caller's buffers are only needed until the copies have run.
-  if (cudaStreamSynchronize(stream) != cudaSuccess && st == ESSA_OK) st = check_cuda(ctx, cudaGetLastError(), "load_adapter: sync");
+  // With host sources the caller's buffers are only needed until the copies have run; device sources stay
+  // asynchronous (the caller keeps them valid until the stream has passed this call).
+  if (!d->on_device && cudaStreamSynchronize(stream) != cudaSuccess && st == ESSA_OK)
+    st = check_cuda(ctx, cudaGetLastError(), "load_adapter: sync");
   if (st != ESSA_OK) {
     essa_free_adapter(ctx, a);
     return st;
@@ -410,6 +429,7 @@ int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* 
   const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
   if (st != ESSA_OK || T == 0) return st;
   ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  order_stream(ctx, static_cast<cudaStream_t>(stream));
   return launch_projection_tc(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 
@@ -425,6 +445,7 @@ int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_
   }
   if (T == 0) return ESSA_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  order_stream(ctx, stream);
   if (T <= kDecodeMaxTokens) {
     BlockItem bi[ESSA_MAX_BLOCK_ITEMS];
     for (int32_t i = 0; i < n_items; ++i)
@@ -458,6 +479,7 @@ int32_t essa_apply_projection_static(essa_ctx* ctx, const essa_adapter* a, const
   const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
   if (st != ESSA_OK || T == 0) return st;
   ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  order_stream(ctx, static_cast<cudaStream_t>(stream));
   return launch_projection_tc_static(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 
@@ -467,6 +489,7 @@ int32_t essa_apply_projection_simt(essa_ctx* ctx, const essa_adapter* a, const v
   const int32_t st = validate_projection_args(ctx, a, x, T, seg, P, sigma, ld_sigma, sA_col, sB_col, y);
   if (st != ESSA_OK || T == 0) return st;
   ProjArgs g{static_cast<const __nv_bfloat16*>(x), T, seg, P, sigma, ld_sigma, sA_col, sB_col, static_cast<__nv_bfloat16*>(y)};
+  order_stream(ctx, static_cast<cudaStream_t>(stream));
   return launch_projection_simt(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 

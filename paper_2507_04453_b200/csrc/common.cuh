@@ -55,6 +55,18 @@ struct essa_ctx {
   cudaStream_t host_h2d = nullptr, host_d2h = nullptr;
   std::vector<cudaEvent_t> host_events;
   void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // Calls that use the context's scratch buffers and counters are ordered on the device: when a call arrives on
+  // another stream than the previous one, the new stream first waits for an event recorded on the old one.
+  cudaStream_t last_stream = nullptr;
+  bool last_stream_valid = false;
+  cudaEvent_t order_event = nullptr;
+  // decode launches: tensor maps of recently used activation buffers (encoding one costs about a microsecond and a
+  // decode step is tens of microseconds), keyed by (pointer, tokens, features, box rows); round-robin replacement
+  struct XMapEntry { const void* ptr = nullptr; int64_t T = 0; int32_t d_in = 0; uint32_t box = 0; CUtensorMap tm; };
+  XMapEntry xmap_cache[16];
+  int xmap_next = 0;
+  CUtensorMap dec_u_map[ESSA_MAX_BLOCK_ITEMS][2];   // maps of the decode u buffers for 64-row boxes / one box of tn rows
+  uint32_t dec_u_map_box[ESSA_MAX_BLOCK_ITEMS][2] = {};
   // essa_profile_begin/end: three events per recorded call
   bool prof_on = false;
   int prof_calls = 0, prof_dropped = 0;
@@ -86,6 +98,7 @@ namespace essa {
 int32_t fail(essa_ctx* ctx, int32_t code, const std::string& msg);
 int32_t check_cuda(essa_ctx* ctx, cudaError_t e, const char* what);
 int32_t ensure_scratch(essa_ctx* ctx, Scratch& s, size_t bytes, bool zero, cudaStream_t stream);
+void order_stream(essa_ctx* ctx, cudaStream_t stream);
 
 // kind: 0 = bf16, 1 = uint8/int8.  rows x cols (cols contiguous), box = box_rows x box_cols, swizzle bytes in {0,64,128}.
 int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void* base, uint64_t rows, uint64_t cols,

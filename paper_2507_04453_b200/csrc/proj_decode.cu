@@ -30,9 +30,10 @@
 //     deterministic), applies the INT8 per-channel scale, rounds to bf16 once and stores y.
 //
 // Slice owners never wait for another CTA before they deliver, the finishing CTAs wait only for the owners, and
-// both are low-numbered CTAs of the first wave, so every wait ends; all are bounded all the same.  Warp roles (192 threads): warp 0 = TMA
-// producer of both rings, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank path + epilogue; INT8 storage
-// adds warps 6..9, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
+// both are low-numbered CTAs of the first wave, so every wait ends; all are bounded all the same.  Warp roles: warp 0 = TMA
+// producer of the frozen operands (W0 ring, V_A^T tiles), warp 1 = TMEM allocator + MMA issuer, warps 2..5 = rank
+// path + epilogue, one more warp (6, or 10 for INT8 storage) = TMA producer of the activations (x ring, u tile);
+// INT8 storage adds warps 6..9, which turn the streamed codes into bf16 operand tiles in shared memory.  A CTA that gives up
 // on a wait records ESSA_ERR_DEVICE_TIMEOUT, still joins both cluster barriers, frees its TMEM and exits.
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -42,12 +43,12 @@ namespace {
 
 constexpr int DEC_M = 128;       // W0 rows per CTA (UMMA M)
 constexpr int DEC_K = 64;        // 64 bf16 = one 128-byte swizzle row
-constexpr int kDecThreads = 192;
+constexpr int kDecThreads = 224;             // warps 0..5 and the activation producer (warp 6)
 constexpr int kDecSmemBudget = 227 * 1024;
 constexpr int W_TILE_BYTES = DEC_M * DEC_K * 2;  // 16 KB
 constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 6;
 constexpr int kInt8ConvStages = 4;  // converted tiles between the converting warps and the tensor core
-constexpr int kDecThreadsInt8 = 320;             // + warps 6..9: INT8 -> bf16 converters
+constexpr int kDecThreadsInt8 = 352;         // warps 0..5, INT8 -> bf16 converters (6..9), activation producer (10)
 constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored INT8 codes
 constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
 static_assert(kFinishTokens == 8, "finish_unit loads four tokens per thread as one float4");
@@ -308,11 +309,9 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
     if (INT8) {  // 128 rows of 64 codes, unswizzled
       tma_load_2d(dst, &tmW, kcol(i), m_tile * DEC_M, fb);
-    } else {     // two 64-row boxes
+    } else {     // one 128-row box
       const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
-      const int col = i < nkb ? kcol(i) : 0;
-      tma_load_2d(dst, tm, col, m_tile * DEC_M, fb);
-      tma_load_2d(dst + 64 * 128, tm, col, m_tile * DEC_M + 64, fb);
+      tma_load_2d(dst, tm, i < nkb ? kcol(i) : 0, m_tile * DEC_M, fb);
     }
   };
   auto load_ub = [&](int e) {  // INT8: U_B slab e goes straight into item nkb + e of the converted ring
@@ -322,7 +321,6 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const uint32_t dst = smem_u32(smem_c + s * W_TILE_BYTES);
     const CUtensorMap* tm = e == 0 ? &tmUB0 : &tmUB1;
     tma_load_2d(dst, tm, 0, m_tile * DEC_M, fb);
-    tma_load_2d(dst + 64 * 128, tm, 0, m_tile * DEC_M + 64, fb);
   };
   auto load_x = [&](int i) {  // item i of the x ring
     const int s = i % SX;
@@ -368,59 +366,64 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // draw); x, the singular values, the scratch buffers and y are touched only after this point.
   grid_dep_wait();
 
+  // ------------------------------------------------------------------ TMA producers: warp 0 streams the frozen
+  // operands (the W0 ring and, during this CTA's slice, the V_A^T tiles), warp kXWarp the activations (the x ring,
+  // then the u tile).  One issuing thread for both rings measured 1.4 times slower per K block than two (a thread
+  // that has just issued a 32 KB box does not get to the other ring's free slot in time).  Each ring is filled in
+  // its own order with a bounded wait for the slot; a thread that gives up waits for its copies in flight.
+  constexpr int kXWarp = INT8 ? 10 : 6;
+  auto drain = [&](int issued, int S, uint32_t bar_f) {
+    const int outstanding = issued < S ? issued : S;
+    for (int j = 0; j < outstanding; ++j) {
+      const int i = issued - 1 - j;
+      const long long t0 = clock64();
+      while (!mbar_try_wait(bar_f + 8 * (i % S), (uint32_t)((i / S) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
+    }
+  };
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer: one thread feeds both rings,
-    // issuing whatever has a free slot (each ring in its own order, so the parity waits stay in step)
     if (lane == 0) {
-      int iw = first_w, ix = 0, iv = 0;  // next item of the W0 ring, of the x ring, of the V_A^T ring
+      int iw = first_w, iv = 0;
       bool ok = true;
-      long long t_idle = 0;
-      while (ok && (iw < n_w || ix < n_x || iv < c_own)) {
-        bool progress = false;
-        if (iv < c_own && (iv < kVatStages || mbar_test_wait(bar_vempty + 8 * (iv % kVatStages), (uint32_t)(((iv / kVatStages) & 1) ^ 1)))) {
-          load_v(iv++);
-          progress = true;
+      while (ok && (iw < n_w || iv < c_own)) {
+        // the V_A^T tile of item iv goes out no later than the W0 tile of the same item
+        if (iv < c_own && iv <= iw) {
+          if (iv >= kVatStages) ok = mbar_wait(bar_vempty + 8 * (iv % kVatStages), (uint32_t)(((iv / kVatStages) & 1) ^ 1), abort_flag, p.status);
+          if (ok) load_v(iv++);
+          continue;
         }
-        if (iw < n_w && (iw < SW || mbar_test_wait(bar_wempty + 8 * (iw % SW), (uint32_t)(((iw / SW) & 1) ^ 1)))) {
-          load_w(iw++);
-          progress = true;
-        }
-        if (ix < n_x && (ix < SX || mbar_test_wait(bar_xempty + 8 * (ix % SX), (uint32_t)(((ix / SX) & 1) ^ 1)))) {
-          // the u tile (item nkb) also needs every row published: acquire the count, then order the
-          // async-proxy read after it
-          const bool ready = ix < nkb || (int32_t)(ld_acquire_u32(p.u_count) - p.u_target) >= 0;
-          if (ready) {
-            if (ix == nkb) fence_proxy_async_global();
-            load_x(ix++);
-            progress = true;
-          }
-        }
-        if (progress) {
-          t_idle = 0;
-        } else {
-          const long long now = clock64();
-          if (t_idle == 0) t_idle = now;
-          if (*abort_flag || now - t_idle > kWaitLimitCycles) {
-            *abort_flag = 1;
-            atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
-            ok = false;
-          }
+        if (iw < n_w) {
+          if (iw >= SW) ok = mbar_wait(bar_wempty + 8 * (iw % SW), (uint32_t)(((iw / SW) & 1) ^ 1), abort_flag, p.status);
+          if (ok) load_w(iw++);
         }
       }
       if (!ok || *abort_flag) {
-        // giving up: let the copies already issued land before the CTA's shared memory is released
-        auto drain = [&](int issued, int S, uint32_t bar_f) {
-          const int outstanding = issued < S ? issued : S;
-          for (int j = 0; j < outstanding; ++j) {
-            const int i = issued - 1 - j;
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar_f + 8 * (i % S), (uint32_t)((i / S) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
-          }
-        };
         drain(iw, SW, bar_wfull);
-        drain(ix, SX, bar_xfull);
         drain(iv, kVatStages, bar_vfull);
       }
+    }
+  } else if (warp == kXWarp) {
+    if (lane == 0) {
+      int ix = 0;
+      bool ok = true;
+      while (ok && ix < n_x) {
+        if (ix >= SX) ok = mbar_wait(bar_xempty + 8 * (ix % SX), (uint32_t)(((ix / SX) & 1) ^ 1), abort_flag, p.status);
+        if (ok && ix == nkb) {
+          // the u tile also needs every row published: acquire the count (bounded), then order the async-proxy
+          // read after it
+          const long long t0 = clock64();
+          while ((int32_t)(ld_acquire_u32(p.u_count) - p.u_target) < 0) {
+            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+              *abort_flag = 1;
+              atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+              ok = false;
+              break;
+            }
+          }
+          if (ok) fence_proxy_async_global();
+        }
+        if (ok) load_x(ix++);
+      }
+      if (!ok || *abort_flag) drain(ix, SX, bar_xfull);
     }
   } else if (warp == 1 && is_main) {
     // ------------------------------------------------------------------ MMA issuer
@@ -555,7 +558,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       }
     }
   };
-  if (INT8 && warp >= 6) convert_loop();
+  if (INT8 && warp >= 6 && warp <= 9) convert_loop();
 
   // ------------------------------------------------------------------ warps 2..5: rank path, then the epilogue
   const int quad = warp & 3;
@@ -768,8 +771,13 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   const void* kernel = int8 ? (const void*)essa_decode_kernel<true> : (const void*)essa_decode_kernel<false>;
   const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
   {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
+    static bool attr_done[64][2] = {};  // the attribute is per device and kernel instance
+    bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][int8 ? 1 : 0];
+    if (!done) {
+      const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
+      if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
+      done = true;
+    }
   }
   if (resident_cache[splits] == 0) {
     cudaLaunchConfig_t q{};
@@ -802,12 +810,15 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   blk.n_proj = n;
   blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
   int cta = 0, unit = 0;
+  // The counters' next values are committed to the context only once the launch has been accepted: after a failed
+  // call the device never reaches them, and a later call must not wait for rows nobody publishes.
+  uint32_t next_pepoch[kMaxBlockProj] = {}, next_epoch[kMaxBlockProj] = {};
   for (int i = 0; i < n; ++i) {
     const essa_adapter* a = items[i].a;
     DParams& p = blk.proj[i];
     p.T = (int)T;
     p.tn = tn;
-    p.xbox = (tn % 64 == 0) ? 64 : tn;
+    p.xbox = tn;  // one box per tile (at most 256 rows)
     p.d_in = a->d_in;
     p.d_out = a->d_out;
     p.main_kb = a->d_in / DEC_K;
@@ -838,8 +849,8 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
         delivered += (nkb_s + p.p_c - 1) / p.p_c;
       }
       p.p_count = ctx->dec_pcnt + i;
-      ctx->dec_pepoch[i] += (uint32_t)delivered;
-      p.p_target = ctx->dec_pepoch[i];
+      next_pepoch[i] = ctx->dec_pepoch[i] + (uint32_t)delivered;
+      p.p_target = next_pepoch[i];
     }
     p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)i * kMaxPSlices * kDecodeMaxTokens * kRankPadMax;
     p.seg = seg;
@@ -852,23 +863,42 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     p.M = a->M;
     p.u = static_cast<__nv_bfloat16*>(ctx->dec_u) + (size_t)i * kDecodeMaxTokens * kRankPadMax;
     p.u_count = ctx->dec_cnt + i;
-    ctx->dec_epoch[i] += (uint32_t)T;
-    p.u_target = ctx->dec_epoch[i];
+    next_epoch[i] = ctx->dec_epoch[i] + (uint32_t)T;
+    p.u_target = next_epoch[i];
     p.status = ctx->d_status;
     blk.cta_begin[i] = cta;
     blk.unit_begin[i] = unit;
     cta += p.m_tiles * splits;
     unit += p.rank_groups;
 
-    maps.tm[i][0] = int8 ? a->tm_W0q : a->tm_W0[0];  // 64-row boxes of bf16 W0 / 128-row boxes of codes
-    int32_t st = make_tensor_map_2d(ctx, &maps.tm[i][1], 0, items[i].x, (uint64_t)T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
-                                    (uint32_t)p.xbox, DEC_K, 128);
-    if (st != ESSA_OK) return st;
-    st = make_tensor_map_2d(ctx, &maps.tm[i][2], 0, p.u, (uint64_t)kDecodeMaxTokens, kRankPadMax, kRankPadMax * 2,
-                            (uint32_t)p.xbox, DEC_K, 128);
-    if (st != ESSA_OK) return st;
-    maps.tm[i][3] = a->tm_UBp[0][0];  // 64-row boxes of the U_B slabs
-    maps.tm[i][4] = a->tm_UBp[0][a->ext_blocks > 1 ? 1 : 0];
+    maps.tm[i][0] = int8 ? a->tm_W0q : a->tm_W0[1];  // 128-row boxes of bf16 W0 / of codes
+    // activation map: looked up by (pointer, tokens, features, box); u map: one per (projection slot, box)
+    {
+      essa_ctx::XMapEntry* hit = nullptr;
+      for (auto& e : ctx->xmap_cache)
+        if (e.ptr == items[i].x && e.T == T && e.d_in == a->d_in && e.box == (uint32_t)p.xbox) { hit = &e; break; }
+      if (!hit) {
+        essa_ctx::XMapEntry fresh;
+        const int32_t st = make_tensor_map_2d(ctx, &fresh.tm, 0, items[i].x, (uint64_t)T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
+                                              (uint32_t)p.xbox, DEC_K, 128);
+        if (st != ESSA_OK) return st;
+        fresh.ptr = items[i].x; fresh.T = T; fresh.d_in = a->d_in; fresh.box = (uint32_t)p.xbox;
+        hit = &ctx->xmap_cache[ctx->xmap_next];
+        ctx->xmap_next = (ctx->xmap_next + 1) % 16;
+        *hit = fresh;
+      }
+      maps.tm[i][1] = hit->tm;
+      const int slot = 0;
+      if (ctx->dec_u_map_box[i][slot] != (uint32_t)p.xbox) {
+        const int32_t st = make_tensor_map_2d(ctx, &ctx->dec_u_map[i][slot], 0, p.u, (uint64_t)kDecodeMaxTokens, kRankPadMax,
+                                              kRankPadMax * 2, (uint32_t)p.xbox, DEC_K, 128);
+        if (st != ESSA_OK) return st;
+        ctx->dec_u_map_box[i][slot] = (uint32_t)p.xbox;
+      }
+      maps.tm[i][2] = ctx->dec_u_map[i][slot];
+    }
+    maps.tm[i][3] = a->tm_UBp[1][0];  // 128-row boxes of the U_B slabs
+    maps.tm[i][4] = a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0];
     maps.tm[i][5] = a->tm_VAt;
   }
   for (int i = n; i <= kMaxBlockProj; ++i) { blk.cta_begin[i] = cta; blk.unit_begin[i] = unit; }
@@ -888,10 +918,15 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  ctx->launches += 1;
   const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, maps, blk)
                              : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, maps, blk);
-  return check_cuda(ctx, e, "essa_decode_kernel launch");
+  if (e != cudaSuccess) return check_cuda(ctx, e, "essa_decode_kernel launch");
+  ctx->launches += 1;
+  for (int i = 0; i < n; ++i) {
+    ctx->dec_pepoch[i] = next_pepoch[i];
+    ctx->dec_epoch[i] = next_epoch[i];
+  }
+  return ESSA_OK;
 }
 
 int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, const essa_plan& pl,

@@ -637,6 +637,7 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     st = launch_base_up_pair(ctx, tm_x, tmW128, tm_u, a->tm_UBp[1][0], a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0], (int)g.T,
                              a->d_out, a->d_in / BLOCK_K, a->ext_blocks, a->r_pad / UMMA_K, g.y, mp.scale, fused ? &pd : nullptr,
                              stream);
+    if (st != ESSA_OK && fused) ctx->pair_epoch -= 1;  // nothing was enqueued: the device never reaches this epoch
     if (ev) cudaEventRecord(ev[2], stream);
     return st;
   }

@@ -399,8 +399,13 @@ int32_t launch_base_up_pair(essa_ctx* ctx, const CUtensorMap& tmA, const CUtenso
                        : rp == 48 ? (const void*)essa_tc2_kernel<48>
                                   : (const void*)essa_tc2_kernel<64>;
   const int smem = p2_smem(rp);
-  const cudaError_t ea = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (ea != cudaSuccess) return check_cuda(ctx, ea, "cudaFuncSetAttribute(essa_tc2_kernel)");
+  static bool attr_done[64][5] = {};  // the attribute is per device and kernel instance
+  bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][rp / 16];
+  if (!done) {
+    const cudaError_t ea = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (ea != cudaSuccess) return check_cuda(ctx, ea, "cudaFuncSetAttribute(essa_tc2_kernel)");
+    done = true;
+  }
   const int sm = ctx->sm_count > 0 ? ctx->sm_count : 148;
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
   int pairs = (int)(tiles < sm / 2 ? tiles : sm / 2);
