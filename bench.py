@@ -328,10 +328,16 @@ def measure_config(key, cfg, args, env):
     stream_handle = stream.cuda_stream
     prep_sample = ctx.prepare_sample(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, sigma, k_begin)
     prep_blocks = [ctx.prepare_block(hs, xs, d_off, sigma, cols, ys) for hs in handle_sets] if block_call else None
+    fused_call = block_call and not args.separate_calls
+    prep_fused = [ctx.prepare_sample_block(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, sigma, hs, xs, d_off, cols, ys, k_begin)
+                  for hs in handle_sets] if fused_call else None
 
     def step():
         c = step_no[0] % copies
         step_no[0] += 1
+        if fused_call:  # draw + block in one call: the block kernel streams W0 while the draw runs
+            prep_fused[c].run(stream_handle)
+            return
         prep_sample.run(stream_handle)
         if block_call:  # decode sizes: the block's projections share tokens, segments and the table -> one call
             prep_blocks[c].run(stream_handle)
@@ -498,7 +504,8 @@ def measure_config(key, cfg, args, env):
            "l2": "inputs larger than L2 (x, W0 and y of the projections exceed 126 MB per step)"
                  if copies == 1 else f"weights rotate through {copies} device copies ({copies * w_bytes / 1e6:.0f} MB > 2 x L2): "
                                      "every step streams W0 from HBM (ms_per_step_l2_warm: one copy, W0 served from L2)",
-           "calls_per_step": "essa_sample_population + 1 x essa_apply_block" if block_call
+           "calls_per_step": "1 x essa_sample_apply_block (population draw + the block's projections)" if fused_call
+                             else "essa_sample_population + 1 x essa_apply_block" if block_call
                              else f"essa_sample_population + {len(handles)} x essa_apply_projection",
            "kernel_timing": "CUDA events around every launch, inside the timed steps" if events_inside
                             else "CUDA events around every launch in a second pass of the same steps (not inside the timed steps)",
@@ -588,6 +595,8 @@ def main():
     ap.add_argument("--fuse-down", type=int, default=-1, help="override ESSA_OPT_FUSE_DOWN (0 / 1)")
     ap.add_argument("--single-calls", action="store_true",
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
+    ap.add_argument("--separate-calls", action="store_true",
+                    help="decode configurations: essa_sample_population then essa_apply_block instead of the fused call")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")
     args = ap.parse_args()
     if args.gpus < 1:

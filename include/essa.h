@@ -20,7 +20,11 @@
  *   - Every call returns an int32 status: ESSA_OK (0) or a negative ESSA_ERR_* code; the text of
  *     the most recent error on a context is available from essa_last_error().
  *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = the
- *     legacy default stream).  Calls do not synchronise unless stated.
+ *     legacy default stream).  Calls do not synchronise unless stated.  The projection calls of
+ *     one context share its scratch buffers and counters, so the library keeps them ordered on
+ *     the device: a call that arrives on another stream than the context's previous projection
+ *     call first makes its stream wait (an event) for that previous call.  Use one context per
+ *     stream for calls that should overlap.
  *   - Ownership: the caller owns every pointer it passes.  essa_load_adapter copies what it
  *     needs into library-owned device memory (released by essa_free_adapter).  Device buffers
  *     passed to asynchronous calls must stay valid until the stream has executed the call.
@@ -111,7 +115,9 @@ typedef struct essa_adapter_desc {
 
 /* Copy and re-lay-out an adapter into library-owned device memory and precompute M = V_B^T U_A.
  * The bases are used as given (orthonormality is not assumed).  Asynchronous on `stream` when the
- * sources are device pointers; with host pointers the call returns after the copies have completed. */
+ * sources are device pointers (they must stay valid until the stream has passed the call); with host
+ * pointers the call returns after the copies have completed.  INT8 storage: every scale must be
+ * positive and finite (a zero scale would drop that channel's rank term together with its W0 row). */
 int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* desc, essa_adapter** out, void* stream);
 /* Free an adapter. Synchronises the device first. */
 int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* adapter);
@@ -197,6 +203,19 @@ typedef struct essa_block_item {
 } essa_block_item;
 int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T,
                          const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma, void* stream);
+
+/* Population draw and block projections in one call (Algorithm 1, lines 5 and 7, for the candidates this worker
+ * evaluates): exactly essa_sample_population_range(mean, step, Bfactor, Dvec, d, seed, k_begin, P, sigma_out)
+ * followed by essa_apply_block(items, n_items, T, seg_offsets, P, sigma_out, ld_sigma = d).  Because the library
+ * itself enqueues the two kernels back to back, at decode sizes the block kernel does not wait for the draw to
+ * finish: it streams W0 and the activations beside it, and only its rank path waits (bounded) until the draw
+ * reports the table complete.  The activations, segment offsets and adapters must therefore be final when the call
+ * is made (they may not be produced by work enqueued after it); sigma_out [P][d] is written and may be read by later
+ * work on the stream as usual.  Results are identical to the two separate calls. */
+int32_t essa_sample_apply_block(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec,
+                                int32_t d, uint64_t seed, int32_t k_begin, int32_t P, float* sigma_out,
+                                const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg_offsets,
+                                void* stream);
 
 /* The same operation with HOST buffers: x, seg_offsets, sigma are copied to the device, the
  * projection runs, y is copied back, and the call returns after `stream` has been synchronised.

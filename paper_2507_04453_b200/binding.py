@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "essa_apply_projection_simt", "essa_plan_projection", "essa_validate_segments", "essa_debug_stream_words",
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
     "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
-    "essa_top_alpha_index", "essa_sample_population_masked", "essa_export_candidates",
+    "essa_top_alpha_index", "essa_sample_population_masked", "essa_export_candidates", "essa_sample_apply_block",
 )
 
 
@@ -111,6 +111,7 @@ def load_library() -> C.CDLL:
         "essa_set_option": (i32, [vp, i32, i32]),
         "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_apply_block_host": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
+        "essa_sample_apply_block": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, C.POINTER(BlockItem), i32, i64, vp, vp]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -195,6 +196,28 @@ class PreparedBlock:
 
     def run(self, stream_handle):
         """stream_handle: the integer cudaStream_t (torch's ``stream.cuda_stream``; 0 / None = default stream)."""
+        st = self.fn(*self.args, stream_handle or None)
+        if st != ESSA_OK:
+            self.ctx._check(st)
+
+
+class PreparedSampleBlock:
+    """essa_sample_apply_block with its arguments marshalled ahead of time (see Context.prepare_sample_block)."""
+
+    def __init__(self, ctx, mean, step, Bfactor, Dvec, seed, P, sigma_out, adapters, xs, seg_offsets, cols, outs, k_begin):
+        n = len(adapters)
+        T = xs[0].shape[0]
+        self.keep = (mean, Bfactor, Dvec, sigma_out, list(adapters), list(xs), seg_offsets, list(outs))
+        self.arr = (BlockItem * n)()
+        for i in range(n):
+            self.arr[i] = BlockItem(adapters[i].handle, xs[i].data_ptr() if T else None, cols[i][0], cols[i][1],
+                                    outs[i].data_ptr() if T else None)
+        self.ctx = ctx
+        self.fn = ctx.lib.essa_sample_apply_block
+        self.args = (ctx.handle, mean.data_ptr(), step, _ptr(Bfactor), _ptr(Dvec), mean.numel(), seed, k_begin, P,
+                     sigma_out.data_ptr(), self.arr, n, T, seg_offsets.data_ptr())
+
+    def run(self, stream_handle):
         st = self.fn(*self.args, stream_handle or None)
         if st != ESSA_OK:
             self.ctx._check(st)
@@ -381,6 +404,29 @@ class Context:
         single foreign-function call (at decode sizes the Python-side marshalling of a step is otherwise comparable
         to the step's device time).  The tensors must stay alive and in place while the object is used."""
         return PreparedBlock(self, adapters, xs, seg_offsets, sigma, cols, outs)
+
+    def prepare_sample_block(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, sigma_out, adapters, xs, seg_offsets,
+                             cols, outs, k_begin: int = 0):
+        """The arguments of one essa_sample_apply_block call (population draw + the block's projections) marshalled
+        once; ``run(stream)`` issues it."""
+        return PreparedSampleBlock(self, mean, step, Bfactor, Dvec, seed, P, sigma_out, adapters, xs, seg_offsets, cols, outs,
+                                   k_begin)
+
+    def sample_apply_block(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, adapters, xs, seg_offsets, cols,
+                           sigma_out=None, outs=None, k_begin: int = 0, stream=None):
+        """essa_sample_apply_block: draw the population into sigma_out[P, d] and run the block's projections on it.
+        Returns (sigma_out, outs)."""
+        torch = self.torch
+        d = mean.numel()
+        T = xs[0].shape[0]
+        if sigma_out is None:
+            sigma_out = torch.empty((P, d), dtype=torch.float32, device=self.device)
+        if outs is None:
+            outs = [torch.empty((T, a.d_out), dtype=torch.bfloat16, device=self.device) for a in adapters]
+        prep = PreparedSampleBlock(self, mean, step, Bfactor, Dvec, seed, P, sigma_out, adapters, xs, seg_offsets, cols, outs,
+                                   k_begin)
+        prep.run(_stream(stream))
+        return sigma_out, outs
 
     def prepare_sample(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, out, k_begin: int = 0):
         """The arguments of one essa_sample_population(_range) call marshalled once; ``run(stream)`` issues it."""

@@ -165,7 +165,9 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
       cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
       cudaMalloc(&ctx->dec_ppart, (size_t)ESSA_MAX_BLOCK_ITEMS * 32 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
       cudaMalloc(&ctx->dec_pcnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
-      cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess) {
+      cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->samp_cnt, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->samp_cnt, 0, sizeof(uint32_t)) != cudaSuccess) {
+    if (ctx->samp_cnt) cudaFree(ctx->samp_cnt);
     if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
     if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -203,6 +205,7 @@ int32_t essa_destroy(essa_ctx* ctx) {
   if (ctx->dec_cnt) cudaFree(ctx->dec_cnt);
   if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
   if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
+  if (ctx->samp_cnt) cudaFree(ctx->samp_cnt);
   delete ctx;
   return ESSA_OK;
 }
@@ -224,6 +227,8 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
     for (uint32_t& e : ctx->dec_epoch) e = 0;
     for (uint32_t& e : ctx->dec_pepoch) e = 0;
+    cudaMemset(ctx->samp_cnt, 0, sizeof(uint32_t));
+    ctx->samp_epoch = 0;
     if (ctx->pair_ready.ptr) cudaMemset(ctx->pair_ready.ptr, 0, ctx->pair_ready.bytes);
     ctx->pair_epoch = 0;
   }
@@ -433,8 +438,12 @@ int32_t essa_apply_projection(essa_ctx* ctx, const essa_adapter* a, const void* 
   return launch_projection_tc(ctx, a, g, static_cast<cudaStream_t>(stream));
 }
 
-int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg,
-                         int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v) {
+// essa_apply_block, optionally right behind a population draw that is still running (sigma_ready: see
+// launch_block_decode; honoured only by the one-launch decode schedule, the other schedules are ordered behind the
+// draw by the stream).
+static int32_t apply_block_impl(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg,
+                                int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v, const uint32_t* sigma_ready,
+                                uint32_t sigma_target) {
   if (!ctx) return ESSA_ERR_INVALID_ARG;
   if (!items || n_items < 1 || n_items > ESSA_MAX_BLOCK_ITEMS)
     return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_block: 1 .. ESSA_MAX_BLOCK_ITEMS items expected");
@@ -457,7 +466,7 @@ int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_
       else ++ctx->prof_dropped;
     }
     if (ev) { cudaEventRecord(ev[0], stream); cudaEventRecord(ev[1], stream); }
-    const int32_t st = launch_block_decode(ctx, bi, n_items, T, seg, P, sigma, ld_sigma, stream);
+    const int32_t st = launch_block_decode(ctx, bi, n_items, T, seg, P, sigma, ld_sigma, stream, sigma_ready, sigma_target);
     if (st != kBlockNotFused) {
       if (ev) { cudaEventRecord(ev[2], stream); ++ctx->prof_calls; }
       return st;
@@ -470,6 +479,34 @@ int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_
     if (st != ESSA_OK) return st;
   }
   return ESSA_OK;
+}
+
+int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg,
+                         int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v) {
+  return apply_block_impl(ctx, items, n_items, T, seg, P, sigma, ld_sigma, stream_v, nullptr, 0);
+}
+
+int32_t essa_sample_apply_block(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
+                                uint64_t seed, int32_t k_begin, int32_t P, float* sigma_out, const essa_block_item* items,
+                                int32_t n_items, int64_t T, const int32_t* seg, void* stream_v) {
+  int32_t st = validate_sampler(ctx, mean, d, k_begin, P, sigma_out);
+  if (st != ESSA_OK) return st;
+  if (!items || n_items < 1 || n_items > ESSA_MAX_BLOCK_ITEMS)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "sample_apply_block: 1 .. ESSA_MAX_BLOCK_ITEMS items expected");
+  // validate the block before anything is enqueued, so that a bad argument leaves no half-done call behind
+  for (int32_t i = 0; i < n_items; ++i) {
+    st = validate_projection_args(ctx, items[i].adapter, items[i].x, T, seg, P, sigma_out, d, items[i].sA_col, items[i].sB_col,
+                                  items[i].y);
+    if (st != ESSA_OK) return st;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  uint32_t blocks = 0;
+  st = launch_sampler(ctx, mean, step, Bfactor, Dvec, d, seed, k_begin, P, nullptr, d, sigma_out, stream, ctx->samp_cnt, &blocks);
+  if (st != ESSA_OK) return st;
+  ctx->samp_epoch += blocks;  // the draw is enqueued: its blocks will be counted
+  if (T == 0) return ESSA_OK;
+  return apply_block_impl(ctx, items, n_items, T, seg, P, sigma_out, d, stream_v, blocks > 0 ? ctx->samp_cnt : nullptr,
+                          ctx->samp_epoch);
 }
 
 // Allocation-free variant: see the comment above g_static_u in proj_tc.cu.

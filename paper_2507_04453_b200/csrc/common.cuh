@@ -44,6 +44,8 @@ struct essa_ctx {
   void* dec_ppart = nullptr;    // [32][kDecodeMaxTokens][64] fp32 per projection: per-slice partial down-projections
   uint32_t* dec_pcnt = nullptr; // slices delivered so far, per projection (monotonic; dec_pepoch is the host's copy)
   uint32_t dec_pepoch[ESSA_MAX_BLOCK_ITEMS] = {};
+  uint32_t* samp_cnt = nullptr; // blocks of fused population draws finished so far (monotonic; samp_epoch is the host's copy)
+  uint32_t samp_epoch = 0;
   // Scratch owned by the context (grown on demand, never shrunk).
   essa::Scratch u_buf;        // [T_cap][64] bf16: rank-path vector u_t, zero-padded to 64 columns
   essa::Scratch splitk_ws;    // fp32 partial tiles for split-K (kept all-zero between calls)
@@ -107,7 +109,7 @@ int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void
 // sampler.cu
 int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
                        uint64_t seed, int32_t k_begin, int32_t k_count, const int32_t* index, int32_t ld_out, float* sigma_out,
-                       cudaStream_t stream);
+                       cudaStream_t stream, uint32_t* done = nullptr, uint32_t* blocks_out = nullptr);
 int32_t launch_fill_rows(essa_ctx* ctx, const float* frozen, int32_t d, int32_t k_count, float* sigma_out, cudaStream_t stream);
 int32_t launch_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count, int32_t n_blocks,
                             uint32_t* words_out, cudaStream_t stream);
@@ -165,8 +167,12 @@ struct BlockItem {
   __nv_bfloat16* y;
 };
 constexpr int32_t kBlockNotFused = 1;  // launch_block_decode: the block does not fit the one-wave decode schedule
+// sigma_ready != NULL: the table is being written by the kernel launched just before on the same stream, which
+// counts its finished blocks in *sigma_ready; the launch does not wait for that kernel as a whole, only (bounded)
+// for the count to reach sigma_target before it reads the table.
 int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
-                            const float* sigma, int32_t ld_sigma, cudaStream_t stream);
+                            const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready = nullptr,
+                            uint32_t sigma_target = 0);
 bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out);
 int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, const essa_plan& plan,
                                  cudaStream_t stream);

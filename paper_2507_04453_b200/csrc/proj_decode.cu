@@ -99,6 +99,11 @@ struct DBlock {
   int cta_begin[kMaxBlockProj + 1];   // multiples of the cluster size; cta_begin[n_proj] = W0-streaming CTAs
   int unit_begin[kMaxBlockProj + 1];  // rank-path units (token group x K slice) per projection
   int rank_ctas;                      // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
+  // Fused draw + block call: the singular-value table is being written by the population-draw kernel launched just
+  // before this one; that kernel counts its finished blocks in *sigma_ready.  The launch then does not wait for the
+  // draw as a whole (it streams W0 and x beside it) and only the rank path waits for the count (bounded).
+  const uint32_t* sigma_ready;
+  uint32_t sigma_target;
   DParams proj[kMaxBlockProj];
 };
 struct DMaps {
@@ -363,8 +368,10 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const uint32_t tmem_base = is_main ? *tmem_slot : 0u;
   // Everything up to here (barriers, TMEM, the first tiles of the frozen W0) depends on no earlier kernel and, with
   // a programmatic dependent launch, overlaps the kernel before this one in the stream (typically the population
-  // draw); x, the singular values, the scratch buffers and y are touched only after this point.
-  grid_dep_wait();
+  // draw); x, the singular values, the scratch buffers and y are touched only after this point.  In a fused draw +
+  // block call the kernel before is known to be the draw, which writes nothing but the table: no wait here, the
+  // rank path waits for the table instead.
+  if (blk.sigma_ready == nullptr) grid_dep_wait();
 
   // ------------------------------------------------------------------ TMA producers: warp 0 streams the frozen
   // operands (the W0 ring and, during this CTA's slice, the V_A^T tiles), warp kXWarp the activations (the x ring,
@@ -599,6 +606,24 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     if ((int)blockIdx.x < blk.rank_ctas) {
       // this CTA's finishing units of the rank path (of any projection of the block), while its K loop streams
       bool fine = true;
+      if (blk.sigma_ready != nullptr && (int)blockIdx.x < blk.unit_begin[blk.n_proj]) {
+        // the table must be complete before its rows are read
+        if (etid == 0) {
+          int ok = 1;
+          const long long w0 = clock64();
+          while ((int32_t)(ld_acquire_u32(blk.sigma_ready) - blk.sigma_target) < 0) {
+            if (*abort_flag || clock64() - w0 > kWaitLimitCycles) { ok = 0; break; }
+          }
+          if (!ok) {
+            *abort_flag = 1;
+            atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+          }
+          *flag = ok;
+        }
+        epi_bar_sync();
+        fine = *flag != 0;
+        epi_bar_sync();  // flag may be reused
+      }
       for (int unit = blockIdx.x; fine && unit < blk.unit_begin[blk.n_proj]; unit += blk.rank_ctas) {
         int pj = 0;
         while (pj + 1 < blk.n_proj && unit >= blk.unit_begin[pj + 1]) ++pj;
@@ -748,7 +773,8 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
 // error, or kBlockNotFused (> 0) when the block does not fit the one-wave decode schedule and the caller should
 // issue the projections one by one.
 int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
-                            const float* sigma, int32_t ld_sigma, cudaStream_t stream) {
+                            const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready,
+                            uint32_t sigma_target) {
   if (n < 1 || n > kMaxBlockProj || T <= 0 || T > kDecodeMaxTokens) return kBlockNotFused;
   const bool int8 = items[0].a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   int d_in[kMaxBlockProj], d_out[kMaxBlockProj];
@@ -808,6 +834,8 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   DBlock blk{};
   DMaps maps{};
   blk.n_proj = n;
+  blk.sigma_ready = sigma_ready;
+  blk.sigma_target = sigma_target;
   blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
   int cta = 0, unit = 0;
   // The counters' next values are committed to the context only once the launch has been accepted: after a failed

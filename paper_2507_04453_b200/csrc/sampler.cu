@@ -42,26 +42,37 @@ __device__ __forceinline__ void normals_block(uint2 key, uint32_t j, uint32_t k,
   box_muller(w.z, w.w, z[2], z[3]);
 }
 
+// Completion count for a consumer that runs concurrently (the decode kernel of a fused draw + block call): every
+// block adds one, after its rows of the table are visible device-wide.
+__device__ __forceinline__ void block_done(uint32_t* done) {
+  if (done == nullptr) return;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) red_release_add_u32(done, 1u);
+}
+
 // Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
 __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, const float* __restrict__ Dvec, int d,
                                    uint2 key, int k_begin, int k_count, const int32_t* __restrict__ index, int ld_out,
-                                   float* __restrict__ sigma_out) {
+                                   float* __restrict__ sigma_out, uint32_t* done) {
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
   const int nb = (d + 3) >> 2;
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-  if (idx >= (long long)k_count * nb) return;
-  const int kk = (int)(idx / nb), j = (int)(idx % nb);
-  double zz[4];
-  normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk), zz);
+  if (idx < (long long)k_count * nb) {
+    const int kk = (int)(idx / nb), j = (int)(idx % nb);
+    double zz[4];
+    normals_block(key, (uint32_t)j, (uint32_t)(k_begin + kk), zz);
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const int i = 4 * j + e;
-    if (i < d) {
-      const double w = Dvec ? (double)Dvec[i] * zz[e] : zz[e];
-      const int col = index ? index[i] : i;  // top-alpha: coordinate i of the optimised vector sits in column index[i]
-      if (col >= 0 && col < ld_out) sigma_out[(size_t)kk * ld_out + col] = (float)((double)mean[i] + (double)step * w);
+    for (int e = 0; e < 4; ++e) {
+      const int i = 4 * j + e;
+      if (i < d) {
+        const double w = Dvec ? (double)Dvec[i] * zz[e] : zz[e];
+        const int col = index ? index[i] : i;  // top-alpha: coordinate i of the optimised vector sits in column index[i]
+        if (col >= 0 && col < ld_out) sigma_out[(size_t)kk * ld_out + col] = (float)((double)mean[i] + (double)step * w);
+      }
     }
   }
+  block_done(done);
 }
 
 // Full covariance factor.  blockIdx.x = group of kCand candidates, blockIdx.y = tile of kRows rows of Bfactor.
@@ -77,7 +88,7 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
                                                                       const float* __restrict__ Dvec, int d, uint2 key,
                                                                       int k_begin, int k_count,
                                                                       const int32_t* __restrict__ index, int ld_out,
-                                                                      float* __restrict__ sigma_out) {
+                                                                      float* __restrict__ sigma_out, uint32_t* done) {
   extern __shared__ __align__(16) double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
   const int nb = (d + 3) >> 2, d4 = nb * 4;
@@ -158,6 +169,7 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
         if (kk0 + c < k_count) sigma_out[(size_t)(kk0 + c) * ld_out + col] = (float)(mi + (double)step * acc[c]);
     }
   }
+  block_done(done);
 }
 
 __global__ void stream_words_kernel(uint2 key, int k_begin, int k_count, int n_blocks, uint32_t* __restrict__ out) {
@@ -197,9 +209,12 @@ int32_t launch_fill_rows(essa_ctx* ctx, const float* frozen, int32_t d, int32_t 
 }
 
 // index != NULL: coordinate i of the sampled vector is written to column index[i] of rows of ld_out floats.
+// done != NULL: every block of the launch adds one to *done when its part of the table is visible; *blocks_out
+// receives the number of blocks launched (0 when nothing was launched).
 int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
                        uint64_t seed, int32_t k_begin, int32_t k_count, const int32_t* index, int32_t ld_out, float* sigma_out,
-                       cudaStream_t stream) {
+                       cudaStream_t stream, uint32_t* done, uint32_t* blocks_out) {
+  if (blocks_out) *blocks_out = 0;
   if (k_count == 0 || d == 0) return ESSA_OK;
   const int nb = (d + 3) / 4;
   if (Bfactor == nullptr) {
@@ -208,7 +223,8 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     const long long blocks = (total + threads - 1) / threads;
     if (blocks > 0x7fffffffLL) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: P*d too large");
     sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count, index,
-                                                                 ld_out, sigma_out);
+                                                                 ld_out, sigma_out, done);
+    if (blocks_out) *blocks_out = (uint32_t)blocks;
   } else {
     if (d > 4096) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 4096 with a full covariance factor");
     const size_t smem = (size_t)kCand * nb * 4 * sizeof(double);
@@ -220,7 +236,8 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     }
     dim3 grid((k_count + kCand - 1) / kCand, (d + kRows - 1) / kRows);
     kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin, k_count, index, ld_out,
-                                                    sigma_out);
+                                                    sigma_out, done);
+    if (blocks_out) *blocks_out = grid.x * grid.y;
   }
   ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "sampler launch");

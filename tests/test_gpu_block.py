@@ -120,3 +120,47 @@ def test_block_host_entry_point(torch, ctx, base, dm, dkv, r, P, L):
         assert orc.relative_error(got, case.oracle_projection(i, xs[i])) <= tol, (cfg.name, cfg.projections[i])
     assert ctx.get_status() == 0
     case.close()
+
+
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 1024, 192, 16, 256, 1),    # decode, full covariance factor
+                                               ("5a", 1024, 256, 64, 128, 1),   # decode, INT8 storage, diagonal draw
+                                               ("2", 256, 64, 16, 3, 100)])     # prefill sizes: plain stream order
+def test_fused_draw_and_block_equals_separate_calls_and_oracle(torch, ctx, base, dm, dkv, r, P, L):
+    """essa_sample_apply_block: the table and every output equal the two separate calls bit for bit (the block
+    kernel only starts earlier), and both match the oracle; repeated calls stay identical (the draw's completion
+    count is monotonic across calls)."""
+    from tests.parity_utils import TOL_SIGMA, sigma_error
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    n = len(cfg.projections)
+    cma = case.cma
+    xs_host = [case.tokens(i) for i in range(n)]
+    xs = [to_dev(torch, x, torch.bfloat16) for x in xs_host]
+    cols = [cfg.sigma_cols(i) for i in range(n)]
+    hs = [case.handles[i] for i in range(n)]
+    d_mean = to_dev(torch, cma.mean)
+    d_B = None if cma.Bfactor is None else to_dev(torch, cma.Bfactor)
+    d_D = None if cma.Dvec is None else to_dev(torch, cma.Dvec)
+    sig_sep = ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P)
+    ys_sep = ctx.apply_block(hs, xs, case.d_offsets, sig_sep, cols)
+    torch.cuda.synchronize()
+    for rep in range(3):
+        sig_f, ys_f = ctx.sample_apply_block(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, hs, xs, case.d_offsets, cols)
+        torch.cuda.synchronize()
+        assert torch.equal(sig_f, sig_sep)
+        for a, b in zip(ys_f, ys_sep):
+            if case.T <= 256:
+                assert torch.equal(a, b), (cfg.name, rep)
+            else:  # prefill split-K adds partial tiles in arrival order: equal to rounding, not bit for bit
+                assert orc.relative_error(a.float().cpu().numpy(), b.float().cpu().numpy()) <= 1e-2
+    want_sigma = orc.sample_population(cma.mean, cma.step, cma.Bfactor, cma.Dvec, cma.seed, cfg.P)
+    assert sigma_error(sig_f.cpu().numpy(), want_sigma) <= TOL_SIGMA
+    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    sig32 = sig_f.cpu().numpy()
+    for i in range(n):
+        ad = case.adapters[i]
+        from tests.parity_utils import oracle_weight
+        want = orc.apply_projection(oracle_weight(ad), ad.U_A, ad.V_A, ad.U_B, ad.V_B, xs_host[i], case.offsets, sig32,
+                                    *cols[i], ad.rank)
+        assert orc.relative_error(ys_f[i].float().cpu().numpy(), want) <= tol
+    case.close()
