@@ -142,6 +142,44 @@ int32_t essa_sample_population_range(essa_ctx* ctx, const float* mean, float ste
                                      const float* Dvec, int32_t d, uint64_t seed, int32_t k_begin,
                                      int32_t k_count, float* sigma_out, void* stream);
 
+/* Search-distribution state and its update (Section 3, "Evolutionary optimization": CMA-ES samples the population from
+ * N(m_t, sigma_t^2 C_t) and, once every candidate's reward is known, updates (m, sigma, C) from the reward ranking;
+ * Algorithm 1: the common state (m_0, sigma_0, C_0) of its initialisation line and the CMA-ES update every worker
+ * performs after the <seed, reward> exchange).  The paper prints no update formulas; the library implements the
+ * (mu/mu_w, lambda)-CMA-ES of Hansen's tutorial with its default strategy parameters for (d, lambda), non-negative
+ * recombination weights (mu = floor(lambda / 2)), c_m = 1, and a fresh decomposition C = B diag(D^2) B^T on every
+ * update.  Rewards are MAXIMISED; ties keep population order; a NaN reward ranks last.
+ * The state lives in device memory (fp64; the sampler reads fp32 copies of m, sigma, B, D), so
+ * ask -> evaluate -> tell -> ask needs no host round trip.  d <= 1024, 2 <= lambda <= 65536. */
+typedef struct essa_cma essa_cma;
+/* m_0 = mean0 [d] fp32 HOST, sigma_0 = step0 > 0, C_0 = I, both evolution paths zero.  Synchronous. */
+int32_t essa_cma_create(essa_ctx* ctx, int32_t d, int32_t lambda, const float* mean0_host, float step0, essa_cma** out);
+/* Synchronises the device, then frees the state. */
+int32_t essa_cma_destroy(essa_ctx* ctx, essa_cma* state);
+/* essa_sample_population_range from the state: rows k_begin .. k_begin + k_count - 1 of the population
+ * m + sigma B (D .* z_k), sigma_out [k_count][d] fp32 dev.  Asynchronous on `stream`. */
+int32_t essa_cma_ask(essa_ctx* ctx, essa_cma* state, uint64_t seed, int32_t k_begin, int32_t k_count, float* sigma_out,
+                     void* stream);
+/* One update from a whole population: population [lambda][ld] fp32 dev (row k = candidate k as it was evaluated,
+ * ld >= d), rewards [lambda] fp32 dev.  Steps, in the tutorial's order: rank; y_i = (x_i:lambda - m) / sigma for the mu
+ * best; m += sigma sum w_i y_i; p_sigma with C^{-1/2} = B D^{-1} B^T; sigma; the stall indicator h_sigma; p_c; rank-one
+ * and rank-mu update of C; decomposition (one-sided Jacobi rotations, at most 30 sweeps, eigenvalues ascending).
+ * Asynchronous on `stream`: the launches are enqueued and the call returns (the number of Jacobi sweeps enqueued adapts to
+ * convergence reports that arrive without blocking).  Calls on one state must be ordered by the caller (one stream). */
+int32_t essa_tell(essa_ctx* ctx, essa_cma* state, const float* population, int32_t ld, const float* rewards, void* stream);
+/* Overwrite parts of the state from HOST fp64 arrays (NULL = keep): mean [d], step [1], C [d][d] symmetric positive
+ * definite (the decomposition is recomputed), p_sigma [d], p_c [d]; generation >= 0 sets the update counter.
+ * Synchronises `stream` first. */
+int32_t essa_cma_set(essa_ctx* ctx, essa_cma* state, const double* mean, const double* step, const double* C,
+                     const double* p_sigma, const double* p_c, int32_t generation, void* stream);
+/* Copy the state to HOST fp64 arrays (NULL = skip): mean [d], step [1], C [d][d], B [d][d] row-major (column j =
+ * eigenvector j), D [d] ascending, p_sigma [d], p_c [d]; *generation = updates done; *sweeps = Jacobi sweeps the last
+ * decomposition ran.  Synchronises the device. */
+int32_t essa_cma_get(essa_ctx* ctx, essa_cma* state, double* mean, double* step, double* C, double* B, double* D,
+                     double* p_sigma, double* p_c, int32_t* generation, int32_t* sweeps);
+/* Strategy parameters in use: out9 = {mu, mu_eff, c_sigma, d_sigma, c_c, c_1, c_mu, c_m, E|N(0,I)|}.  Needs no device. */
+int32_t essa_cma_params(essa_cma* state, double* out9);
+
 /* Candidate reconstruction for hand-off to an external inference engine (Algorithm 1, line 7, as the paper's
  * workers do it: A'_k = U_A diag(sA_k) V_A^T, B'_k = U_B diag(sB_k) V_B^T, the engine then runs W0 + B'_k A'_k).
  * The projection entry points above never form these matrices; this call does, for candidates

@@ -36,6 +36,7 @@ EXPORTED_SYMBOLS = (
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
     "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
     "essa_top_alpha_index", "essa_sample_population_masked", "essa_export_candidates", "essa_sample_apply_block",
+    "essa_cma_create", "essa_cma_destroy", "essa_cma_ask", "essa_tell", "essa_cma_set", "essa_cma_get", "essa_cma_params",
 )
 
 
@@ -112,6 +113,13 @@ def load_library() -> C.CDLL:
         "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_apply_block_host": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_sample_apply_block": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, C.POINTER(BlockItem), i32, i64, vp, vp]),
+        "essa_cma_create": (i32, [vp, i32, i32, vp, f32, C.POINTER(vp)]),
+        "essa_cma_destroy": (i32, [vp, vp]),
+        "essa_cma_ask": (i32, [vp, vp, u64, i32, i32, vp, vp]),
+        "essa_tell": (i32, [vp, vp, vp, i32, vp, vp]),
+        "essa_cma_set": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, vp]),
+        "essa_cma_get": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32), C.POINTER(i32)]),
+        "essa_cma_params": (i32, [vp, vp]),
         "essa_load_adapter": (i32, [vp, C.POINTER(AdapterDesc), C.POINTER(vp), vp]),
         "essa_free_adapter": (i32, [vp, vp]),
         "essa_sample_population": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, vp, vp]),
@@ -243,6 +251,70 @@ class PreparedSample:
             self.ctx._check(st)
 
 
+class CmaState:
+    """Device-resident search-distribution state (essa_cma_*): argument marshalling only."""
+
+    def __init__(self, ctx, d: int, lam: int, mean0, step0: float):
+        self.ctx, self.d, self.lam = ctx, d, lam
+        m = np.ascontiguousarray(mean0, dtype=np.float32)
+        h = C.c_void_p()
+        ctx._check(ctx.lib.essa_cma_create(ctx.handle, d, lam, m.ctypes.data_as(C.c_void_p), float(step0), C.byref(h)))
+        self.handle = h.value
+
+    def close(self):
+        if self.handle:
+            self.ctx.lib.essa_cma_destroy(self.ctx.handle, self.handle)
+            self.handle = None
+
+    def ask(self, seed: int, P=None, out=None, k_begin: int = 0, stream=None):
+        """essa_cma_ask: candidates k_begin .. k_begin + P - 1 of the population, [P, d] fp32 on the device."""
+        torch = self.ctx.torch
+        P = self.lam if P is None else P
+        if out is None:
+            out = torch.empty((P, self.d), dtype=torch.float32, device=self.ctx.device)
+        self.ctx._check(self.ctx.lib.essa_cma_ask(self.ctx.handle, self.handle, seed, k_begin, P, out.data_ptr(), _stream(stream)))
+        return out
+
+    def tell(self, population, rewards, stream=None):
+        """essa_tell: population [lambda, ld] fp32 and rewards [lambda] fp32, both on the device."""
+        self.ctx._check(self.ctx.lib.essa_tell(self.ctx.handle, self.handle, population.data_ptr(), population.stride(0),
+                                               rewards.data_ptr(), _stream(stream)))
+
+    def set(self, mean=None, step=None, C_=None, p_sigma=None, p_c=None, generation: int = -1, stream=None):
+        """essa_cma_set from host fp64 arrays (None = keep)."""
+        keep = []
+
+        def ptr(a, shape):
+            if a is None:
+                return None
+            a = np.ascontiguousarray(np.asarray(a, dtype=np.float64).reshape(shape))
+            keep.append(a)
+            return a.ctypes.data_as(C.c_void_p)
+        d = self.d
+        self.ctx._check(self.ctx.lib.essa_cma_set(self.ctx.handle, self.handle, ptr(mean, (d,)), ptr(step, (1,)), ptr(C_, (d, d)),
+                                                  ptr(p_sigma, (d,)), ptr(p_c, (d,)), generation, _stream(stream)))
+
+    def get(self) -> dict:
+        """essa_cma_get: the whole state as host fp64 arrays."""
+        d = self.d
+        out = {"mean": np.empty(d), "step": np.empty(1), "C": np.empty((d, d)), "B": np.empty((d, d)), "D": np.empty(d),
+               "p_sigma": np.empty(d), "p_c": np.empty(d)}
+        gen, sweeps = C.c_int32(0), C.c_int32(0)
+        p = lambda k: out[k].ctypes.data_as(C.c_void_p)
+        self.ctx._check(self.ctx.lib.essa_cma_get(self.ctx.handle, self.handle, p("mean"), p("step"), p("C"), p("B"), p("D"),
+                                                  p("p_sigma"), p("p_c"), C.byref(gen), C.byref(sweeps)))
+        out["step"] = float(out["step"][0])
+        out["generation"], out["sweeps"] = gen.value, sweeps.value
+        return out
+
+    def params(self) -> dict:
+        """essa_cma_params: the strategy parameters in use."""
+        v = np.empty(9)
+        self.ctx._check(self.ctx.lib.essa_cma_params(self.handle, v.ctypes.data_as(C.c_void_p)))
+        names = ("mu", "mu_eff", "c_sigma", "d_sigma", "c_c", "c_1", "c_mu", "c_m", "chi_n")
+        return dict(zip(names, (float(x) for x in v)))
+
+
 class Context:
     """Owns one essa_ctx on a CUDA device."""
 
@@ -317,6 +389,10 @@ class Context:
         h = C.c_void_p()
         self._check(self.lib.essa_load_adapter(self.handle, C.byref(desc), C.byref(h), _stream(None)))
         return AdapterHandle(self, h.value, d_in, d_out, rank, dtype)
+
+    def cma_state(self, d: int, lam: int, mean0, step0: float) -> "CmaState":
+        """essa_cma_create: search-distribution state (m_0 = mean0 host array, sigma_0 = step0, C_0 = I) on the device."""
+        return CmaState(self, d, lam, mean0, step0)
 
     # -- sampling
     def sample_population(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, out=None, k_begin: int = 0,

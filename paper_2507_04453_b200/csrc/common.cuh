@@ -109,7 +109,8 @@ int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void
 // sampler.cu
 int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
                        uint64_t seed, int32_t k_begin, int32_t k_count, const int32_t* index, int32_t ld_out, float* sigma_out,
-                       cudaStream_t stream, uint32_t* done = nullptr, uint32_t* blocks_out = nullptr);
+                       cudaStream_t stream, uint32_t* done = nullptr, uint32_t* blocks_out = nullptr,
+                       const float* step_dev = nullptr);
 int32_t launch_fill_rows(essa_ctx* ctx, const float* frozen, int32_t d, int32_t k_count, float* sigma_out, cudaStream_t stream);
 int32_t launch_stream_words(essa_ctx* ctx, uint64_t seed, int32_t k_begin, int32_t k_count, int32_t n_blocks,
                             uint32_t* words_out, cudaStream_t stream);

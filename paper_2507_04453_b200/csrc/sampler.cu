@@ -54,8 +54,9 @@ __device__ __forceinline__ void block_done(uint32_t* done) {
 // Identity covariance factor: sigma[k][i] = mean[i] + step * Dvec[i] * z_k[i].  One thread per (k, block j).
 __global__ void sample_diag_kernel(const float* __restrict__ mean, float step, const float* __restrict__ Dvec, int d,
                                    uint2 key, int k_begin, int k_count, const int32_t* __restrict__ index, int ld_out,
-                                   float* __restrict__ sigma_out, uint32_t* done) {
+                                   float* __restrict__ sigma_out, uint32_t* done, const float* __restrict__ step_ptr) {
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
+  if (step_ptr != nullptr) step = *step_ptr;  // step size kept in device memory (search-distribution state)
   const int nb = (d + 3) >> 2;
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (idx < (long long)k_count * nb) {
@@ -88,9 +89,11 @@ __global__ void __launch_bounds__(kSamplerThreads) sample_full_kernel(const floa
                                                                       const float* __restrict__ Dvec, int d, uint2 key,
                                                                       int k_begin, int k_count,
                                                                       const int32_t* __restrict__ index, int ld_out,
-                                                                      float* __restrict__ sigma_out, uint32_t* done) {
+                                                                      float* __restrict__ sigma_out, uint32_t* done,
+                                                                      const float* __restrict__ step_ptr) {
   extern __shared__ __align__(16) double w_smem[];  // [kCand][d4], d4 = 4*ceil(d/4)
   grid_dep_launch();  // a dependent launch of the next kernel may begin its set-up; it reads sigma after its own wait
+  if (step_ptr != nullptr) step = *step_ptr;  // step size kept in device memory (search-distribution state)
   const int nb = (d + 3) >> 2, d4 = nb * 4;
   const int kk0 = blockIdx.x * kCand;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -210,10 +213,11 @@ int32_t launch_fill_rows(essa_ctx* ctx, const float* frozen, int32_t d, int32_t 
 
 // index != NULL: coordinate i of the sampled vector is written to column index[i] of rows of ld_out floats.
 // done != NULL: every block of the launch adds one to *done when its part of the table is visible; *blocks_out
-// receives the number of blocks launched (0 when nothing was launched).
+// receives the number of blocks launched (0 when nothing was launched).  step_dev != NULL: the step size is read
+// from device memory instead of `step`.
 int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,
                        uint64_t seed, int32_t k_begin, int32_t k_count, const int32_t* index, int32_t ld_out, float* sigma_out,
-                       cudaStream_t stream, uint32_t* done, uint32_t* blocks_out) {
+                       cudaStream_t stream, uint32_t* done, uint32_t* blocks_out, const float* step_dev) {
   if (blocks_out) *blocks_out = 0;
   if (k_count == 0 || d == 0) return ESSA_OK;
   const int nb = (d + 3) / 4;
@@ -223,7 +227,7 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     const long long blocks = (total + threads - 1) / threads;
     if (blocks > 0x7fffffffLL) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: P*d too large");
     sample_diag_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mean, step, Dvec, d, key_of(seed), k_begin, k_count, index,
-                                                                 ld_out, sigma_out, done);
+                                                                 ld_out, sigma_out, done, step_dev);
     if (blocks_out) *blocks_out = (uint32_t)blocks;
   } else {
     if (d > 4096) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "sample_population: d > 4096 with a full covariance factor");
@@ -236,7 +240,7 @@ int32_t launch_sampler(essa_ctx* ctx, const float* mean, float step, const float
     }
     dim3 grid((k_count + kCand - 1) / kCand, (d + kRows - 1) / kRows);
     kernel<<<grid, kSamplerThreads, smem, stream>>>(mean, step, Bfactor, Dvec, d, key_of(seed), k_begin, k_count, index, ld_out,
-                                                    sigma_out, done);
+                                                    sigma_out, done, step_dev);
     if (blocks_out) *blocks_out = grid.x * grid.y;
   }
   ctx->launches += 1;
