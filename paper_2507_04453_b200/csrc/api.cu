@@ -73,6 +73,7 @@ int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void
   const cuuint32_t estr[2] = {1, 1};
   const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                       : CU_TENSOR_MAP_SWIZZLE_NONE;
   const CUtensorMapDataType dt = kind == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
   const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
@@ -337,6 +338,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
                                 kRankPadMax * 2, rows[i], 64, 128);
     }
     if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q, 1, a->W0q, m, n, n, 128, 64, 0);
+    if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q64, 1, a->W0q, m, n, n, 128, 64, 64);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAtH, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad / 2, 64, 128);
   }

@@ -93,6 +93,7 @@ struct essa_adapter {
   CUtensorMap tm_VAt;
   CUtensorMap tm_VAtH;           // the same with boxes of r_pad / 2 rows (one CTA's half in the pair kernel)
   CUtensorMap tm_W0q;            // INT8 storage: the codes, 128-row x 64-byte boxes, unswizzled
+  CUtensorMap tm_W0q64;          // ... the same boxes with the 64-byte swizzle (row-per-thread readers)
 };
 
 namespace essa {
@@ -102,7 +103,7 @@ int32_t check_cuda(essa_ctx* ctx, cudaError_t e, const char* what);
 int32_t ensure_scratch(essa_ctx* ctx, Scratch& s, size_t bytes, bool zero, cudaStream_t stream);
 void order_stream(essa_ctx* ctx, cudaStream_t stream);
 
-// kind: 0 = bf16, 1 = uint8/int8.  rows x cols (cols contiguous), box = box_rows x box_cols, swizzle bytes in {0,64,128}.
+// kind: 0 = bf16, 1 = uint8/int8.  rows x cols (cols contiguous), box = box_rows x box_cols, swizzle bytes in {0,32,64,128}.
 int32_t make_tensor_map_2d(essa_ctx* ctx, CUtensorMap* out, int kind, const void* base, uint64_t rows, uint64_t cols,
                            uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols, int swizzle_bytes);
 

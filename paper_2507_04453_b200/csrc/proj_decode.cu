@@ -46,10 +46,18 @@ constexpr int DEC_K = 64;        // 64 bf16 = one 128-byte swizzle row
 constexpr int kDecThreads = 224;             // warps 0..5 and the activation producer (warp 6)
 constexpr int kDecSmemBudget = 227 * 1024;
 constexpr int W_TILE_BYTES = DEC_M * DEC_K * 2;  // 16 KB
-constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 6;
+constexpr int kMaxWStages = 16, kMaxXStages = 6, kMaxCStages = 8;
 constexpr int kInt8ConvStages = 4;  // converted tiles between the converting warps and the tensor core
 constexpr int kDecThreadsInt8 = 352;         // warps 0..5, INT8 -> bf16 converters (6..9), activation producer (10)
 constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored INT8 codes
+// Storage / conversion modes of the kernel.  kModeBf16: W0 tiles are the MMA operand as stored.  kModeInt8Smem: four
+// warps turn tiles of INT8 codes into bf16 operand tiles in shared memory (any token count).  kModeInt8Tmem (at
+// most 128 tokens, so that tensor memory has room): the four warps write the converted tile straight into TENSOR
+// memory (tcgen05.st, thread = row of the tile) and the MMA takes its A operand from there, which removes the
+// write and the read of the converted tile from the shared-memory traffic that bounds the other INT8 mode.
+constexpr int kModeBf16 = 0, kModeInt8Smem = 1, kModeInt8Tmem = 2;
+constexpr int kTmemAStages = 8;                  // converted tiles in tensor memory (32 columns each)
+constexpr int kUbSlots = 2;                      // kModeInt8Tmem: the U_B slabs have shared-memory slots of their own
 constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
 static_assert(kFinishTokens == 8, "finish_unit loads four tokens per thread as one float4");
 constexpr int kMaxPSlices = 32;    // slots of partial down-projections per projection
@@ -247,9 +255,14 @@ __device__ __forceinline__ void sum_store(uint32_t mine /*shared-space address*/
   }
 }
 
-template <bool INT8>
-__global__ void __launch_bounds__(INT8 ? kDecThreadsInt8 : kDecThreads, 1)
+__host__ __device__ constexpr uint32_t tmem_a_col(int stage) { return stage < 4 ? 128u + 32u * stage : 384u + 32u * (stage - 4); }
+
+template <int MODE>
+__global__ void __launch_bounds__(MODE != kModeBf16 ? kDecThreadsInt8 : kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ DBlock blk) {
+  constexpr bool INT8 = MODE == kModeInt8Smem;   // codes converted through shared memory
+  constexpr bool TS = MODE == kModeInt8Tmem;     // codes converted into tensor memory (A operand from TMEM)
+  constexpr bool QUANT = MODE != kModeBf16;
   // which projection this CTA streams (CTAs past the last one only take rank-path units)
   int pi = 0;
   while (pi + 1 < blk.n_proj && (int)blockIdx.x >= blk.cta_begin[pi + 1]) ++pi;
@@ -264,8 +277,9 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
   const int x_bytes = p.tn * 128;
-  constexpr int W_SLOT = INT8 ? RAW_TILE_BYTES : W_TILE_BYTES;
-  const int SC = INT8 ? p.c_stages : 0;
+  constexpr int W_SLOT = QUANT ? RAW_TILE_BYTES : W_TILE_BYTES;
+  const int SC = INT8 ? p.c_stages : (TS ? kUbSlots : 0);   // 16 KB slots behind the W0 ring
+  const int SA = TS ? p.c_stages : 1;                       // kModeInt8Tmem: converted tiles in tensor memory
   // V_A^T tiles first: their MMA descriptor spans 128 rows, of which only the r_pad rows of the TMA box are data
   // (the accumulator rows beyond are never read), so the 16 KB it covers must lie inside the allocation
   uint8_t* smem_v = smem;
@@ -277,7 +291,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // dead once every MMA of the cluster has completed
   float* recv = reinterpret_cast<float*>(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2 + 2 * kVatStages + 1));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2 + 2 * kVatStages + 1 + kUbSlots));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* qbuf = reinterpret_cast<float*>(aux + 1024);      // [kFinishTokens][64]
 
@@ -286,6 +300,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const uint32_t bar_cfull = bar_xempty + 8 * kMaxXStages, bar_cempty = bar_cfull + 8 * kMaxCStages;
   const uint32_t bar_d = bar_cempty + 8 * kMaxCStages, bar_drain = bar_d + 8;
   const uint32_t bar_vfull = bar_drain + 8, bar_vempty = bar_vfull + 8 * kVatStages, bar_p = bar_vempty + 8 * kVatStages;
+  const uint32_t bar_ub = bar_p + 8;  // kModeInt8Tmem: one per U_B slab
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = (int)cluster_ctarank();
@@ -297,7 +312,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const int kb1 = kb0 + kbase + (split < krem ? 1 : 0);
   const int nkb = is_main ? kb1 - kb0 : 0;
   const int n_ext = (is_main && split == 0) ? p.ext : 0;  // K split 0 adds the rank term
-  const int n_w = INT8 ? nkb : nkb + n_ext;  // items of the W0 ring: the K blocks (bf16: then the U_B slabs)
+  const int n_w = QUANT ? nkb : nkb + n_ext;  // items of the W0 ring: the K blocks (bf16: then the U_B slabs)
   const int n_x = nkb + (n_ext ? 1 : 0);     // items of the x ring: the K blocks, then the u tile
   const int per = dec_rows_per_owner(p.tn, p.splits);
   constexpr uint32_t TMEM_COLS = 512;  // main accumulator (up to 256 tokens) + down-projection accumulator
@@ -312,7 +327,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const uint32_t fb = bar_wfull + 8 * s;
     mbar_expect_tx(fb, (uint32_t)W_SLOT);
     const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
-    if (INT8) {  // 128 rows of 64 codes, unswizzled
+    if (QUANT) {  // 128 rows of 64 codes (unswizzled; kModeInt8Tmem: 64-byte swizzle)
       tma_load_2d(dst, &tmW, kcol(i), m_tile * DEC_M, fb);
     } else {     // one 128-row box
       const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
@@ -326,6 +341,11 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const uint32_t dst = smem_u32(smem_c + s * W_TILE_BYTES);
     const CUtensorMap* tm = e == 0 ? &tmUB0 : &tmUB1;
     tma_load_2d(dst, tm, 0, m_tile * DEC_M, fb);
+  };
+  auto load_ub_slot = [&](int e) {  // kModeInt8Tmem: U_B slab e into its own slot
+    const uint32_t fb = bar_ub + 8 * e;
+    mbar_expect_tx(fb, (uint32_t)W_TILE_BYTES);
+    tma_load_2d(smem_u32(smem_c + e * W_TILE_BYTES), e == 0 ? &tmUB0 : &tmUB1, 0, m_tile * DEC_M, fb);
   };
   auto load_x = [&](int i) {  // item i of the x ring
     const int s = i % SX;
@@ -345,9 +365,15 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
 
   const int first_w = n_w < SW ? n_w : SW;  // the ring starts empty: its first fill needs no wait
   if (threadIdx.x == 0) {
-    for (int s = 0; s < SW; ++s) { mbar_init(bar_wfull + 8 * s, 1); mbar_init(bar_wempty + 8 * s, 1); }
+    // kModeInt8Tmem: a tile of codes is read, and its converted tile written, by four warps (one arrival each)
+    for (int s = 0; s < SW; ++s) { mbar_init(bar_wfull + 8 * s, 1); mbar_init(bar_wempty + 8 * s, TS ? 4 : 1); }
     for (int s = 0; s < SX; ++s) { mbar_init(bar_xfull + 8 * s, 1); mbar_init(bar_xempty + 8 * s, 1); }
-    for (int s = 0; s < SC; ++s) { mbar_init(bar_cfull + 8 * s, 1); mbar_init(bar_cempty + 8 * s, 1); }
+    if (TS) {
+      for (int s = 0; s < SA; ++s) { mbar_init(bar_cfull + 8 * s, 4); mbar_init(bar_cempty + 8 * s, 1); }
+      for (int e = 0; e < kUbSlots; ++e) mbar_init(bar_ub + 8 * e, 1);
+    } else {
+      for (int s = 0; s < SC; ++s) { mbar_init(bar_cfull + 8 * s, 1); mbar_init(bar_cempty + 8 * s, 1); }
+    }
     mbar_init(bar_d, 1);
     mbar_init(bar_drain, 1);
     for (int s = 0; s < kVatStages; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 1); }
@@ -357,6 +383,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     *reinterpret_cast<volatile int*>(tmem_slot + 4) = 0;  // ... and whose turn it is to claim a slot
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int i = 0; i < first_w; ++i) load_w(i);  // the frozen weights depend on nothing: stream at once
+    if (TS) for (int e = 0; e < n_ext; ++e) load_ub_slot(e);
   }
   if (warp == 1 && is_main) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -378,7 +405,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // then the u tile).  One issuing thread for both rings measured 1.4 times slower per K block than two (a thread
   // that has just issued a 32 KB box does not get to the other ring's free slot in time).  Each ring is filled in
   // its own order with a bounded wait for the slot; a thread that gives up waits for its copies in flight.
-  constexpr int kXWarp = INT8 ? 10 : 6;
+  constexpr int kXWarp = QUANT ? 10 : 6;
   auto drain = [&](int issued, int S, uint32_t bar_f) {
     const int outstanding = issued < S ? issued : S;
     for (int j = 0; j < outstanding; ++j) {
@@ -438,16 +465,22 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       const uint32_t idesc = make_idesc(DEC_M, p.tn);
       bool ok = true;
       for (int i = 0; i < nkb; ++i) {
-        const int sw = INT8 ? i % SC : i % SW, sx = i % SX;
-        const uint32_t wf = INT8 ? bar_cfull + 8 * sw : bar_wfull + 8 * sw;
-        const uint32_t wph = (uint32_t)((INT8 ? i / SC : i / SW) & 1);
+        const int sw = INT8 ? i % SC : TS ? i % SA : i % SW, sx = i % SX;
+        const uint32_t wf = (INT8 || TS) ? bar_cfull + 8 * sw : bar_wfull + 8 * sw;
+        const uint32_t wph = (uint32_t)((INT8 ? i / SC : TS ? i / SA : i / SW) & 1);
         if (!mbar_wait(bar_xfull + 8 * sx, (uint32_t)((i / SX) & 1), abort_flag, p.status) ||
             !mbar_wait(wf, wph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint64_t dw = make_smem_desc(smem_u32((INT8 ? smem_c : smem_w) + sw * W_TILE_BYTES));
         const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
+        if (TS) {  // A operand: the converted tile in tensor memory, 8 columns (16 bf16) per K step
+          const uint32_t ta = tmem_base + tmem_a_col(sw);
 #pragma unroll
-        for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16_ts(tmem_base, ta + 8 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        } else {
+#pragma unroll
+          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+        }
         if (i < c_own) {
           // this CTA's slice of the down-projection: V_A^T tile against the same x tile, second accumulator
           const int sv = i % kVatStages;
@@ -459,7 +492,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
           umma_commit(bar_vempty + 8 * sv);
           if (i == c_own - 1) umma_commit(bar_p);  // the slice is complete
         }
-        umma_commit((INT8 ? bar_cempty : bar_wempty) + 8 * sw);
+        umma_commit(((INT8 || TS) ? bar_cempty : bar_wempty) + 8 * sw);
         umma_commit(bar_xempty + 8 * sx);
       }
       if (ok && n_ext > 0) {
@@ -469,10 +502,11 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         const int ksteps = (p.r + 15) / 16;
         for (int e = 0; ok && e < n_ext; ++e) {
           const int i = nkb + e;
-          const int su = INT8 ? i % SC : i % SW;
-          if (!mbar_wait((INT8 ? bar_cfull : bar_wfull) + 8 * su, (uint32_t)((INT8 ? i / SC : i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
+          const int su = INT8 ? i % SC : TS ? e : i % SW;
+          const uint32_t ubar = INT8 ? bar_cfull + 8 * su : TS ? bar_ub + 8 * e : bar_wfull + 8 * su;
+          if (!mbar_wait(ubar, TS ? 0u : (uint32_t)((INT8 ? i / SC : i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t dub = make_smem_desc(smem_u32((INT8 ? smem_c : smem_w) + su * W_TILE_BYTES));
+          const uint64_t dub = make_smem_desc(smem_u32(((INT8 || TS) ? smem_c : smem_w) + su * W_TILE_BYTES));
           for (int k = 0; k < ksteps; ++k) umma_bf16(tmem_base, dub + 2 * k, du + 2 * k, idesc, 1u);
         }
       }
@@ -566,6 +600,49 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     }
   };
   if (INT8 && warp >= 6 && warp <= 9) convert_loop();
+  // kModeInt8Tmem.  Warp w of the four converting warps owns rows (= tensor-memory lanes) 32 (w mod 4) .. + 31 of
+  // EVERY tile, a thread one row: it reads the row's 64 codes (four 16-byte chunks; the tile was loaded with the
+  // 64-byte swizzle, chunk c of row r at position c ^ ((r >> 1) & 3), so the eight rows a quarter-warp reads at once
+  // fall into eight different bank groups), converts them exactly and stores the 32 packed bf16 pairs into the
+  // 32 columns of the tile's stage with one tcgen05.st.  The stage is handed to the MMA warp when all four warps
+  // have arrived; the slot of codes goes back to the TMA producer the same way.
+  if (TS && warp >= 6 && warp <= 9) {
+    const int band = warp & 3;
+    const int r = band * 32 + lane;
+    for (int i = 0; i < nkb; ++i) {
+      const int sa = i % SA, sr = i % SW;
+      int got_c = 1;
+      if (lane == 0) {
+        if (i >= SA) got_c = mbar_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1), abort_flag, p.status) ? 1 : 0;
+        if (got_c) got_c = mbar_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1), abort_flag, p.status) ? 1 : 0;
+      }
+      got_c = __shfl_sync(0xffffffffu, got_c, 0);
+      if (!got_c) break;
+      // both phases are complete: these return at once (acquire for every lane)
+      if (i >= SA) while (!mbar_try_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1))) {}
+      while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}
+      tc_fence_after();  // the MMAs that read this stage have completed (their commit released it)
+      const uint32_t raw = smem_u32(smem_w + sr * RAW_TILE_BYTES) + (uint32_t)(r * 64);
+      uint4 w[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) w[c] = lds_v4(raw + (uint32_t)((c ^ ((r >> 1) & 3)) << 4));
+      uint32_t v[32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        int8x4_to_bf16x4(w[c].x, v[8 * c + 0], v[8 * c + 1]);
+        int8x4_to_bf16x4(w[c].y, v[8 * c + 2], v[8 * c + 3]);
+        int8x4_to_bf16x4(w[c].z, v[8 * c + 4], v[8 * c + 5]);
+        int8x4_to_bf16x4(w[c].w, v[8 * c + 6], v[8 * c + 7]);
+      }
+      tmem_st32(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(sa), v);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar_cfull + 8 * sa);
+        mbar_arrive(bar_wempty + 8 * sr);
+      }
+    }
+  }
 
   // ------------------------------------------------------------------ warps 2..5: rank path, then the epilogue
   const int quad = warp & 3;
@@ -692,21 +769,25 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   }
 }
 
-// c_stages > 0 means INT8 storage: the W0 ring holds 8 KB tiles of codes and c_stages converted tiles follow it
-inline int dec_ring_bytes(int w_stages, int c_stages, int x_stages, int tn) {
-  return kVatStages * VAT_SLOT_BYTES + w_stages * (c_stages > 0 ? RAW_TILE_BYTES : W_TILE_BYTES) + c_stages * W_TILE_BYTES +
+// Shared-memory rings: V_A^T tiles, the W0 ring (16 KB bf16 tiles, or 8 KB tiles of codes), the 16 KB slots behind it
+// (kModeInt8Smem: c_stages converted tiles; kModeInt8Tmem: the U_B slabs), the x ring.
+inline int dec_ring_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
+  const int slots16k = mode == kModeInt8Smem ? c_stages : mode == kModeInt8Tmem ? kUbSlots : 0;
+  return kVatStages * VAT_SLOT_BYTES + w_stages * (mode != kModeBf16 ? RAW_TILE_BYTES : W_TILE_BYTES) + slots16k * W_TILE_BYTES +
          x_stages * tn * 128;
 }
-inline int dec_smem_bytes(int w_stages, int c_stages, int x_stages, int tn) {
-  return 1024 + dec_ring_bytes(w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
+inline int dec_smem_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
+  return 1024 + dec_ring_bytes(mode, w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
 }
+// INT8 storage converts into tensor memory whenever the accumulators leave room for the converted tiles there.
+inline int dec_mode(bool int8, int tn) { return !int8 ? kModeBf16 : tn <= 128 ? kModeInt8Tmem : kModeInt8Smem; }
 
 }  // namespace
 
 // Schedule shared by the projections of one decode launch (n of them, sizes d_in[i] -> d_out[i], same storage type):
 // cluster size, ring depths.  Returns false when the launch would not fit one wave of the GPU.
 static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int8, int64_t T, int sm_count, int* splits_out,
-                              int* w_stages_out, int* x_stages_out, int* m_tiles_total_out) {
+                              int* w_stages_out, int* x_stages_out, int* m_tiles_total_out, int* c_stages_out = nullptr) {
   if (T <= 0 || T > kDecodeMaxTokens || n < 1 || n > kMaxBlockProj) return false;
   const int sm = sm_count > 0 ? sm_count : 148;
   const int tn = (int)((T + 15) / 16) * 16;
@@ -727,10 +808,11 @@ static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int
   // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
   // INT8 storage: W0 tiles travel as 8 KB of codes; a ring of converted bf16 tiles (which also takes the U_B slabs,
   // loaded into it directly) sits between the converting warps and the tensor core.
-  const int c_stages = int8 ? kInt8ConvStages : 0;
+  const int mode = dec_mode(int8, tn);
+  const int c_stages = mode == kModeInt8Smem ? kInt8ConvStages : mode == kModeInt8Tmem ? kTmemAStages : 0;
   const int w_slot = int8 ? RAW_TILE_BYTES : W_TILE_BYTES;
   const int xb = tn * 128;
-  const int budget = kDecSmemBudget - dec_smem_bytes(0, c_stages, 0, tn);
+  const int budget = kDecSmemBudget - dec_smem_bytes(mode, 0, c_stages, 0, tn);
   int x_stages = budget / (w_slot + xb);
   if (x_stages > kMaxXStages) x_stages = kMaxXStages;
   if (x_stages < 1) return false;
@@ -738,7 +820,8 @@ static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
   if (w_stages < 1) return false;
   // the receive buffer of the cluster reduction overlays the rings
-  if (dec_ring_bytes(w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) return false;
+  if (dec_ring_bytes(mode, w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) return false;
+  if (c_stages_out) *c_stages_out = c_stages;
   *splits_out = splits;
   *w_stages_out = w_stages;
   *x_stages_out = x_stages;
@@ -783,22 +866,24 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     d_in[i] = items[i].a->d_in;
     d_out[i] = items[i].a->d_out;
   }
-  int splits, w_stages, x_stages, m_total;
-  if (!plan_decode_block(n, d_in, d_out, int8, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total)) {
+  int splits, w_stages, x_stages, m_total, c_stages;
+  if (!plan_decode_block(n, d_in, d_out, int8, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total, &c_stages)) {
     if (n > 1) return kBlockNotFused;
     return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: no decode schedule fits shared memory");
   }
   const int tn = (int)((T + 15) / 16) * 16;
-  const int c_stages = int8 ? kInt8ConvStages : 0;
+  const int mode = dec_mode(int8, tn);
 
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
-  static int resident_caches[64][2][9] = {};  // per device, storage type, cluster size
-  int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][int8 ? 1 : 0];
-  const void* kernel = int8 ? (const void*)essa_decode_kernel<true> : (const void*)essa_decode_kernel<false>;
+  static int resident_caches[64][3][9] = {};  // per device, kernel mode, cluster size
+  int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
+  const void* kernel = mode == kModeBf16      ? (const void*)essa_decode_kernel<kModeBf16>
+                       : mode == kModeInt8Smem ? (const void*)essa_decode_kernel<kModeInt8Smem>
+                                               : (const void*)essa_decode_kernel<kModeInt8Tmem>;
   const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
   {
-    static bool attr_done[64][2] = {};  // the attribute is per device and kernel instance
-    bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][int8 ? 1 : 0];
+    static bool attr_done[64][3] = {};  // the attribute is per device and kernel instance
+    bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
     if (!done) {
       const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
       if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
@@ -899,7 +984,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     cta += p.m_tiles * splits;
     unit += p.rank_groups;
 
-    maps.tm[i][0] = int8 ? a->tm_W0q : a->tm_W0[1];  // 128-row boxes of bf16 W0 / of codes
+    maps.tm[i][0] = mode == kModeInt8Tmem ? a->tm_W0q64 : int8 ? a->tm_W0q : a->tm_W0[1];  // 128-row boxes of bf16 W0 / of codes
     // activation map: looked up by (pointer, tokens, features, box); u map: one per (projection slot, box)
     {
       essa_ctx::XMapEntry* hit = nullptr;
@@ -931,7 +1016,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   }
   for (int i = n; i <= kMaxBlockProj; ++i) { blk.cta_begin[i] = cta; blk.unit_begin[i] = unit; }
 
-  const int smem_bytes = dec_smem_bytes(w_stages, c_stages, x_stages, tn);
+  const int smem_bytes = dec_smem_bytes(mode, w_stages, c_stages, x_stages, tn);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid_total, 1, 1);
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
@@ -946,8 +1031,9 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = int8 ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<true>, maps, blk)
-                             : cudaLaunchKernelEx(&cfg, essa_decode_kernel<false>, maps, blk);
+  const cudaError_t e = mode == kModeBf16      ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeBf16>, maps, blk)
+                        : mode == kModeInt8Smem ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Smem>, maps, blk)
+                                                : cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Tmem>, maps, blk);
   if (e != cudaSuccess) return check_cuda(ctx, e, "essa_decode_kernel launch");
   ctx->launches += 1;
   for (int i = 0; i < n; ++i) {
