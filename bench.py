@@ -40,7 +40,7 @@ METRIC = "candidate-tokens/sec through q/k/v/o SVD-LoRA projections"
 UNIT = "candidate-tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}  # chip figures, printed beside the measured ones
-ALL_CONFIGS = ("2", "3", "4", "5a", "5b")
+ALL_CONFIGS = ("2", "3", "4", "5a", "5b", "6a", "6b")  # 6a / 6b: the 72B-shaped block with INT4 group-wise weights
 HEADLINE = "4"
 L2_BYTES = 126e6
 CSRC = os.path.join(ROOT, "paper_2507_04453_b200", "csrc")
@@ -82,7 +82,7 @@ def load_peaks():
 def projection_work(n, m, r, T, P, w_bytes):
     """Algorithmic FLOPs and bytes of one projection call and of its dominant (base + up) kernel."""
     flops_call = 2.0 * T * m * n + 2.0 * T * r * (n + m + r) + 3.0 * T * r
-    bytes_call = m * n * w_bytes + (2 * m if w_bytes == 1 else 0) + 2.0 * T * n + 2.0 * T * m + 2.0 * n * r + 2.0 * m * r \
+    bytes_call = m * n * w_bytes + (2 * m if w_bytes == 1 else 2 * m * n / 128 if w_bytes == 0.5 else 0) + 2.0 * T * n + 2.0 * T * m + 2.0 * n * r + 2.0 * m * r \
         + 4.0 * r * r + 8.0 * P * r + 4.0 * (P + 1)
     flops_main = 2.0 * T * m * (n + r)                       # base contraction + up-projection
     bytes_main = m * n * w_bytes + 2.0 * T * n + 2.0 * T * m + 2.0 * m * r + 2.0 * T * r  # W0, x, y, U_B, u
@@ -93,7 +93,7 @@ def block_model(cfg, T):
     """Algorithmic work of the block's projection calls, each bounded by whichever of its FLOPs and bytes is slower
     at NOMINAL peak ratios (the bound does not depend on which measured peak is used: the configurations are far
     from the ridge except 3 and 5a, which are HBM-bound by bytes / copy bandwidth vs FLOPs / burst peak)."""
-    w = 1 if cfg.w0_dtype == "int8" else 2
+    w = {"int8": 1, "int4": 0.5}.get(cfg.w0_dtype, 2)  # bytes per weight as stored
     rows = []
     for _, n, m in cfg.projections:
         rows.append(projection_work(n, m, cfg.rank, T, cfg.P, w))
@@ -198,7 +198,8 @@ def oracle_setup(cfg, max_candidates=None):
     offsets = wl.make_segments(cfg)
     T = int(offsets[-1])
     cma = wl.make_cma_state(cfg, adapters)
-    weights = [a.W0.astype(np.float64) if a.w0_dtype == "bf16" else orc.dequantize_int8(a.W0_q, a.W0_scale) for a in adapters]
+    weights = [a.W0.astype(np.float64) if a.w0_dtype == "bf16" else orc.dequantize_int4(a.W0_q, a.W0_scale) if a.w0_dtype == "int4"
+               else orc.dequantize_int8(a.W0_q, a.W0_scale) for a in adapters]
     kmax = cfg.P if max_candidates is None else min(cfg.P, max_candidates)
     t_need = int(offsets[kmax])
     xs = []
@@ -296,7 +297,7 @@ def measure_config(key, cfg, args, env):
     # Weights that fit L2 (decode configurations) would be served from it on every step: rotate through enough
     # device copies of the block's adapters that each step streams its W0 from HBM, as a forward pass over many
     # layers does.
-    w_bytes = sum(a.d_in * a.d_out * (1 if cfg.w0_dtype == 'int8' else 2) for a in adapters)  # as stored
+    w_bytes = int(sum(a.d_in * a.d_out * {"int8": 1, "int4": 0.5}.get(cfg.w0_dtype, 2) for a in adapters))  # as stored
     copies = 1 if w_bytes > 2 * L2_BYTES else int(np.ceil(2 * L2_BYTES / w_bytes)) + 1
     handle_sets = [[ctx.load_adapter(a) for a in adapters] for _ in range(copies)]
     handles = handle_sets[0]
@@ -314,7 +315,7 @@ def measure_config(key, cfg, args, env):
     sigma = torch.empty((cfg.P, cfg.d), dtype=torch.float32, device="cuda")
     k_begin = rank * cfg.P  # weak scaling: rank g evaluates candidates [g*P, (g+1)*P) of an N*P population
     ctx.reserve(T, max(h.d_in for h in handles), max(h.d_out for h in handles))
-    if cfg.w0_dtype == "int8":
+    if cfg.w0_dtype != "bf16":
         ctx.reserve_dequant(max(h.d_in for h in handles), max(h.d_out for h in handles))
     stream = torch.cuda.current_stream()
 
@@ -496,7 +497,7 @@ def measure_config(key, cfg, args, env):
                 "block_frac_of_nominal": nominal["time_s"] * 1e3 / ms_per_step}
 
     rec = {"workload": cfg.name, "tokens_per_gpu_step": T, "candidates_per_gpu": cfg.P, "rank": cfg.rank,
-           "dtype": "bf16" if cfg.w0_dtype == "bf16" else "bf16 (int8 weights)",
+           "dtype": "bf16" if cfg.w0_dtype == "bf16" else f"bf16 ({cfg.w0_dtype} weights)",
            "projections": [f"{nm}:{n}->{m}" for nm, n, m in cfg.projections],
            "value": value, "steps": steps, "warmup": warmup,
            "ms_per_step": ms_per_step, "ms_per_step_median": float(np.median(per_group)), "ms_per_step_min": float(np.min(per_group)),

@@ -53,6 +53,11 @@ extern "C" {
 
 #define ESSA_W0_BF16 0            /* W0 stored as bf16                                               */
 #define ESSA_W0_INT8_PERCHANNEL 1 /* W0[o][i] = q[o][i] * scale[o], q int8, scale fp16 per out-channel */
+#define ESSA_W0_INT4_GROUP128 2   /* W0[o][i] = q[o][i] * scale[o][i / 128], q a 4-bit two's-complement code in [-8, 7]:
+                                     byte j of a row packs the codes of features 2j (low nibble) and 2j+1 (high
+                                     nibble); scale fp16 per (out-channel, group of 128 input features).  The paper
+                                     names the precision only (Section 5, precision study; the 72B runs); this
+                                     storage scheme is the library's reading.  d_in must be a multiple of 128. */
 
 #define ESSA_MAX_RANK 64
 #define ESSA_MAX_BLOCK_ITEMS 4 /* projections one essa_apply_block call takes (q, k, v, o of an attention block) */
@@ -103,9 +108,9 @@ typedef struct essa_adapter_desc {
   int32_t d_in;     /* n: input features.  Must be a multiple of 64.                           */
   int32_t d_out;    /* m: output features. Must be a multiple of 8.                            */
   int32_t rank;     /* r: LoRA rank, 1..ESSA_MAX_RANK                                          */
-  int32_t w0_dtype; /* ESSA_W0_BF16 or ESSA_W0_INT8_PERCHANNEL                                 */
-  const void* W0;       /* [d_out][d_in], bf16 or int8                                         */
-  const void* w0_scale; /* [d_out] fp16 (INT8 only; NULL for bf16)                             */
+  int32_t w0_dtype; /* ESSA_W0_BF16, ESSA_W0_INT8_PERCHANNEL or ESSA_W0_INT4_GROUP128          */
+  const void* W0;       /* [d_out][d_in] bf16 or int8; INT4: [d_out][d_in / 2] bytes           */
+  const void* w0_scale; /* INT8: [d_out] fp16; INT4: [d_out][d_in / 128] fp16; NULL for bf16   */
   const void* U_A;      /* [r][r]      bf16: left singular vectors of A                        */
   const void* V_A;      /* [d_in][r]   bf16: right singular vectors of A                       */
   const void* U_B;      /* [d_out][r]  bf16: left singular vectors of B                        */

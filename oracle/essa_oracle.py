@@ -22,7 +22,9 @@ test against the normal CDF; identity/orthogonal covariance special cases and th
 empirical covariance; SVD round trip (sigma = singular values of the LoRA factors
 reproduces B.A); the M = I special case checked with a library SVD; zero sigma
 reproduces W0.x exactly; bilinearity in (sA, sB); brute-force scalar loops on tiny
-shapes; linear-scan segment map vs a library search.
+shapes; linear-scan segment map vs a library search; INT4 dequantisation against
+scalar loops, against the nibble table written out, and against the INT8 path when
+the codes fit four bits and a row's groups share one scale.
 
 Parity unpinned: the paper prints no worked numeric example for either function,
 so both are pinned by identities, special cases, library routines and brute force
@@ -155,6 +157,22 @@ def candidate_of_token(offsets, T: int) -> np.ndarray:
 def dequantize_int8(q, scale) -> np.ndarray:
     """W0[o,i] = q[o,i] * scale[o] in fp64 (weight-only INT8 storage of the frozen base)."""
     return np.asarray(q).astype(np.float64) * np.asarray(scale).astype(np.float64)[:, None]
+
+
+def dequantize_int4(packed, scale, group: int = 128) -> np.ndarray:
+    """W0[o,i] = q[o,i] * scale[o, i // group] in fp64 (weight-only INT4 storage of the frozen base, group-wise scales).
+
+    packed is uint8 [m, n/2]: byte j of a row holds the codes of input features 2j (low nibble) and 2j+1 (high nibble),
+    each a 4-bit two's-complement integer in [-8, 7]; scale is fp16 [m, n/group].  The paper only names the precision
+    ("INT4", Section 5 precision study); this storage scheme is the build's reading of it."""
+    packed = np.asarray(packed, dtype=np.uint8)
+    m, half = packed.shape
+    codes = np.empty((m, 2 * half), dtype=np.int64)
+    codes[:, 0::2] = packed & 0x0F
+    codes[:, 1::2] = packed >> 4
+    codes = np.where(codes >= 8, codes - 16, codes)
+    sc = np.asarray(scale).astype(np.float64)
+    return codes.astype(np.float64) * np.repeat(sc, group, axis=1)
 
 
 def reconstruct_factors(U_A, V_A, U_B, V_B, sA, sB):

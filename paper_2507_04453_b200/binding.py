@@ -25,6 +25,7 @@ ESSA_ERR_DEVICE_TIMEOUT = -5
 ESSA_ERR_NO_DEVICE = -6
 ESSA_W0_BF16 = 0
 ESSA_W0_INT8_PERCHANNEL = 1
+ESSA_W0_INT4_GROUP128 = 2
 ESSA_OPT_PAIR_TILES = 1
 ESSA_OPT_FUSE_DOWN = 2
 
@@ -371,6 +372,10 @@ class Context:
         if ad.w0_dtype == "bf16":
             keep["W0"] = bf(ad.W0)
             dtype, scale_ptr = ESSA_W0_BF16, None
+        elif ad.w0_dtype == "int4":  # two 4-bit codes per byte, fp16 scale per (channel, group of 128 features)
+            keep["W0"] = torch.from_numpy(np.ascontiguousarray(ad.W0_q, dtype=np.uint8))
+            keep["scale"] = torch.from_numpy(np.ascontiguousarray(ad.W0_scale, dtype=np.float16))
+            dtype, scale_ptr = ESSA_W0_INT4_GROUP128, keep["scale"].data_ptr()
         else:
             keep["W0"] = torch.from_numpy(np.ascontiguousarray(ad.W0_q, dtype=np.int8))
             keep["scale"] = torch.from_numpy(np.ascontiguousarray(ad.W0_scale, dtype=np.float16))

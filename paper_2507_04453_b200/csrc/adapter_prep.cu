@@ -58,6 +58,24 @@ __global__ void widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* _
   reinterpret_cast<uint4*>(out + i)[1] = o1;
 }
 
+// INT4 group-wise codes -> bf16 weights (code * group scale, rounded once), 32 codes (16 bytes) per thread; the 32
+// codes of a thread share a group (groups are 128 wide and d_in is a multiple of 128).
+__global__ void widen_int4_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ gscale, __nv_bfloat16* __restrict__ out,
+                                  int d_in, size_t count) {
+  const size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 32;  // first weight of this thread
+  if (i >= count) return;
+  const size_t o = i / d_in, c = i % d_in;
+  const float s = __half2float(gscale[o * (d_in / 128) + c / 128]);
+  const uint4 w = *reinterpret_cast<const uint4*>(packed + i / 2);
+  const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    uint32_t v[4];
+    int4x8_to_bf16x8(ws[k], s, v);
+    *reinterpret_cast<uint4*>(out + i + 8 * k) = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
 // Candidate reconstruction (Algorithm 1, line 7: A' = U_A diag(sA_k) V_A^T, B' = U_B diag(sB_k) V_B^T), for export to
 // an engine that wants the dense LoRA factors.  CUDA cores: 2 r^2 (n + m) FLOP per candidate against 2 r (n + m)
 // bytes written, i.e. r FLOP per byte; RP = rank rounded up to 16 keeps the per-thread vectors in registers.
@@ -167,6 +185,16 @@ int32_t launch_export_candidates(essa_ctx* ctx, const essa_adapter* a, const flo
     ctx->launches += 1;
   }
   return check_cuda(ctx, cudaGetLastError(), "export_candidates launch");
+}
+
+int32_t launch_widen_int4(essa_ctx* ctx, const uint8_t* packed, const __half* gscale, __nv_bfloat16* out, int d_out, int d_in,
+                          cudaStream_t stream) {
+  const size_t count = (size_t)d_out * d_in;
+  if (count == 0) return ESSA_OK;
+  const size_t threads = count / 32;
+  widen_int4_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(packed, gscale, out, d_in, count);
+  ctx->launches += 1;
+  return check_cuda(ctx, cudaGetLastError(), "widen_int4 launch");
 }
 
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream) {

@@ -286,11 +286,13 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   if (d->rank > ESSA_MAX_RANK) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: rank > 64");
   if (d->d_in % 64 != 0) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: d_in must be a multiple of 64");
   if (d->d_out % 8 != 0) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: d_out must be a multiple of 8");
-  if (d->w0_dtype != ESSA_W0_BF16 && d->w0_dtype != ESSA_W0_INT8_PERCHANNEL)
+  if (d->w0_dtype != ESSA_W0_BF16 && d->w0_dtype != ESSA_W0_INT8_PERCHANNEL && d->w0_dtype != ESSA_W0_INT4_GROUP128)
     return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: unknown w0_dtype");
   if (!d->W0 || !d->U_A || !d->V_A || !d->U_B || !d->V_B) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: NULL matrix");
   const bool int8 = d->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
-  if (int8 && !d->w0_scale) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: INT8 W0 needs w0_scale");
+  const bool int4 = d->w0_dtype == ESSA_W0_INT4_GROUP128;
+  if ((int8 || int4) && !d->w0_scale) return fail(ctx, ESSA_ERR_INVALID_ARG, "load_adapter: quantised W0 needs w0_scale");
+  if (int4 && d->d_in % 128 != 0) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "load_adapter: INT4 storage needs d_in to be a multiple of 128");
 
   essa_adapter* a = new (std::nothrow) essa_adapter();
   if (!a) return fail(ctx, ESSA_ERR_ALLOC, "load_adapter: host allocation failed");
@@ -304,8 +306,9 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   const size_t w0_bytes = m * n * 2;
   cudaError_t e = cudaSuccess;
   auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
-  if (!int8) alloc(&a->W0, w0_bytes);
+  if (!int8 && !int4) alloc(&a->W0, w0_bytes);
   if (int8) { alloc((void**)&a->w0_scale, m * 2); alloc((void**)&a->W0q, m * n); }
+  if (int4) { alloc((void**)&a->w0_gscale, m * (n / 128) * 2); alloc((void**)&a->W0q, m * n / 2); }
   alloc((void**)&a->VAt, (size_t)kRankPadMax * n * 2);
   alloc((void**)&a->UBp, (size_t)a->ext_blocks * m * kRankPadMax * 2);
   alloc((void**)&a->U_B, m * r * 2);
@@ -322,8 +325,9 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   auto copy = [&](void* dst, const void* src, size_t bytes) {
     if (st == ESSA_OK) st = check_cuda(ctx, cudaMemcpyAsync(dst, src, bytes, kind, stream), "load_adapter: copy");
   };
-  copy(int8 ? (void*)a->W0q : a->W0, d->W0, int8 ? m * n : w0_bytes);
+  copy((int8 || int4) ? (void*)a->W0q : a->W0, d->W0, int8 ? m * n : int4 ? m * n / 2 : w0_bytes);
   if (int8) copy(a->w0_scale, d->w0_scale, m * 2);
+  if (int4) copy(a->w0_gscale, d->w0_scale, m * (n / 128) * 2);
   copy(a->U_B, d->U_B, m * r * 2);
   copy(a->V_A, d->V_A, n * r * 2);
   copy(a->U_A, d->U_A, r * r * 2);
@@ -332,13 +336,14 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
   if (st == ESSA_OK) {
     const uint32_t rows[3] = {64, 128, 256};
     for (int i = 0; i < 3 && st == ESSA_OK; ++i) {
-      if (!int8) st = make_tensor_map_2d(ctx, &a->tm_W0[i], 0, a->W0, m, n, n * 2, rows[i], 64, 128);
+      if (!int8 && !int4) st = make_tensor_map_2d(ctx, &a->tm_W0[i], 0, a->W0, m, n, n * 2, rows[i], 64, 128);
       for (int e2 = 0; e2 < a->ext_blocks && st == ESSA_OK; ++e2)
         st = make_tensor_map_2d(ctx, &a->tm_UBp[i][e2], 0, a->UBp + (size_t)e2 * m * kRankPadMax, m, kRankPadMax,
                                 kRankPadMax * 2, rows[i], 64, 128);
     }
     if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q, 1, a->W0q, m, n, n, 128, 64, 0);
     if (st == ESSA_OK && int8) st = make_tensor_map_2d(ctx, &a->tm_W0q64, 1, a->W0q, m, n, n, 128, 64, 64);
+    if (st == ESSA_OK && int4) st = make_tensor_map_2d(ctx, &a->tm_W0q4, 1, a->W0q, m, n / 2, n / 2, 128, 32, 32);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAt, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad, 64, 128);
     if (st == ESSA_OK) st = make_tensor_map_2d(ctx, &a->tm_VAtH, 0, a->VAt, kRankPadMax, n, n * 2, a->r_pad / 2, 64, 128);
   }
@@ -357,7 +362,7 @@ int32_t essa_load_adapter(essa_ctx* ctx, const essa_adapter_desc* d, essa_adapte
 int32_t essa_free_adapter(essa_ctx* ctx, essa_adapter* a) {
   if (!ctx || !a) return ESSA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->VAt, a->UBp, a->U_B, a->V_A, a->U_A, a->V_B, a->M};
+  void* ptrs[] = {a->W0, a->W0q, a->w0_scale, a->w0_gscale, a->VAt, a->UBp, a->U_B, a->V_A, a->U_A, a->V_B, a->M};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   delete a;
@@ -670,7 +675,7 @@ int32_t essa_plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t 
                              essa_plan* out) {
   if (!out || d_in <= 0 || d_out <= 0 || rank <= 0 || T < 0) return ESSA_ERR_INVALID_ARG;
   if (rank > ESSA_MAX_RANK || d_in % 64 != 0 || d_out % 8 != 0) return ESSA_ERR_UNSUPPORTED_SHAPE;
-  if (w0_dtype != ESSA_W0_BF16 && w0_dtype != ESSA_W0_INT8_PERCHANNEL) return ESSA_ERR_INVALID_ARG;
+  if (w0_dtype != ESSA_W0_BF16 && w0_dtype != ESSA_W0_INT8_PERCHANNEL && w0_dtype != ESSA_W0_INT4_GROUP128) return ESSA_ERR_INVALID_ARG;
   plan_projection(d_in, d_out, rank, w0_dtype, T, sm_count, out);
   return ESSA_OK;
 }

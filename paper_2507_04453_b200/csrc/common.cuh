@@ -80,6 +80,7 @@ struct essa_adapter {
   void* W0 = nullptr;            // [d_out][d_in] bf16 (bf16 storage only)
   int8_t* W0q = nullptr;         // [d_out][d_in] int8 codes as given (INT8 storage only)
   __half* w0_scale = nullptr;    // [d_out] fp16 (INT8)
+  __half* w0_gscale = nullptr;   // [d_out][d_in / 128] fp16 (INT4; W0q then holds two codes per byte, [d_out][d_in / 2])
   __nv_bfloat16* VAt = nullptr;  // [64][d_in]: V_A^T, rows >= rank are zero (K-major operand of the down-projection)
   __nv_bfloat16* UBp = nullptr;  // [ext][d_out][64]: U_B zero-padded to 64 columns; INT8: (U_B/scale) split hi, lo
   __nv_bfloat16* U_B = nullptr;  // [d_out][rank] as given (CUDA-core path)
@@ -94,6 +95,7 @@ struct essa_adapter {
   CUtensorMap tm_VAtH;           // the same with boxes of r_pad / 2 rows (one CTA's half in the pair kernel)
   CUtensorMap tm_W0q;            // INT8 storage: the codes, 128-row x 64-byte boxes, unswizzled
   CUtensorMap tm_W0q64;          // ... the same boxes with the 64-byte swizzle (row-per-thread readers)
+  CUtensorMap tm_W0q4;           // INT4 storage: the packed codes, 128-row x 32-byte boxes, 32-byte swizzle
 };
 
 namespace essa {
@@ -121,6 +123,9 @@ int32_t launch_segment_map(essa_ctx* ctx, const int32_t* seg_offsets, int32_t P,
 
 // adapter_prep.cu
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream);
+// INT4 group-wise storage -> bf16 weights (code * group scale, one rounding): out [d_out][d_in].
+int32_t launch_widen_int4(essa_ctx* ctx, const uint8_t* packed, const __half* gscale, __nv_bfloat16* out, int d_out, int d_in,
+                          cudaStream_t stream);
 int32_t launch_adapter_prep(essa_ctx* ctx, essa_adapter* a, const __nv_bfloat16* U_A, const __nv_bfloat16* V_B,
                             cudaStream_t stream);
 // Reconstructed factors of candidates k_begin .. k_begin + k_count - 1: A_out [k][rank][d_in], B_out [k][d_out][rank] bf16.
@@ -193,6 +198,24 @@ __device__ __forceinline__ void int8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint3
   const __nv_bfloat162 q1 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&p1), *reinterpret_cast<const __nv_bfloat162*>(&d1));
   lo = *reinterpret_cast<const uint32_t*>(&q0);
   hi = *reinterpret_cast<const uint32_t*>(&q1);
+}
+
+// Four packed INT4 bytes (eight codes, memory order: low nibble first) -> eight bf16 values = code * s, one rounding
+// each.  A nibble n is the two's-complement code (n ^ 8) - 8; 0x4300 | (n ^ 8) is the bf16 number 128 + (n ^ 8), and
+// subtracting 136 leaves the code exactly; the product with the fp16 group scale is formed in fp32.
+__device__ __forceinline__ void int4x8_to_bf16x8(uint32_t w, float s, uint32_t (&out)[4]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t t = (w >> (8 * j)) & 0xffu;
+    uint32_t pair = ((t & 0x0fu) | ((t & 0xf0u) << 12)) ^ 0x00080008u;
+    pair |= 0x43004300u;
+    const uint32_t bias = 0x43084308u;
+    const __nv_bfloat162 q = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&pair), *reinterpret_cast<const __nv_bfloat162*>(&bias));
+    const uint32_t qb = *reinterpret_cast<const uint32_t*>(&q);
+    const float lo = __uint_as_float(qb << 16) * s, hi = __uint_as_float(qb & 0xffff0000u) * s;
+    const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+    out[j] = *reinterpret_cast<const uint32_t*>(&r);
+  }
 }
 
 // Largest k in [0, P-1] with off[k] <= t (candidate that owns token t; empty segments own nothing).

@@ -55,7 +55,10 @@ constexpr int RAW_TILE_BYTES = DEC_M * DEC_K;    // 8 KB: one W0 tile as stored 
 // most 128 tokens, so that tensor memory has room): the four warps write the converted tile straight into TENSOR
 // memory (tcgen05.st, thread = row of the tile) and the MMA takes its A operand from there, which removes the
 // write and the read of the converted tile from the shared-memory traffic that bounds the other INT8 mode.
-constexpr int kModeBf16 = 0, kModeInt8Smem = 1, kModeInt8Tmem = 2;
+// kModeInt4Tmem: the same for INT4 group-wise storage (4 KB tiles of packed codes, the group scale folded into the
+// bf16 value by the converting thread).
+constexpr int kModeBf16 = 0, kModeInt8Smem = 1, kModeInt8Tmem = 2, kModeInt4Tmem = 3;
+constexpr int RAW4_TILE_BYTES = DEC_M * DEC_K / 2;  // 4 KB: one W0 tile as packed INT4 codes
 constexpr int kTmemAStages = 8;                  // converted tiles in tensor memory (32 columns each)
 constexpr int kUbSlots = 2;                      // kModeInt8Tmem: the U_B slabs have shared-memory slots of their own
 constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
@@ -79,6 +82,7 @@ struct DParams {
   __nv_bfloat16* y;
   int ldy;
   const __half* scale;
+  const __half* gscale;      // INT4 storage: [d_out][d_in / 128] group scales (folded into the converted values)
   // rank path
   int r_pad;                 // rank rows of a V_A^T tile (the TMA box): 16 / 32 / 48 / 64
   int p_c;                   // K blocks per slice: CTA (m_tile j, split s) owns local K blocks [j p_c, (j+1) p_c)
@@ -261,7 +265,8 @@ template <int MODE>
 __global__ void __launch_bounds__(MODE != kModeBf16 ? kDecThreadsInt8 : kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ DBlock blk) {
   constexpr bool INT8 = MODE == kModeInt8Smem;   // codes converted through shared memory
-  constexpr bool TS = MODE == kModeInt8Tmem;     // codes converted into tensor memory (A operand from TMEM)
+  constexpr bool TS = MODE >= kModeInt8Tmem;     // codes converted into tensor memory (A operand from TMEM)
+  constexpr bool I4 = MODE == kModeInt4Tmem;     // ... from packed INT4 codes with group-wise scales
   constexpr bool QUANT = MODE != kModeBf16;
   // which projection this CTA streams (CTAs past the last one only take rank-path units)
   int pi = 0;
@@ -277,7 +282,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
   const int x_bytes = p.tn * 128;
-  constexpr int W_SLOT = QUANT ? RAW_TILE_BYTES : W_TILE_BYTES;
+  constexpr int W_SLOT = I4 ? RAW4_TILE_BYTES : QUANT ? RAW_TILE_BYTES : W_TILE_BYTES;
   const int SC = INT8 ? p.c_stages : (TS ? kUbSlots : 0);   // 16 KB slots behind the W0 ring
   const int SA = TS ? p.c_stages : 1;                       // kModeInt8Tmem: converted tiles in tensor memory
   // V_A^T tiles first: their MMA descriptor spans 128 rows, of which only the r_pad rows of the TMA box are data
@@ -328,7 +333,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     mbar_expect_tx(fb, (uint32_t)W_SLOT);
     const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
     if (QUANT) {  // 128 rows of 64 codes (unswizzled; kModeInt8Tmem: 64-byte swizzle)
-      tma_load_2d(dst, &tmW, kcol(i), m_tile * DEC_M, fb);
+      tma_load_2d(dst, &tmW, I4 ? kcol(i) / 2 : kcol(i), m_tile * DEC_M, fb);
     } else {     // one 128-row box
       const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
       tma_load_2d(dst, tm, i < nkb ? kcol(i) : 0, m_tile * DEC_M, fb);
@@ -622,17 +627,40 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       if (i >= SA) while (!mbar_try_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1))) {}
       while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}
       tc_fence_after();  // the MMAs that read this stage have completed (their commit released it)
-      const uint32_t raw = smem_u32(smem_w + sr * RAW_TILE_BYTES) + (uint32_t)(r * 64);
-      uint4 w[4];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) w[c] = lds_v4(raw + (uint32_t)((c ^ ((r >> 1) & 3)) << 4));
       uint32_t v[32];
+      if (I4) {
+        // a row of the tile is 32 bytes = two 16-byte chunks, loaded with the 32-byte swizzle (chunk c of row r at
+        // position c ^ ((r >> 2) & 1): again eight different bank groups per quarter-warp); the 64 codes of the row
+        // lie in one group of 128 input features and share its scale
+        const uint32_t raw = smem_u32(smem_w + sr * W_SLOT) + (uint32_t)(r * 32);
+        const int ch = m_tile * DEC_M + r;
+        const float gs = ch < p.d_out ? __half2float(__ldg(p.gscale + (size_t)ch * (p.d_in >> 7) + (kcol(i) >> 7))) : 0.f;
+        uint4 w[2];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        int8x4_to_bf16x4(w[c].x, v[8 * c + 0], v[8 * c + 1]);
-        int8x4_to_bf16x4(w[c].y, v[8 * c + 2], v[8 * c + 3]);
-        int8x4_to_bf16x4(w[c].z, v[8 * c + 4], v[8 * c + 5]);
-        int8x4_to_bf16x4(w[c].w, v[8 * c + 6], v[8 * c + 7]);
+        for (int c = 0; c < 2; ++c) w[c] = lds_v4(raw + (uint32_t)((c ^ ((r >> 2) & 1)) << 4));
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const uint32_t ws[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            uint32_t o4[4];
+            int4x8_to_bf16x8(ws[k], gs, o4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[16 * c + 4 * k + e] = o4[e];
+          }
+        }
+      } else {
+        const uint32_t raw = smem_u32(smem_w + sr * W_SLOT) + (uint32_t)(r * 64);
+        uint4 w[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[c] = lds_v4(raw + (uint32_t)((c ^ ((r >> 1) & 3)) << 4));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          int8x4_to_bf16x4(w[c].x, v[8 * c + 0], v[8 * c + 1]);
+          int8x4_to_bf16x4(w[c].y, v[8 * c + 2], v[8 * c + 3]);
+          int8x4_to_bf16x4(w[c].z, v[8 * c + 4], v[8 * c + 5]);
+          int8x4_to_bf16x4(w[c].w, v[8 * c + 6], v[8 * c + 7]);
+        }
       }
       tmem_st32(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(sa), v);
       tc_fence_before();
@@ -771,22 +799,27 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
 
 // Shared-memory rings: V_A^T tiles, the W0 ring (16 KB bf16 tiles, or 8 KB tiles of codes), the 16 KB slots behind it
 // (kModeInt8Smem: c_stages converted tiles; kModeInt8Tmem: the U_B slabs), the x ring.
+inline int dec_w_slot(int mode) { return mode == kModeBf16 ? W_TILE_BYTES : mode == kModeInt4Tmem ? RAW4_TILE_BYTES : RAW_TILE_BYTES; }
 inline int dec_ring_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
-  const int slots16k = mode == kModeInt8Smem ? c_stages : mode == kModeInt8Tmem ? kUbSlots : 0;
-  return kVatStages * VAT_SLOT_BYTES + w_stages * (mode != kModeBf16 ? RAW_TILE_BYTES : W_TILE_BYTES) + slots16k * W_TILE_BYTES +
-         x_stages * tn * 128;
+  const int slots16k = mode == kModeInt8Smem ? c_stages : mode >= kModeInt8Tmem ? kUbSlots : 0;
+  return kVatStages * VAT_SLOT_BYTES + w_stages * dec_w_slot(mode) + slots16k * W_TILE_BYTES + x_stages * tn * 128;
 }
 inline int dec_smem_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
   return 1024 + dec_ring_bytes(mode, w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
 }
 // INT8 storage converts into tensor memory whenever the accumulators leave room for the converted tiles there.
-inline int dec_mode(bool int8, int tn) { return !int8 ? kModeBf16 : tn <= 128 ? kModeInt8Tmem : kModeInt8Smem; }
+// INT4 storage has the tensor-memory mode only: larger calls take the prefill kernels (negative: no decode schedule).
+inline int dec_mode(int w0_dtype, int tn) {
+  if (w0_dtype == ESSA_W0_BF16) return kModeBf16;
+  if (w0_dtype == ESSA_W0_INT4_GROUP128) return tn <= 128 ? kModeInt4Tmem : -1;
+  return tn <= 128 ? kModeInt8Tmem : kModeInt8Smem;
+}
 
 }  // namespace
 
 // Schedule shared by the projections of one decode launch (n of them, sizes d_in[i] -> d_out[i], same storage type):
 // cluster size, ring depths.  Returns false when the launch would not fit one wave of the GPU.
-static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int8, int64_t T, int sm_count, int* splits_out,
+static bool plan_decode_block(int n, const int* d_in, const int* d_out, int w0_dtype, int64_t T, int sm_count, int* splits_out,
                               int* w_stages_out, int* x_stages_out, int* m_tiles_total_out, int* c_stages_out = nullptr) {
   if (T <= 0 || T > kDecodeMaxTokens || n < 1 || n > kMaxBlockProj) return false;
   const int sm = sm_count > 0 ? sm_count : 148;
@@ -808,9 +841,10 @@ static bool plan_decode_block(int n, const int* d_in, const int* d_out, bool int
   // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
   // INT8 storage: W0 tiles travel as 8 KB of codes; a ring of converted bf16 tiles (which also takes the U_B slabs,
   // loaded into it directly) sits between the converting warps and the tensor core.
-  const int mode = dec_mode(int8, tn);
-  const int c_stages = mode == kModeInt8Smem ? kInt8ConvStages : mode == kModeInt8Tmem ? kTmemAStages : 0;
-  const int w_slot = int8 ? RAW_TILE_BYTES : W_TILE_BYTES;
+  const int mode = dec_mode(w0_dtype, tn);
+  if (mode < 0) return false;
+  const int c_stages = mode == kModeInt8Smem ? kInt8ConvStages : mode >= kModeInt8Tmem ? kTmemAStages : 0;
+  const int w_slot = dec_w_slot(mode);
   const int xb = tn * 128;
   const int budget = kDecSmemBudget - dec_smem_bytes(mode, 0, c_stages, 0, tn);
   int x_stages = budget / (w_slot + xb);
@@ -835,7 +869,7 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
   const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   int splits, w_stages, x_stages, m_tiles;
   const int di = d_in, dout = d_out;
-  if (!plan_decode_block(1, &di, &dout, int8, T, sm_count, &splits, &w_stages, &x_stages, &m_tiles)) return false;
+  if (!plan_decode_block(1, &di, &dout, w0_dtype, T, sm_count, &splits, &w_stages, &x_stages, &m_tiles)) return false;
   out->block_m = DEC_M;
   out->block_n = (int)((T + 15) / 16) * 16;
   out->block_k = DEC_K;
@@ -859,30 +893,33 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
                             const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready,
                             uint32_t sigma_target) {
   if (n < 1 || n > kMaxBlockProj || T <= 0 || T > kDecodeMaxTokens) return kBlockNotFused;
-  const bool int8 = items[0].a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  const int w0_dtype = items[0].a->w0_dtype;
+  const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   int d_in[kMaxBlockProj], d_out[kMaxBlockProj];
   for (int i = 0; i < n; ++i) {
-    if ((items[i].a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) != int8) return kBlockNotFused;
+    if (items[i].a->w0_dtype != w0_dtype) return kBlockNotFused;
     d_in[i] = items[i].a->d_in;
     d_out[i] = items[i].a->d_out;
   }
   int splits, w_stages, x_stages, m_total, c_stages;
-  if (!plan_decode_block(n, d_in, d_out, int8, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total, &c_stages)) {
+  if (!plan_decode_block(n, d_in, d_out, w0_dtype, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total, &c_stages)) {
     if (n > 1) return kBlockNotFused;
     return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: no decode schedule fits shared memory");
   }
   const int tn = (int)((T + 15) / 16) * 16;
-  const int mode = dec_mode(int8, tn);
+  const int mode = dec_mode(w0_dtype, tn);
+  if (mode < 0) return kBlockNotFused;
 
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
-  static int resident_caches[64][3][9] = {};  // per device, kernel mode, cluster size
+  static int resident_caches[64][4][9] = {};  // per device, kernel mode, cluster size
   int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
   const void* kernel = mode == kModeBf16      ? (const void*)essa_decode_kernel<kModeBf16>
                        : mode == kModeInt8Smem ? (const void*)essa_decode_kernel<kModeInt8Smem>
-                                               : (const void*)essa_decode_kernel<kModeInt8Tmem>;
-  const int threads = int8 ? kDecThreadsInt8 : kDecThreads;
+                       : mode == kModeInt8Tmem ? (const void*)essa_decode_kernel<kModeInt8Tmem>
+                                               : (const void*)essa_decode_kernel<kModeInt4Tmem>;
+  const int threads = mode != kModeBf16 ? kDecThreadsInt8 : kDecThreads;
   {
-    static bool attr_done[64][3] = {};  // the attribute is per device and kernel instance
+    static bool attr_done[64][4] = {};  // the attribute is per device and kernel instance
     bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
     if (!done) {
       const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
@@ -944,6 +981,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     p.y = items[i].y;
     p.ldy = a->d_out;
     p.scale = int8 ? a->w0_scale : nullptr;
+    p.gscale = a->w0_gscale;
     p.r_pad = a->r_pad;
     p.rank_groups = ((int)T + kFinishTokens - 1) / kFinishTokens;
     // slices of the down-projection: the K blocks of a split are dealt to the first row tiles, p_c each, at most
@@ -984,7 +1022,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     cta += p.m_tiles * splits;
     unit += p.rank_groups;
 
-    maps.tm[i][0] = mode == kModeInt8Tmem ? a->tm_W0q64 : int8 ? a->tm_W0q : a->tm_W0[1];  // 128-row boxes of bf16 W0 / of codes
+    maps.tm[i][0] = mode == kModeInt4Tmem ? a->tm_W0q4 : mode == kModeInt8Tmem ? a->tm_W0q64 : int8 ? a->tm_W0q : a->tm_W0[1];  // 128-row boxes of bf16 W0 / of codes
     // activation map: looked up by (pointer, tokens, features, box); u map: one per (projection slot, box)
     {
       essa_ctx::XMapEntry* hit = nullptr;
@@ -1033,7 +1071,8 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   cfg.numAttrs = 2;
   const cudaError_t e = mode == kModeBf16      ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeBf16>, maps, blk)
                         : mode == kModeInt8Smem ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Smem>, maps, blk)
-                                                : cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Tmem>, maps, blk);
+                        : mode == kModeInt8Tmem ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Tmem>, maps, blk)
+                                                : cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt4Tmem>, maps, blk);
   if (e != cudaSuccess) return check_cuda(ctx, e, "essa_decode_kernel launch");
   ctx->launches += 1;
   for (int i = 0; i < n; ++i) {

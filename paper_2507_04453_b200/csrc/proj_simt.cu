@@ -45,7 +45,8 @@ __global__ void __launch_bounds__(256) simt_rank_kernel(const __nv_bfloat16* __r
 }
 
 // 64 x 64 output tile per CTA, 16-wide K chunks, 4 x 4 outputs per thread.
-template <bool kInt8>
+// kQ: 0 = bf16 W0, 1 = INT8 codes with a per-channel scale, 2 = INT4 codes (two per byte) with per-group scales.
+template <int kQ>
 __global__ void __launch_bounds__(256) simt_gemm_kernel(const __nv_bfloat16* __restrict__ x, int T, int n, int m, int r,
                                                         const void* __restrict__ W0v, const __half* __restrict__ scale,
                                                         const __nv_bfloat16* __restrict__ U_B,
@@ -87,11 +88,18 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const __nv_bfloat16* __r
   // base contraction W0 x
   tile_pass([&](int t, int c) { return __bfloat162float(x[(size_t)t * n + c]); },
             [&](int o, int c) {
-              if constexpr (kInt8) return (float)reinterpret_cast<const int8_t*>(W0v)[(size_t)o * n + c];
-              else return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W0v)[(size_t)o * n + c]);
+              if constexpr (kQ == 1) {
+                return (float)reinterpret_cast<const int8_t*>(W0v)[(size_t)o * n + c];
+              } else if constexpr (kQ == 2) {
+                const uint32_t byte = reinterpret_cast<const uint8_t*>(W0v)[((size_t)o * n + c) >> 1];
+                const int nib = (c & 1) ? (int)(byte >> 4) : (int)(byte & 15u);
+                return (float)((nib ^ 8) - 8) * __half2float(scale[(size_t)o * (n / 128) + c / 128]);
+              } else {
+                return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W0v)[(size_t)o * n + c]);
+              }
             },
             n);
-  if constexpr (kInt8) {
+  if constexpr (kQ == 1) {
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
       const int o = o0 + tx * 4 + b;
@@ -127,11 +135,11 @@ int32_t launch_projection_simt(essa_ctx* ctx, const essa_adapter* a, const ProjA
                                                       g.ld_sigma, g.sA_col, g.sB_col, u);
   dim3 grid((a->d_out + 63) / 64, (unsigned)((g.T + 63) / 64));
   if (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL)
-    simt_gemm_kernel<true><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0q, a->w0_scale,
-                                                     a->U_B, u, g.y);
+    simt_gemm_kernel<1><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0q, a->w0_scale, a->U_B, u, g.y);
+  else if (a->w0_dtype == ESSA_W0_INT4_GROUP128)
+    simt_gemm_kernel<2><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0q, a->w0_gscale, a->U_B, u, g.y);
   else
-    simt_gemm_kernel<false><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0, nullptr, a->U_B,
-                                                      u, g.y);
+    simt_gemm_kernel<0><<<grid, 256, 0, stream>>>(g.x, (int)g.T, a->d_in, a->d_out, a->rank, a->W0, nullptr, a->U_B, u, g.y);
   ctx->launches += 2;
   return check_cuda(ctx, cudaGetLastError(), "simt projection launch");
 }

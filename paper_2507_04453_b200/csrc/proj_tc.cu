@@ -540,11 +540,14 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
 
   // ---- INT8 storage: dequantise the codes (unscaled, exact) into the context's scratch for this call's GEMM
   CUtensorMap tm_wdeq;
-  if (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) {
+  if (a->w0_dtype != ESSA_W0_BF16) {
     const size_t cnt = (size_t)a->d_out * a->d_in;
     st = ensure_scratch(ctx, ctx->w_deq, cnt * 2, false, stream);
     if (st != ESSA_OK) return st;
-    st = launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr), cnt, stream);
+    st = a->w0_dtype == ESSA_W0_INT8_PERCHANNEL
+             ? launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr), cnt, stream)
+             : launch_widen_int4(ctx, reinterpret_cast<const uint8_t*>(a->W0q), a->w0_gscale, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr),
+                                 a->d_out, a->d_in, stream);
     if (st != ESSA_OK) return st;
     st = make_tensor_map_2d(ctx, &tm_wdeq, 0, ctx->w_deq.ptr, (uint64_t)a->d_out, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
                             (uint32_t)(use_pairs ? 128 : pl.block_n), BLOCK_K, 128);
@@ -633,7 +636,7 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   mp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
   mp.status = ctx->d_status;
   if (use_pairs) {
-    const CUtensorMap& tmW128 = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? tm_wdeq : a->tm_W0[1];
+    const CUtensorMap& tmW128 = (a->w0_dtype != ESSA_W0_BF16) ? tm_wdeq : a->tm_W0[1];
     st = launch_base_up_pair(ctx, tm_x, tmW128, tm_u, a->tm_UBp[1][0], a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0], (int)g.T,
                              a->d_out, a->d_in / BLOCK_K, a->ext_blocks, a->r_pad / UMMA_K, g.y, mp.scale, fused ? &pd : nullptr,
                              stream);
@@ -642,7 +645,7 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     return st;
   }
   const int bi = pl.block_n == 64 ? 0 : pl.block_n == 128 ? 1 : 2;
-  const CUtensorMap& tmW = (a->w0_dtype == ESSA_W0_INT8_PERCHANNEL) ? tm_wdeq : a->tm_W0[bi];
+  const CUtensorMap& tmW = (a->w0_dtype != ESSA_W0_BF16) ? tm_wdeq : a->tm_W0[bi];
   const CUtensorMap& tmU0 = a->tm_UBp[bi][0];
   const CUtensorMap& tmU1 = a->tm_UBp[bi][a->ext_blocks > 1 ? 1 : 0];
   switch (pl.block_n) {
@@ -690,11 +693,11 @@ int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const 
     g_static_u_addr[cur] = p;
   }
   __nv_bfloat16* u = static_cast<__nv_bfloat16*>(g_static_u_addr[cur]);
-  // INT8 storage: the call dequantises W0 into the context's scratch, which this entry point will not grow.
-  const bool int8 = a->w0_dtype == ESSA_W0_INT8_PERCHANNEL;
+  // INT8 / INT4 storage: the call dequantises W0 into the context's scratch, which this entry point will not grow.
+  const bool int8 = a->w0_dtype != ESSA_W0_BF16;  // (any quantised storage)
   if (int8 && ctx->w_deq.bytes < (size_t)a->d_out * a->d_in * 2)
     return fail(ctx, ESSA_ERR_ALLOC,
-                "apply_projection_static: INT8 weights need the context's dequantisation scratch, which is not large "
+                "apply_projection_static: quantised weights need the context's dequantisation scratch, which is not large "
                 "enough yet; size it once with essa_reserve_dequant (this entry point does not allocate)");
 
   // Same two launches as essa_apply_projection, with split-K off so that u is the only scratch.  Nothing in u has
@@ -757,7 +760,10 @@ int32_t launch_projection_tc_static(essa_ctx* ctx, const essa_adapter* a, const 
   const int bi = pl.block_n == 64 ? 0 : pl.block_n == 128 ? 1 : 2;
   CUtensorMap tm_wdeq;
   if (int8) {
-    st = launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr), (size_t)a->d_out * a->d_in, stream);
+    st = a->w0_dtype == ESSA_W0_INT8_PERCHANNEL
+             ? launch_widen_int8(ctx, a->W0q, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr), (size_t)a->d_out * a->d_in, stream)
+             : launch_widen_int4(ctx, reinterpret_cast<const uint8_t*>(a->W0q), a->w0_gscale, static_cast<__nv_bfloat16*>(ctx->w_deq.ptr),
+                                 a->d_out, a->d_in, stream);
     if (st != ESSA_OK) return st;
     st = make_tensor_map_2d(ctx, &tm_wdeq, 0, ctx->w_deq.ptr, (uint64_t)a->d_out, (uint64_t)a->d_in, (uint64_t)a->d_in * 2,
                             (uint32_t)pl.block_n, BLOCK_K, 128);

@@ -61,7 +61,7 @@ class WorkloadConfig:
     P: int
     seg_kind: str  # "fixed" | "uniform" | "mixed"
     seg_len: int  # fixed length, or the upper end of U{1..seg_len}
-    w0_dtype: str  # "bf16" | "int8"
+    w0_dtype: str  # "bf16" | "int8" | "int4"
     step: float
     full_B: bool
     random_D: bool
@@ -94,6 +94,9 @@ CONFIGS: Dict[str, WorkloadConfig] = {
     "5a": WorkloadConfig(5, "qwen2.5-72b-int8-decode-r64-P128x1", _qkvo(8192, 1024), 64, 128, "fixed", 1, "int8", 0.05, False, False, 5),
     "5b": WorkloadConfig(5, "qwen2.5-72b-int8-prefill-r64-P128x256", _qkvo(8192, 1024), 64, 128, "fixed", 256, "int8", 0.05, False, False, 5),
     "5c": WorkloadConfig(5, "qwen2.5-72b-int8-mixed-r64-P128", _qkvo(8192, 1024), 64, 128, "mixed", 256, "int8", 0.05, False, False, 5),
+    # the 72B-shaped block with INT4 group-wise weights (the paper's 72B runs are INT4, one candidate per GPU)
+    "6a": WorkloadConfig(6, "qwen2.5-72b-int4-decode-r64-P128x1", _qkvo(8192, 1024), 64, 128, "fixed", 1, "int4", 0.05, False, False, 6),
+    "6b": WorkloadConfig(6, "qwen2.5-72b-int4-prefill-r64-P128x256", _qkvo(8192, 1024), 64, 128, "fixed", 256, "int4", 0.05, False, False, 6),
 }
 
 
@@ -129,8 +132,8 @@ class Adapter:
     rank: int
     w0_dtype: str
     W0: Optional[np.ndarray]  # [d_out, d_in] float32 (bf16-exact) when w0_dtype == "bf16"
-    W0_q: Optional[np.ndarray]  # [d_out, d_in] int8 when w0_dtype == "int8"
-    W0_scale: Optional[np.ndarray]  # [d_out] float16 when w0_dtype == "int8"
+    W0_q: Optional[np.ndarray]  # [d_out, d_in] int8 when w0_dtype == "int8"; [d_out, d_in/2] uint8 (two codes per byte) for "int4"
+    W0_scale: Optional[np.ndarray]  # [d_out] float16 for "int8"; [d_out, d_in/128] float16 for "int4"
     U_A: np.ndarray  # [r, r]
     V_A: np.ndarray  # [d_in, r]
     U_B: np.ndarray  # [d_out, r]
@@ -154,6 +157,26 @@ def quantize_int8_per_channel(W: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     return q, scale
 
 
+INT4_GROUP = 128
+
+
+def quantize_int4_groupwise(W: np.ndarray, group: int = INT4_GROUP) -> Tuple[np.ndarray, np.ndarray]:
+    """Symmetric group-wise INT4 storage of a float weight: (packed uint8 [m, n/2], scale fp16 [m, n/group]).
+
+    scale[o,g] = max |W[o, g*group:(g+1)*group]| / 7 rounded to fp16; q = clip(rint(W / scale), -7, 7); byte j of a row
+    packs the codes of features 2j (low nibble) and 2j+1 (high nibble) as 4-bit two's complement.  As with INT8 this is
+    how the synthetic checkpoint is *produced*; both sides consume the stored (packed, scale) pair."""
+    W = np.asarray(W, dtype=np.float32)
+    m, n = W.shape
+    g = W.reshape(m, n // group, group)
+    amax = np.maximum(np.abs(g).max(axis=2), 1e-12)
+    scale = (amax / 7.0).astype(np.float16)
+    q = np.clip(np.rint(g / scale.astype(np.float32)[:, :, None]), -7, 7).astype(np.int8).reshape(m, n)
+    u = (q.astype(np.int16) & 0x0F).astype(np.uint8)
+    packed = (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+    return np.ascontiguousarray(packed), np.ascontiguousarray(scale)
+
+
 def make_adapter(cfg: WorkloadConfig, proj_idx: int) -> Adapter:
     name, n, m = cfg.projections[proj_idx]
     r = cfg.rank
@@ -162,6 +185,8 @@ def make_adapter(cfg: WorkloadConfig, proj_idx: int) -> Adapter:
     W0 = W0_q = W0_scale = None
     if cfg.w0_dtype == "bf16":
         W0 = round_to_bf16(w)
+    elif cfg.w0_dtype == "int4":
+        W0_q, W0_scale = quantize_int4_groupwise(w)
     else:
         W0_q, W0_scale = quantize_int8_per_channel(w)
     del w

@@ -22,7 +22,11 @@ def sigma_error(got: np.ndarray, want: np.ndarray) -> float:
 
 
 def oracle_weight(ad: wl.Adapter) -> np.ndarray:
-    return ad.W0.astype(np.float64) if ad.w0_dtype == "bf16" else orc.dequantize_int8(ad.W0_q, ad.W0_scale)
+    if ad.w0_dtype == "bf16":
+        return ad.W0.astype(np.float64)
+    if ad.w0_dtype == "int4":
+        return orc.dequantize_int4(ad.W0_q, ad.W0_scale)
+    return orc.dequantize_int8(ad.W0_q, ad.W0_scale)
 
 
 def oracle_sigma_fp32(cma: wl.CmaState, P: int) -> np.ndarray:

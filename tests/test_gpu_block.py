@@ -39,7 +39,7 @@ def _block(torch, ctx, case, candidates=None):
     ys = ctx.apply_block([case.handles[i] for i in range(n)], xs, case.d_offsets, case.d_sigma, cols)
     torch.cuda.synchronize()
     launches = ctx.gpu_launches - launches0
-    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    tol = TOL_BF16 if cfg.w0_dtype == "bf16" else TOL_INT8
     for i in range(n):
         got = ys[i].float().cpu().numpy()
         want = case.oracle_projection(i, xs_host[i], candidates)
@@ -51,6 +51,7 @@ def _block(torch, ctx, case, candidates=None):
 
 @pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 1024, 192, 16, 256, 1),      # decode block, bf16: one launch
                                                ("5a", 1024, 256, 64, 128, 1),     # decode block, INT8, rank 64
+                                               ("6a", 1024, 256, 64, 128, 1),     # decode block, INT4 group-wise
                                                ("4", 512, 128, 32, 9, 20),        # ragged segments, T = sum L_k <= 180
                                                ("2", 256, 64, 16, 3, 100)])       # T = 300: prefill sizes, one call each
 def test_block_matches_oracle(torch, ctx, base, dm, dkv, r, P, L):

@@ -35,9 +35,10 @@ def _run(torch, ctx, case, i, offsets, T, tol):
     ad, h = case.adapters[i], case.handles[i]
     sA, sB = cfg.sigma_cols(i)
     offsets = np.asarray(offsets, dtype=np.int32)
-    plan = binding.plan_projection(ad.d_in, ad.d_out, ad.rank,
-                                   binding.ESSA_W0_INT8_PERCHANNEL if ad.w0_dtype == "int8" else binding.ESSA_W0_BF16, T)
-    assert plan["decode"] == 1
+    dtype = {"bf16": binding.ESSA_W0_BF16, "int8": binding.ESSA_W0_INT8_PERCHANNEL, "int4": binding.ESSA_W0_INT4_GROUP128}[ad.w0_dtype]
+    plan = binding.plan_projection(ad.d_in, ad.d_out, ad.rank, dtype, T)
+    # INT4 storage has the tensor-memory decode mode only (at most 128 tokens); larger calls take the prefill kernels
+    assert plan["decode"] == (0 if ad.w0_dtype == "int4" and T > 128 else 1)
     x = wl.make_tokens(cfg, i, T)
     want = orc.apply_projection(oracle_weight(ad), ad.U_A, ad.V_A, ad.U_B, ad.V_B, x, offsets, case.sigma32, sA, sB, ad.rank)
     y = ctx.apply_projection(h, to_dev(torch, x, torch.bfloat16), to_dev(torch, offsets), case.d_sigma, sA, sB)
@@ -66,12 +67,12 @@ def test_token_counts(torch, ctx, T):
 
 
 @pytest.mark.parametrize("rank", [1, 3, 8, 17, 33, 48, 64])
-@pytest.mark.parametrize("w0", ["bf16", "int8"])
+@pytest.mark.parametrize("w0", ["bf16", "int8", "int4"])
 def test_ranks_and_storage(torch, ctx, rank, w0):
-    cfg = wl.scaled_config("5a" if w0 == "int8" else "3", d_model=512, d_kv=200, rank=rank, P=7, seg_len=1)
+    cfg = wl.scaled_config({"int8": "5a", "int4": "6a", "bf16": "3"}[w0], d_model=512, d_kv=200, rank=rank, P=7, seg_len=1)
     case = Case(torch, ctx, cfg)
     rng = np.random.default_rng(rank)
-    tol = TOL_INT8 if w0 == "int8" else TOL_BF16
+    tol = TOL_BF16 if w0 == "bf16" else TOL_INT8
     for i, T in ((0, 77), (1, 192)):
         _run(torch, ctx, case, i, _offsets(rng, cfg.P, T), T, tol)
     case.close()
@@ -113,4 +114,17 @@ def test_zero_sigma_gives_base_projection(torch, ctx):
                              torch.zeros_like(case.d_sigma), sA, sB).float().cpu().numpy()
     base = x.astype(np.float64) @ oracle_weight(case.adapters[0]).T
     assert orc.relative_error(y, base) <= 6e-3  # only the final bf16 rounding
+    case.close()
+
+
+@pytest.mark.parametrize("w0", ["int8", "int4"])
+@pytest.mark.parametrize("T", [1, 16, 33, 100, 128])
+def test_quantised_storage_token_counts_in_tensor_memory_mode(torch, ctx, w0, T):
+    """At most 128 tokens: the codes are converted straight into tensor memory (INT8 and INT4 storage alike); several
+    row tiles, a ragged last row tile (d_kv = 200), more K blocks than ring slots, ragged and empty segments."""
+    cfg = wl.scaled_config("5a" if w0 == "int8" else "6a", d_model=1280, d_kv=200, rank=24, P=6, seg_len=1)
+    case = Case(torch, ctx, cfg)
+    rng = np.random.default_rng(7 * T)
+    for i in (0, 1):
+        y, _ = _run(torch, ctx, case, i, _offsets(rng, cfg.P, T), T, TOL_INT8)
     case.close()

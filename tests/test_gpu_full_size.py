@@ -15,7 +15,7 @@ from tests.parity_utils import TOL_BF16, TOL_INT8, Case
 
 pytestmark = pytest.mark.gpu
 
-MAX_ORACLE_CANDIDATES = {"2": 6, "3": 24, "4": 6, "5a": 12, "5b": 5}
+MAX_ORACLE_CANDIDATES = {"2": 6, "3": 24, "4": 6, "5a": 12, "5b": 5, "6a": 12, "6b": 4}
 
 
 @pytest.fixture(scope="module")
@@ -35,11 +35,11 @@ def ctx(torch):
     c.close()
 
 
-@pytest.mark.parametrize("name", ["2", "3", "4", "5a", "5b"])
+@pytest.mark.parametrize("name", ["2", "3", "4", "5a", "5b", "6a", "6b"])
 def test_full_size_config(torch, ctx, name):
     cfg = wl.CONFIGS[name]
     case = Case(torch, ctx, cfg)
-    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    tol = TOL_BF16 if cfg.w0_dtype == "bf16" else TOL_INT8
     cands = wl.stratified_candidates(cfg, case.offsets)[:MAX_ORACLE_CANDIDATES[name]]
     assert case.T == int(case.offsets[-1]) and len(cands) >= 2
     for i in range(len(cfg.projections)):

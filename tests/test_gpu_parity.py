@@ -176,6 +176,9 @@ SCALED = {
     "int8-decode-r64": ("5a", 1024, 256, 64, 128, 1),
     "int8-prefill-r64": ("5b", 768, 128, 64, 16, 100),
     "int8-mixed-r64": ("5c", 512, 128, 64, 32, 90),
+    "int4-decode-r64": ("6a", 1024, 256, 64, 128, 1),     # INT4 group-wise storage, tensor-memory decode mode
+    "int4-prefill-r64": ("6b", 768, 128, 64, 16, 100),    # ... dequantised per call for the prefill kernels
+    "int4-decode-256": ("6a", 512, 128, 32, 200, 1),      # 200 tokens: above the decode mode's limit, prefill kernels
 }
 
 
@@ -184,7 +187,7 @@ def test_scaled_configs_full_outputs(torch, ctx, name):
     base, dm, dkv, r, P, L = SCALED[name]
     cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
     case = Case(torch, ctx, cfg)
-    tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
+    tol = TOL_BF16 if cfg.w0_dtype == "bf16" else TOL_INT8
     for i in range(len(cfg.projections)):
         _check_projection(case, i, tol)
     case.close()

@@ -379,3 +379,44 @@ def test_reconstructed_factors_round_trip_the_svd():
         for c in range(n):
             A4[i, c] = sum(UA[i, j] * SA[j] * VAt[j, c] for j in range(r))
     assert np.allclose(A4, A2, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------- INT4 storage
+def test_int4_dequant_scalar_loops_and_nibble_table():
+    rng = np.random.default_rng(41)
+    m, n, group = 5, 256, 128
+    packed = rng.integers(0, 256, size=(m, n // 2), dtype=np.uint8)
+    scale = rng.uniform(0.01, 0.2, size=(m, n // group)).astype(np.float16)
+    got = orc.dequantize_int4(packed, scale, group)
+    table = [0, 1, 2, 3, 4, 5, 6, 7, -8, -7, -6, -5, -4, -3, -2, -1]  # 4-bit two's complement, written out
+    for o in range(m):
+        for i in range(n):
+            byte = int(packed[o, i // 2])
+            nib = (byte >> 4) if (i & 1) else (byte & 15)
+            assert got[o, i] == table[nib] * float(scale[o, i // group])
+
+
+def test_int4_agrees_with_int8_when_codes_fit_and_groups_share_a_scale():
+    rng = np.random.default_rng(42)
+    m, n = 6, 384
+    q = rng.integers(-8, 8, size=(m, n)).astype(np.int8)
+    row_scale = rng.uniform(0.01, 0.1, size=m).astype(np.float16)
+    u = (q.astype(np.int16) & 15).astype(np.uint8)
+    packed = (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+    w4 = orc.dequantize_int4(packed, np.repeat(row_scale[:, None], n // 128, axis=1))
+    w8 = orc.dequantize_int8(q, row_scale)
+    assert np.array_equal(w4, w8)
+
+
+def test_int4_workload_quantiser_round_trip_error_bound():
+    """The generator's codes stay in [-7, 7] and the stored pair reproduces the weight to half a step per entry."""
+    rng = np.random.default_rng(43)
+    W = (rng.standard_normal((8, 512)) / np.sqrt(512)).astype(np.float32)
+    from paper_2507_04453_b200 import workloads as wl
+    packed, scale = wl.quantize_int4_groupwise(W)
+    assert packed.shape == (8, 256) and scale.shape == (8, 4) and scale.dtype == np.float16
+    deq = orc.dequantize_int4(packed, scale)
+    step = np.repeat(scale.astype(np.float64), 128, axis=1)
+    # half a step, plus the clip at +-7 when the fp16 rounding made the scale a little smaller than max / 7
+    assert np.all(np.abs(deq - W) <= (0.5 + 7 * 2.0 ** -11) * step + 1e-12)
+    assert np.max(np.abs(deq / step)) <= 7
