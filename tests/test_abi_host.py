@@ -61,14 +61,14 @@ def test_validate_segments(lib):
         assert binding.validate_segments(off, int(off[-1])) == ok
 
 
-@pytest.mark.parametrize("name", ["1", "2", "3", "4", "5a", "5b", "5c"])
+@pytest.mark.parametrize("name", ["1", "2", "3", "4", "5a", "5b", "5c", "6a", "6b"])
 def test_plan_is_consistent(lib, name):
     cfg = wl.CONFIGS[name]
     T = int(wl.make_segments(cfg)[-1])
-    dtype = binding.ESSA_W0_INT8_PERCHANNEL if cfg.w0_dtype == "int8" else binding.ESSA_W0_BF16
+    dtype = {"bf16": binding.ESSA_W0_BF16, "int8": binding.ESSA_W0_INT8_PERCHANNEL, "int4": binding.ESSA_W0_INT4_GROUP128}[cfg.w0_dtype]
     for _, n, m in cfg.projections:
         p = binding.plan_projection(n, m, cfg.rank, dtype, T, 148)
-        ext = 2 if dtype else 1
+        ext = 2 if dtype == binding.ESSA_W0_INT8_PERCHANNEL else 1
         assert p["k_blocks"] == n // 64 + ext
         if T <= 256:
             # decode schedule: 128 W0 rows per CTA, all tokens in one tile, reduction split over a cluster
@@ -76,10 +76,12 @@ def test_plan_is_consistent(lib, name):
             assert p["block_n"] == -(-T // 16) * 16 and p["tiles"] == -(-m // 128)
             assert p["splits"] in (1, 2, 4, 8) and p["splits"] <= n // 64 and p["grid"] <= {1: 148, 2: 148, 4: 132, 8: 120}[p["splits"]]
             assert p["grid"] == p["tiles"] * p["splits"] and p["scratch_bytes"] == 0
-            # bf16 storage: 16 KB W0 tiles; INT8 storage: 8 KB tiles of codes plus four converted tiles
-            # ... and two 8 KB tiles of V_A^T for the down-projection slices
-            rings = (2 * 64 * 128 + p["stages"] * (64 * 128 if dtype else 128 * 128) + (4 * 128 * 128 if dtype else 0)
-                     + p["x_stages"] * p["block_n"] * 128)
+            # bf16 storage: 16 KB W0 tiles.  Quantised storage: 8 KB (INT8) or 4 KB (INT4) tiles of codes; at most 128
+            # tokens the converted tiles live in tensor memory and two 16 KB slots hold the U_B slabs, above that
+            # (INT8 only) four converted tiles sit in shared memory.  Two 8 KB tiles of V_A^T in every mode.
+            w_slot = {binding.ESSA_W0_BF16: 128 * 128, binding.ESSA_W0_INT8_PERCHANNEL: 64 * 128, binding.ESSA_W0_INT4_GROUP128: 32 * 128}[dtype]
+            slots16k = 0 if dtype == binding.ESSA_W0_BF16 else 2 if p["block_n"] <= 128 else 4
+            rings = 2 * 64 * 128 + p["stages"] * w_slot + slots16k * 128 * 128 + p["x_stages"] * p["block_n"] * 128
             assert 1 <= p["stages"] <= 16 and 1 <= p["x_stages"] <= 6
             assert 1024 + rings + 8192 <= 227 * 1024
             per = -(-(-(-p["block_n"] // p["splits"])) // 16) * 16
