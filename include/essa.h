@@ -92,6 +92,15 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   ESSA_OPT_PAIR_TILES defaults to 1. */
 #define ESSA_OPT_PAIR_TILES 1
 #define ESSA_OPT_FUSE_DOWN 2
+/*   ESSA_OPT_WAIT_LIMIT_MCYCLES (1 .. 100000, default 3000): how long, in millions of SM cycles, the decode kernel's
+ *   waits on counters that other thread blocks advance may last before the kernel gives up and records
+ *   ESSA_ERR_DEVICE_TIMEOUT (the waits on its own copies and MMAs keep their fixed limit and end at once when a
+ *   thread of the block has given up).
+ *   ESSA_OPT_DEBUG_STALL_RANK_ROWS (0 / 1; for testing the give-up path without a fault): while set, a decode launch
+ *   waits for one more row of the rank-path vector than the call publishes, so its up-projection never becomes
+ *   ready, the wait runs out, the output is undefined and essa_get_status reports ESSA_ERR_DEVICE_TIMEOUT. */
+#define ESSA_OPT_WAIT_LIMIT_MCYCLES 3
+#define ESSA_OPT_DEBUG_STALL_RANK_ROWS 4
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);
@@ -246,6 +255,19 @@ typedef struct essa_block_item {
 } essa_block_item;
 int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T,
                          const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma, void* stream);
+
+/* The blocks of several layers in one call ("Slice n" of Figure 1: the table holds one contiguous slice of singular
+ * values per LoRA matrix of every layer; the appendix's bookkeeping counts layers x 4 matrices x 2 r coordinates).
+ * items holds n_layers x n_items entries, layer-major: items[l * n_items + i] is projection i of layer l with its own
+ * adapter, activations x, output y and table columns; tokens, segments and the table are shared by all of them.  The
+ * result is what n_layers calls of essa_apply_block give.  Every layer's activations are the caller's (whatever runs
+ * between the projections of consecutive layers is outside this library), so they must all be final when the call is
+ * made.  At decode sizes (T <= 256) each layer is one launch and the launches are chained WITHOUT waiting for one
+ * another: a layer's thread blocks start wherever the layer before has released an SM, so launch gaps and the tail of
+ * one layer overlap the weight streaming of the next; the launches still complete in order.  Larger calls, and layers
+ * that do not fit the one-launch schedule, are issued like essa_apply_block. */
+int32_t essa_apply_layers(essa_ctx* ctx, const essa_block_item* items, int32_t n_layers, int32_t n_items, int64_t T,
+                          const int32_t* seg_offsets, int32_t P, const float* sigma, int32_t ld_sigma, void* stream);
 
 /* Population draw and block projections in one call (Algorithm 1, lines 5 and 7, for the candidates this worker
  * evaluates): exactly essa_sample_population_range(mean, step, Bfactor, Dvec, d, seed, k_begin, P, sigma_out)

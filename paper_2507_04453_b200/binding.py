@@ -28,6 +28,8 @@ ESSA_W0_INT8_PERCHANNEL = 1
 ESSA_W0_INT4_GROUP128 = 2
 ESSA_OPT_PAIR_TILES = 1
 ESSA_OPT_FUSE_DOWN = 2
+ESSA_OPT_WAIT_LIMIT_MCYCLES = 3
+ESSA_OPT_DEBUG_STALL_RANK_ROWS = 4
 
 EXPORTED_SYMBOLS = (
     "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",
@@ -37,7 +39,7 @@ EXPORTED_SYMBOLS = (
     "essa_debug_philox", "essa_debug_segment_map", "essa_debug_core_matrix", "essa_profile_begin", "essa_profile_end",
     "essa_apply_projection_static", "essa_get_launch_count", "essa_reserve_dequant", "essa_apply_block", "essa_apply_block_host", "essa_set_option",
     "essa_top_alpha_index", "essa_sample_population_masked", "essa_export_candidates", "essa_sample_apply_block",
-    "essa_cma_create", "essa_cma_destroy", "essa_cma_ask", "essa_tell", "essa_cma_set", "essa_cma_get", "essa_cma_params",
+    "essa_apply_layers", "essa_cma_create", "essa_cma_destroy", "essa_cma_ask", "essa_tell", "essa_cma_set", "essa_cma_get", "essa_cma_params",
 )
 
 
@@ -113,6 +115,7 @@ def load_library() -> C.CDLL:
         "essa_set_option": (i32, [vp, i32, i32]),
         "essa_apply_block": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
         "essa_apply_block_host": (i32, [vp, C.POINTER(BlockItem), i32, i64, vp, i32, vp, i32, vp]),
+        "essa_apply_layers": (i32, [vp, C.POINTER(BlockItem), i32, i32, i64, vp, i32, vp, i32, vp]),
         "essa_sample_apply_block": (i32, [vp, vp, f32, vp, vp, i32, u64, i32, i32, vp, C.POINTER(BlockItem), i32, i64, vp, vp]),
         "essa_cma_create": (i32, [vp, i32, i32, vp, f32, C.POINTER(vp)]),
         "essa_cma_destroy": (i32, [vp, vp]),
@@ -205,6 +208,30 @@ class PreparedBlock:
 
     def run(self, stream_handle):
         """stream_handle: the integer cudaStream_t (torch's ``stream.cuda_stream``; 0 / None = default stream)."""
+        st = self.fn(*self.args, stream_handle or None)
+        if st != ESSA_OK:
+            self.ctx._check(st)
+
+
+class PreparedLayers:
+    """essa_apply_layers with its arguments marshalled ahead of time (see Context.prepare_layers)."""
+
+    def __init__(self, ctx, layers, seg_offsets, sigma):
+        n_layers, n_items = len(layers), len(layers[0])
+        T = layers[0][0][1].shape[0]
+        self.keep = (layers, seg_offsets, sigma)
+        self.arr = (BlockItem * (n_layers * n_items))()
+        for l, layer in enumerate(layers):
+            assert len(layer) == n_items
+            for i, (ad, x, cols, y) in enumerate(layer):
+                self.arr[l * n_items + i] = BlockItem(ad.handle, x.data_ptr() if T else None, cols[0], cols[1],
+                                                      y.data_ptr() if T else None)
+        self.ctx = ctx
+        self.fn = ctx.lib.essa_apply_layers
+        self.args = (ctx.handle, self.arr, n_layers, n_items, T, seg_offsets.data_ptr(), seg_offsets.numel() - 1,
+                     sigma.data_ptr(), sigma.stride(0) if sigma.dim() == 2 else sigma.numel())
+
+    def run(self, stream_handle):
         st = self.fn(*self.args, stream_handle or None)
         if st != ESSA_OK:
             self.ctx._check(st)
@@ -485,6 +512,15 @@ class Context:
         single foreign-function call (at decode sizes the Python-side marshalling of a step is otherwise comparable
         to the step's device time).  The tensors must stay alive and in place while the object is used."""
         return PreparedBlock(self, adapters, xs, seg_offsets, sigma, cols, outs)
+
+    def prepare_layers(self, layers, seg_offsets, sigma):
+        """The arguments of one essa_apply_layers call marshalled once.  layers: a list (one entry per layer) of lists
+        of (adapter, x, (sA_col, sB_col), y) tuples; ``run(stream)`` issues the call."""
+        return PreparedLayers(self, layers, seg_offsets, sigma)
+
+    def apply_layers(self, layers, seg_offsets, sigma, stream=None):
+        """essa_apply_layers: the blocks of several layers in one call (see prepare_layers for the argument layout)."""
+        PreparedLayers(self, layers, seg_offsets, sigma).run(_stream(stream))
 
     def prepare_sample_block(self, mean, step: float, Bfactor, Dvec, seed: int, P: int, sigma_out, adapters, xs, seg_offsets,
                              cols, outs, k_begin: int = 0):

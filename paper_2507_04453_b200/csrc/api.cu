@@ -160,15 +160,20 @@ int32_t essa_create(essa_ctx** out, int32_t device) {
   else
     cudaGetLastError();
   if (cudaMalloc(&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_u, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
-      cudaMemset(ctx->dec_u, 0, (size_t)ESSA_MAX_BLOCK_ITEMS * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_cnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
-      cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_ppart, (size_t)ESSA_MAX_BLOCK_ITEMS * 32 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
-      cudaMalloc(&ctx->dec_pcnt, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
-      cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_u, (size_t)kDecSlots * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMemset(ctx->dec_u, 0, (size_t)kDecSlots * kDecodeMaxTokens * kRankPadMax * 2) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_cnt, kDecSlots * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->dec_cnt, 0, kDecSlots * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_ppart, (size_t)kDecSlots * 32 * kDecodeMaxTokens * kRankPadMax * 4) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_pcnt, kDecSlots * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->dec_pcnt, 0, kDecSlots * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->dec_set_done, kDecSets * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->dec_set_done, 0, kDecSets * sizeof(uint32_t)) != cudaSuccess ||
+      cudaMalloc(&ctx->layers_flag, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->layers_flag, 0, sizeof(uint32_t)) != cudaSuccess ||
       cudaMalloc(&ctx->samp_cnt, sizeof(uint32_t)) != cudaSuccess || cudaMemset(ctx->samp_cnt, 0, sizeof(uint32_t)) != cudaSuccess) {
     if (ctx->samp_cnt) cudaFree(ctx->samp_cnt);
+    if (ctx->layers_flag) cudaFree(ctx->layers_flag);
+    if (ctx->dec_set_done) cudaFree(ctx->dec_set_done);
     if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
     if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -207,6 +212,8 @@ int32_t essa_destroy(essa_ctx* ctx) {
   if (ctx->dec_ppart) cudaFree(ctx->dec_ppart);
   if (ctx->dec_pcnt) cudaFree(ctx->dec_pcnt);
   if (ctx->samp_cnt) cudaFree(ctx->samp_cnt);
+  if (ctx->layers_flag) cudaFree(ctx->layers_flag);
+  if (ctx->dec_set_done) cudaFree(ctx->dec_set_done);
   delete ctx;
   return ESSA_OK;
 }
@@ -224,8 +231,12 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status) {
     cudaMemset(ctx->d_status, 0, sizeof(int32_t));
     if (ctx->splitk_ws.ptr) cudaMemset(ctx->splitk_ws.ptr, 0, ctx->splitk_ws.bytes);
     if (ctx->splitk_cnt.ptr) cudaMemset(ctx->splitk_cnt.ptr, 0, ctx->splitk_cnt.bytes);
-    cudaMemset(ctx->dec_cnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
-    cudaMemset(ctx->dec_pcnt, 0, ESSA_MAX_BLOCK_ITEMS * sizeof(uint32_t));
+    cudaMemset(ctx->dec_cnt, 0, kDecSlots * sizeof(uint32_t));
+    cudaMemset(ctx->dec_pcnt, 0, kDecSlots * sizeof(uint32_t));
+    cudaMemset(ctx->layers_flag, 0, sizeof(uint32_t));
+    cudaMemset(ctx->dec_set_done, 0, kDecSets * sizeof(uint32_t));
+    for (uint32_t& e : ctx->dec_set_issued) e = 0;
+    ctx->layers_epoch = 0;
     for (uint32_t& e : ctx->dec_epoch) e = 0;
     for (uint32_t& e : ctx->dec_pepoch) e = 0;
     cudaMemset(ctx->samp_cnt, 0, sizeof(uint32_t));
@@ -244,6 +255,11 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
       if (value < 0 || value > 2) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_FUSE_DOWN takes 0, 1 or 2");
       ctx->fuse_down = value;
       return ESSA_OK;
+    case ESSA_OPT_WAIT_LIMIT_MCYCLES:
+      if (value < 1 || value > 100000) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_WAIT_LIMIT_MCYCLES takes 1 .. 100000");
+      ctx->wait_limit_mcycles = value;
+      return ESSA_OK;
+    case ESSA_OPT_DEBUG_STALL_RANK_ROWS: ctx->debug_stall_rank_rows = value != 0; return ESSA_OK;
     default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
   }
 }
@@ -491,6 +507,42 @@ static int32_t apply_block_impl(essa_ctx* ctx, const essa_block_item* items, int
 int32_t essa_apply_block(essa_ctx* ctx, const essa_block_item* items, int32_t n_items, int64_t T, const int32_t* seg,
                          int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v) {
   return apply_block_impl(ctx, items, n_items, T, seg, P, sigma, ld_sigma, stream_v, nullptr, 0);
+}
+
+int32_t essa_apply_layers(essa_ctx* ctx, const essa_block_item* items, int32_t n_layers, int32_t n_items, int64_t T,
+                          const int32_t* seg, int32_t P, const float* sigma, int32_t ld_sigma, void* stream_v) {
+  if (!ctx) return ESSA_ERR_INVALID_ARG;
+  if (!items || n_layers < 1 || n_items < 1 || n_items > ESSA_MAX_BLOCK_ITEMS)
+    return fail(ctx, ESSA_ERR_INVALID_ARG, "apply_layers: need n_layers >= 1 and 1 .. ESSA_MAX_BLOCK_ITEMS items per layer");
+  for (int64_t j = 0; j < (int64_t)n_layers * n_items; ++j) {
+    const int32_t st = validate_projection_args(ctx, items[j].adapter, items[j].x, T, seg, P, sigma, ld_sigma, items[j].sA_col,
+                                                items[j].sB_col, items[j].y);
+    if (st != ESSA_OK) return st;
+  }
+  if (T == 0) return ESSA_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  order_stream(ctx, stream);
+  // Decode sizes: one launch per layer; consecutive launches alternate between the context's two scratch sets and do
+  // not wait for one another, so a layer's CTAs start wherever the layer before has freed an SM.  A layer that does
+  // not fit the one-launch schedule (and every layer of a larger call) is issued like essa_apply_block.
+  bool chain = T <= kDecodeMaxTokens && n_layers > 1;
+  if (chain) ctx->layers_epoch += 1;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    const essa_block_item* it = items + (size_t)l * n_items;
+    int32_t st = kBlockNotFused;
+    if (T <= kDecodeMaxTokens) {
+      BlockItem bi[ESSA_MAX_BLOCK_ITEMS];
+      for (int32_t i = 0; i < n_items; ++i)
+        bi[i] = BlockItem{it[i].adapter, static_cast<const __nv_bfloat16*>(it[i].x), it[i].sA_col, it[i].sB_col,
+                          static_cast<__nv_bfloat16*>(it[i].y)};
+      st = launch_block_decode(ctx, bi, n_items, T, seg, P, sigma, ld_sigma, stream, nullptr, 0, l & 1,
+                               !chain ? 0 : l == 0 ? 1 : 2);
+      if (st == kBlockNotFused && l == 0) chain = false;  // nobody would publish the flag the later layers wait for
+    }
+    if (st == kBlockNotFused) st = apply_block_impl(ctx, it, n_items, T, seg, P, sigma, ld_sigma, stream_v, nullptr, 0);
+    if (st != ESSA_OK) return st;
+  }
+  return ESSA_OK;
 }
 
 int32_t essa_sample_apply_block(essa_ctx* ctx, const float* mean, float step, const float* Bfactor, const float* Dvec, int32_t d,

@@ -15,6 +15,8 @@
 namespace essa {
 
 constexpr int kRankPadMax = 64;
+constexpr int kDecSets = 2;  // decode scratch sets: consecutive blocks of a multi-layer call alternate between them
+constexpr int kDecSlots = kDecSets * ESSA_MAX_BLOCK_ITEMS;
 constexpr int kDecodeMaxTokens = 256;  // calls with at most this many tokens use the decode schedule (proj_decode.cu)  // rank-path operands are stored 64 columns wide (one 128-byte swizzle row)
 
 // Device status word values are the ESSA_ERR_* codes; 0 = nothing recorded.
@@ -31,6 +33,8 @@ struct essa_ctx {
   std::string last_error;
   int32_t* d_status = nullptr;  // device status word
   int64_t launches = 0;         // kernels of this library enqueued through this context
+  int wait_limit_mcycles = 3000;  // ESSA_OPT_WAIT_LIMIT_MCYCLES
+  bool debug_stall_rank_rows = false;  // ESSA_OPT_DEBUG_STALL_RANK_ROWS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
   int fuse_down = 0;            // ... which also compute the down-projection (no rank-down launch): 0 never (default),
                                 // 1 in the token range where it measured faster, 2 whenever pair tiles are used
@@ -40,10 +44,14 @@ struct essa_ctx {
   // published so far (monotonic across calls; dec_epoch is the host's copy of where the next call starts)
   void* dec_u = nullptr;
   uint32_t* dec_cnt = nullptr;
-  uint32_t dec_epoch[ESSA_MAX_BLOCK_ITEMS] = {};  // (one buffer / counter set per projection of a block launch)
+  uint32_t dec_epoch[essa::kDecSlots] = {};  // (one buffer / counter set per scratch set and projection of a block launch)
   void* dec_ppart = nullptr;    // [32][kDecodeMaxTokens][64] fp32 per projection: per-slice partial down-projections
   uint32_t* dec_pcnt = nullptr; // slices delivered so far, per projection (monotonic; dec_pepoch is the host's copy)
-  uint32_t dec_pepoch[ESSA_MAX_BLOCK_ITEMS] = {};
+  uint32_t dec_pepoch[essa::kDecSlots] = {};
+  uint32_t* dec_set_done = nullptr;  // [kDecSets] CTAs of decode launches on each scratch set that have finished (monotonic)
+  uint32_t dec_set_issued[essa::kDecSets] = {};  // ... and how many have been launched (host count)
+  uint32_t* layers_flag = nullptr;  // multi-layer calls: epoch of the latest call whose first block has seen its inputs complete
+  uint32_t layers_epoch = 0;
   uint32_t* samp_cnt = nullptr; // blocks of fused population draws finished so far (monotonic; samp_epoch is the host's copy)
   uint32_t samp_epoch = 0;
   // Scratch owned by the context (grown on demand, never shrunk).
@@ -67,8 +75,8 @@ struct essa_ctx {
   struct XMapEntry { const void* ptr = nullptr; int64_t T = 0; int32_t d_in = 0; uint32_t box = 0; CUtensorMap tm; };
   XMapEntry xmap_cache[16];
   int xmap_next = 0;
-  CUtensorMap dec_u_map[ESSA_MAX_BLOCK_ITEMS][2];   // maps of the decode u buffers for 64-row boxes / one box of tn rows
-  uint32_t dec_u_map_box[ESSA_MAX_BLOCK_ITEMS][2] = {};
+  CUtensorMap dec_u_map[essa::kDecSlots];           // maps of the decode u buffers (one box of tn rows)
+  uint32_t dec_u_map_box[essa::kDecSlots] = {};
   // essa_profile_begin/end: three events per recorded call
   bool prof_on = false;
   int prof_calls = 0, prof_dropped = 0;
@@ -177,9 +185,13 @@ constexpr int32_t kBlockNotFused = 1;  // launch_block_decode: the block does no
 // sigma_ready != NULL: the table is being written by the kernel launched just before on the same stream, which
 // counts its finished blocks in *sigma_ready; the launch does not wait for that kernel as a whole, only (bounded)
 // for the count to reach sigma_target before it reads the table.
+// set: which of the context's decode scratch sets the launch uses.  layer_mode: 0 = a call of its own; 1 = first block
+// of a multi-layer call (after its own wait for earlier work it publishes layers_epoch in the context's flag);
+// 2 = later block of a multi-layer call (does not wait for the block before it, which it overlaps; waits, bounded,
+// for that flag before it touches the activations and the table).
 int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
                             const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready = nullptr,
-                            uint32_t sigma_target = 0);
+                            uint32_t sigma_target = 0, int set = 0, int layer_mode = 0);
 bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out);
 int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, const essa_plan& plan,
                                  cudaStream_t stream);

@@ -116,6 +116,22 @@ struct DBlock {
   // draw as a whole (it streams W0 and x beside it) and only the rank path waits for the count (bounded).
   const uint32_t* sigma_ready;
   uint32_t sigma_target;
+  // Multi-layer call: blocks of consecutive layers overlap (a CTA of the next block starts as soon as an SM is free),
+  // so a later block may not wait for the one before it.  layer_mode 1 (first block): after its own wait for earlier
+  // work it publishes layers_epoch in *layers_flag; 2 (later blocks): no wait for the previous kernel, but the
+  // activations and the table are touched only once *layers_flag has reached layers_epoch (bounded wait).
+  int layer_mode;
+  uint32_t* layers_flag;
+  uint32_t layers_epoch;
+  // Every CTA adds one to *set_done when it is through with the scratch set of its launch.  A later block of a
+  // multi-layer call starts only once the earlier launches on ITS set have finished (set_wait_target CTAs), and its
+  // CTA 0 leaves only once the launches on the OTHER set issued before it have (other_wait_target), so that the
+  // launches of a context complete in the order they were issued although they do not wait for one another.
+  long long wait_limit;  // cycles a wait on another thread block's counter may last
+  uint32_t* set_done;
+  uint32_t set_wait_target;
+  const uint32_t* other_done;
+  uint32_t other_wait_target;
   DParams proj[kMaxBlockProj];
 };
 struct DMaps {
@@ -403,7 +419,25 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // draw); x, the singular values, the scratch buffers and y are touched only after this point.  In a fused draw +
   // block call the kernel before is known to be the draw, which writes nothing but the table: no wait here, the
   // rank path waits for the table instead.
-  if (blk.sigma_ready == nullptr) grid_dep_wait();
+  grid_dep_launch();  // the next launch may start its CTAs wherever an SM is free (it waits, or not, on its own terms)
+  if (blk.sigma_ready == nullptr && blk.layer_mode != 2) grid_dep_wait();
+  if (blk.layer_mode == 1 && blockIdx.x == 0 && threadIdx.x == 0) st_release_u32(blk.layers_flag, blk.layers_epoch);
+  auto wait_count = [&](const uint32_t* counter, uint32_t target) -> bool {  // bounded; by one thread
+    const long long w0 = clock64();
+    while ((int32_t)(ld_acquire_u32(counter) - target) < 0) {
+      if (*abort_flag || clock64() - w0 > blk.wait_limit) {
+        *abort_flag = 1;
+        atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
+        return false;
+      }
+    }
+    return true;
+  };
+  auto wait_layers_flag = [&]() -> bool { return wait_count(blk.layers_flag, blk.layers_epoch); };
+  if (blk.layer_mode == 2) {  // the scratch set must be free of the launch two blocks back
+    if (threadIdx.x == 0) wait_count(blk.set_done, blk.set_wait_target);
+    __syncthreads();
+  }
 
   // ------------------------------------------------------------------ TMA producers: warp 0 streams the frozen
   // operands (the W0 ring and, during this CTA's slice, the V_A^T tiles), warp kXWarp the activations (the x ring,
@@ -444,6 +478,10 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     if (lane == 0) {
       int ix = 0;
       bool ok = true;
+      if (blk.layer_mode == 2) {  // the activations may only just have been written by the work before the call
+        ok = wait_layers_flag();
+        if (ok) fence_proxy_async_global();
+      }
       while (ok && ix < n_x) {
         if (ix >= SX) ok = mbar_wait(bar_xempty + 8 * (ix % SX), (uint32_t)(((ix / SX) & 1) ^ 1), abort_flag, p.status);
         if (ok && ix == nkb) {
@@ -451,7 +489,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
           // read after it
           const long long t0 = clock64();
           while ((int32_t)(ld_acquire_u32(p.u_count) - p.u_target) < 0) {
-            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) {
+            if (*abort_flag || clock64() - t0 > blk.wait_limit) {
               *abort_flag = 1;
               atomicCAS(p.status, 0, ESSA_ERR_DEVICE_TIMEOUT);
               ok = false;
@@ -711,7 +749,13 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     if ((int)blockIdx.x < blk.rank_ctas) {
       // this CTA's finishing units of the rank path (of any projection of the block), while its K loop streams
       bool fine = true;
-      if (blk.sigma_ready != nullptr && (int)blockIdx.x < blk.unit_begin[blk.n_proj]) {
+      if (blk.layer_mode == 2 && (int)blockIdx.x < blk.unit_begin[blk.n_proj]) {
+        if (etid == 0) *flag = wait_layers_flag() ? 1 : 0;
+        epi_bar_sync();
+        fine = *flag != 0;
+        epi_bar_sync();  // flag may be reused
+      }
+      if (fine && blk.sigma_ready != nullptr && (int)blockIdx.x < blk.unit_begin[blk.n_proj]) {
         // the table must be complete before its rows are read
         if (etid == 0) {
           int ok = 1;
@@ -794,6 +838,10 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   if (warp == 1 && is_main) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0) {
+    if (blk.layer_mode == 2 && blockIdx.x == 0) wait_count(blk.other_done, blk.other_wait_target);
+    red_release_add_u32(blk.set_done, 1u);
   }
 }
 
@@ -891,7 +939,7 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
 // issue the projections one by one.
 int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
                             const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready,
-                            uint32_t sigma_target) {
+                            uint32_t sigma_target, int set, int layer_mode) {
   if (n < 1 || n > kMaxBlockProj || T <= 0 || T > kDecodeMaxTokens) return kBlockNotFused;
   const int w0_dtype = items[0].a->w0_dtype;
   const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
@@ -958,6 +1006,15 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   blk.n_proj = n;
   blk.sigma_ready = sigma_ready;
   blk.sigma_target = sigma_target;
+  blk.layer_mode = layer_mode;
+  blk.layers_flag = ctx->layers_flag;
+  blk.layers_epoch = ctx->layers_epoch;
+  blk.wait_limit = (long long)ctx->wait_limit_mcycles * 1000000LL;
+  blk.set_done = ctx->dec_set_done + (set & 1);
+  blk.set_wait_target = ctx->dec_set_issued[set & 1];
+  blk.other_done = ctx->dec_set_done + ((set & 1) ^ 1);
+  blk.other_wait_target = ctx->dec_set_issued[(set & 1) ^ 1];
+  const int s0 = (set & 1) * kMaxBlockProj;  // first scratch slot of this launch
   blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
   int cta = 0, unit = 0;
   // The counters' next values are committed to the context only once the launch has been accepted: after a failed
@@ -999,11 +1056,11 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
         const int nkb_s = p.main_kb / splits + (sp < p.main_kb % splits ? 1 : 0);
         delivered += (nkb_s + p.p_c - 1) / p.p_c;
       }
-      p.p_count = ctx->dec_pcnt + i;
-      next_pepoch[i] = ctx->dec_pepoch[i] + (uint32_t)delivered;
+      p.p_count = ctx->dec_pcnt + s0 + i;
+      next_pepoch[i] = ctx->dec_pepoch[s0 + i] + (uint32_t)delivered;
       p.p_target = next_pepoch[i];
     }
-    p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)i * kMaxPSlices * kDecodeMaxTokens * kRankPadMax;
+    p.p_part = static_cast<float*>(ctx->dec_ppart) + (size_t)(s0 + i) * kMaxPSlices * kDecodeMaxTokens * kRankPadMax;
     p.seg = seg;
     p.P = P;
     p.sigma = sigma;
@@ -1012,10 +1069,10 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     p.sB_col = items[i].sB_col;
     p.r = a->rank;
     p.M = a->M;
-    p.u = static_cast<__nv_bfloat16*>(ctx->dec_u) + (size_t)i * kDecodeMaxTokens * kRankPadMax;
-    p.u_count = ctx->dec_cnt + i;
-    next_epoch[i] = ctx->dec_epoch[i] + (uint32_t)T;
-    p.u_target = next_epoch[i];
+    p.u = static_cast<__nv_bfloat16*>(ctx->dec_u) + (size_t)(s0 + i) * kDecodeMaxTokens * kRankPadMax;
+    p.u_count = ctx->dec_cnt + s0 + i;
+    next_epoch[i] = ctx->dec_epoch[s0 + i] + (uint32_t)T;
+    p.u_target = next_epoch[i] + (ctx->debug_stall_rank_rows ? 1u : 0u);  // (testing: a row nobody publishes)
     p.status = ctx->d_status;
     blk.cta_begin[i] = cta;
     blk.unit_begin[i] = unit;
@@ -1039,14 +1096,13 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
         *hit = fresh;
       }
       maps.tm[i][1] = hit->tm;
-      const int slot = 0;
-      if (ctx->dec_u_map_box[i][slot] != (uint32_t)p.xbox) {
-        const int32_t st = make_tensor_map_2d(ctx, &ctx->dec_u_map[i][slot], 0, p.u, (uint64_t)kDecodeMaxTokens, kRankPadMax,
+      if (ctx->dec_u_map_box[s0 + i] != (uint32_t)p.xbox) {
+        const int32_t st = make_tensor_map_2d(ctx, &ctx->dec_u_map[s0 + i], 0, p.u, (uint64_t)kDecodeMaxTokens, kRankPadMax,
                                               kRankPadMax * 2, (uint32_t)p.xbox, DEC_K, 128);
         if (st != ESSA_OK) return st;
-        ctx->dec_u_map_box[i][slot] = (uint32_t)p.xbox;
+        ctx->dec_u_map_box[s0 + i] = (uint32_t)p.xbox;
       }
-      maps.tm[i][2] = ctx->dec_u_map[i][slot];
+      maps.tm[i][2] = ctx->dec_u_map[s0 + i];
     }
     maps.tm[i][3] = a->tm_UBp[1][0];  // 128-row boxes of the U_B slabs
     maps.tm[i][4] = a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0];
@@ -1075,9 +1131,10 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
                                                 : cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt4Tmem>, maps, blk);
   if (e != cudaSuccess) return check_cuda(ctx, e, "essa_decode_kernel launch");
   ctx->launches += 1;
+  ctx->dec_set_issued[set & 1] += (uint32_t)grid_total;
   for (int i = 0; i < n; ++i) {
-    ctx->dec_pepoch[i] = next_pepoch[i];
-    ctx->dec_epoch[i] = next_epoch[i];
+    ctx->dec_pepoch[s0 + i] = next_pepoch[i];
+    ctx->dec_epoch[s0 + i] = next_epoch[i];
   }
   return ESSA_OK;
 }

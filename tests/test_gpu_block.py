@@ -165,3 +165,60 @@ def test_fused_draw_and_block_equals_separate_calls_and_oracle(torch, ctx, base,
                                     *cols[i], ad.rank)
         assert orc.relative_error(ys_f[i].float().cpu().numpy(), want) <= tol
     case.close()
+
+
+@pytest.mark.parametrize("base,dm,dkv,r,P,L,n_layers", [("3", 768, 128, 16, 200, 1, 2),     # decode, bf16, two layers
+                                                        ("3", 512, 192, 16, 64, 1, 8),      # eight layers (both scratch sets reused)
+                                                        ("5a", 512, 128, 64, 100, 1, 3),    # INT8 storage, tensor-memory mode
+                                                        ("2", 256, 64, 16, 3, 100, 2)])     # prefill sizes: issued block by block
+def test_layers_call_matches_block_calls_and_oracle(torch, ctx, base, dm, dkv, r, P, L, n_layers):
+    """essa_apply_layers over n_layers blocks (each layer its own adapters, activations and slice of the table):
+    every output equals the per-block call bit for bit at decode sizes and matches the oracle; repeated calls agree."""
+    import dataclasses
+    from tests.parity_utils import oracle_weight
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    n = len(cfg.projections)
+    offsets = wl.make_segments(cfg)
+    T = int(offsets[-1])
+    d_off = to_dev(torch, offsets)
+    # one table for all layers: layer l owns columns [l * d, (l + 1) * d), drawn by the oracle
+    rng = np.random.default_rng(77)
+    sigma = rng.uniform(0.05, 1.0, size=(cfg.P, n_layers * cfg.d)).astype(np.float32)
+    d_sigma = to_dev(torch, sigma)
+    layers, host = [], []
+    for l in range(n_layers):
+        cfg_l = dataclasses.replace(cfg, cfg_id=cfg.cfg_id * 100 + l)  # another seed per layer: distinct weights and tokens
+        ads = [wl.make_adapter(cfg_l, i) for i in range(n)]
+        hs = [ctx.load_adapter(a) for a in ads]
+        xs_h = [wl.make_tokens(cfg_l, i, T) for i in range(n)]
+        xs = [to_dev(torch, x, torch.bfloat16) for x in xs_h]
+        ys = [torch.empty((T, a.d_out), dtype=torch.bfloat16, device="cuda") for a in ads]
+        cols = [(l * cfg.d + a, l * cfg.d + b) for a, b in (cfg.sigma_cols(i) for i in range(n))]
+        layers.append([(hs[i], xs[i], cols[i], ys[i]) for i in range(n)])
+        host.append((ads, xs_h, cols))
+    launches0 = ctx.gpu_launches
+    ctx.apply_layers(layers, d_off, d_sigma)
+    torch.cuda.synchronize()
+    if T <= 256:
+        assert ctx.gpu_launches - launches0 == n_layers, "one launch per layer at decode sizes"
+    first = [[y.clone() for (_, _, _, y) in layer] for layer in layers]
+    tol = TOL_BF16 if cfg.w0_dtype == "bf16" else TOL_INT8
+    for l, (ads, xs_h, cols) in enumerate(host):
+        ys_blk = ctx.apply_block([it[0] for it in layers[l]], [it[1] for it in layers[l]], d_off, d_sigma, cols)
+        torch.cuda.synchronize()
+        for i in range(n):
+            if T <= 256:
+                assert torch.equal(first[l][i], ys_blk[i]), (l, i)
+            want = orc.apply_projection(oracle_weight(ads[i]), ads[i].U_A, ads[i].V_A, ads[i].U_B, ads[i].V_B, xs_h[i], offsets,
+                                        sigma, cols[i][0], cols[i][1], ads[i].rank)
+            assert orc.relative_error(first[l][i].float().cpu().numpy(), want) <= tol, (l, i)
+    for _ in range(3):  # the chained launches reuse the two scratch sets: results must not depend on timing
+        ctx.apply_layers(layers, d_off, d_sigma)
+    torch.cuda.synchronize()
+    if T <= 256:
+        for l in range(n_layers):
+            for i in range(n):
+                assert torch.equal(first[l][i], layers[l][i][3]), (l, i)
+    for layer in layers:
+        for it in layer:
+            it[0].free()
