@@ -431,6 +431,33 @@ def measure_config(key, cfg, args, env):
         barrier()
         warm_ms = max_over_ranks(w0.elapsed_time(w1)) / steps
 
+    # ---- multi-layer call (decode configurations): L layers' blocks in ONE essa_apply_layers call, each layer with its
+    # own device copy of the adapters (so every layer streams its W0 from HBM); per-layer time beside the single block's
+    layers_rec = None
+    if block_call and world == 1 and not args.no_layers:
+        L = {"3": 28, "5a": 80, "6a": 80}.get(key, 8)  # decoder layers of the backbone the shapes come from
+        adapters_again = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
+        while len(handle_sets) < L:
+            handle_sets.append([ctx.load_adapter(a) for a in adapters_again])
+        del adapters_again
+        ys_alt = [torch.empty_like(y) for y in ys]
+        layers = [[(handle_sets[l][i], xs[i], cols[i], (ys if l % 2 == 0 else ys_alt)[i]) for i in range(len(handles))]
+                  for l in range(L)]
+        prep_layers = ctx.prepare_layers(layers, d_off, sigma)
+        reps = 5
+        for _ in range(2):
+            prep_layers.run(stream_handle)
+        barrier()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0.record(stream)
+        for _ in range(reps):
+            prep_layers.run(stream_handle)
+        l1.record(stream)
+        barrier()
+        ms_layers = l0.elapsed_time(l1) / reps
+        layers_rec = {"n_layers": L, "ms_per_call": ms_layers, "ms_per_layer": ms_layers / L,
+                      "block_frac_per_layer": None, "note": "one essa_apply_layers call; the population draw is not part of it"}
+
     # ---- end to end through the host-buffer entry points (H2D of x/offsets/sigma and D2H of y inside the call)
     xh = [x.pin_memory() for x in xs_host]
     del xs_host
@@ -458,6 +485,26 @@ def measure_config(key, cfg, args, env):
         step_e2e()
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+    # the same with q, k and v reading ONE activation buffer (as in an attention block): it is copied in once
+    e2e_shared = None
+    if len(handles) == 4 and not args.single_calls and handles[0].d_in == handles[1].d_in == handles[2].d_in:
+        xh_shared = [xh[0], xh[0], xh[0], xh[3]]
+
+        def step_e2e_shared():
+            ctx.sample_population(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, out=sigma, k_begin=k_begin)
+            sig_h.copy_(sigma, non_blocking=True)
+            stream.synchronize()
+            ctx.apply_block_host(handles, xh_shared, off_h, sig_h, cols, yh)
+        for _ in range(2):
+            step_e2e_shared()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_e2e_shared()
+        torch.cuda.synchronize()
+        es_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+        e2e_shared = {"value": world * T * e2e_steps / (es_ms * 1e-3), "unit": UNIT, "ms_per_step": es_ms / e2e_steps,
+                      "h2d_bytes_per_step": int(xh[0].numel() * 2 + xh[3].numel() * 2 + off_h.numel() * 4 + sig_h.numel() * 4)}
     h2d = sum(x.numel() * 2 for x in xh) + (len(handles) if args.single_calls else 1) * (off_h.numel() * 4 + sig_h.numel() * 4)
     d2h = sum(y.numel() * 2 for y in yh) + sig_h.numel() * 4
     e2e = {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
@@ -511,6 +558,11 @@ def measure_config(key, cfg, args, env):
            "kernel_timing": "CUDA events around every launch, inside the timed steps" if events_inside
                             else "CUDA events around every launch in a second pass of the same steps (not inside the timed steps)",
            "roofline": roofline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+    if layers_rec is not None:
+        layers_rec["block_frac_per_layer"] = model["time_s"] * 1e3 / layers_rec["ms_per_layer"]
+        rec["layers"] = layers_rec
+    if e2e_shared is not None:
+        rec["e2e_shared_x"] = e2e_shared
     for hs in handle_sets:
         for h in hs:
             h.free()
@@ -596,6 +648,7 @@ def main():
     ap.add_argument("--fuse-down", type=int, default=-1, help="override ESSA_OPT_FUSE_DOWN (0 / 1)")
     ap.add_argument("--single-calls", action="store_true",
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
+    ap.add_argument("--no-layers", action="store_true", help="skip the multi-layer (essa_apply_layers) measurement of decode configurations")
     ap.add_argument("--separate-calls", action="store_true",
                     help="decode configurations: essa_sample_population then essa_apply_block instead of the fused call")
     ap.add_argument("--candidates", type=int, default=0, help="override the population size (smaller case for profiler captures)")

@@ -604,10 +604,18 @@ static int32_t host_pipeline(essa_ctx* ctx, const essa_block_item* items, int32_
   if (essa_validate_segments(seg_host, P, T) != ESSA_OK)
     return fail(ctx, ESSA_ERR_INVALID_ARG, std::string(who) + ": seg_offsets must rise from 0 to T");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  // staging: the items' x (and y) one after the other, each 256-byte aligned
+  // staging: the items' x (and y) one after the other, each 256-byte aligned.  Items that pass the SAME host
+  // activations (the q, k, v projections of a block read one x) share one staged copy: x_src[i] is the first item
+  // with that pointer and width, and only such first items are copied in.
   size_t x_off[ESSA_MAX_BLOCK_ITEMS + 1] = {0}, y_off[ESSA_MAX_BLOCK_ITEMS + 1] = {0};
+  int x_src[ESSA_MAX_BLOCK_ITEMS];
+  size_t x_at[ESSA_MAX_BLOCK_ITEMS];
   for (int32_t i = 0; i < n; ++i) {
-    x_off[i + 1] = x_off[i] + (((size_t)T * items[i].adapter->d_in * 2 + 255) & ~(size_t)255);
+    x_src[i] = i;
+    for (int32_t j = 0; j < i; ++j)
+      if (items[j].x == items[i].x && items[j].adapter->d_in == items[i].adapter->d_in) { x_src[i] = x_src[j]; break; }
+    x_at[i] = x_src[i] == i ? x_off[i] : x_at[x_src[i]];
+    x_off[i + 1] = x_off[i] + (x_src[i] == i ? (((size_t)T * items[i].adapter->d_in * 2 + 255) & ~(size_t)255) : 0);
     y_off[i + 1] = y_off[i] + (((size_t)T * items[i].adapter->d_out * 2 + 255) & ~(size_t)255);
   }
   const size_t ob = (size_t)(P + 1) * 4, sb = (size_t)P * ld_sigma * 4;
@@ -640,8 +648,9 @@ static int32_t host_pipeline(essa_ctx* ctx, const essa_block_item* items, int32_
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_sigma.ptr, sigma_host, sb, cudaMemcpyHostToDevice, stream);
     essa_block_item dev[ESSA_MAX_BLOCK_ITEMS];
     for (int32_t i = 0; i < n && e == cudaSuccess; ++i) {
-      e = cudaMemcpyAsync(xd + x_off[i], items[i].x, (size_t)T * items[i].adapter->d_in * 2, cudaMemcpyHostToDevice, stream);
-      dev[i] = essa_block_item{items[i].adapter, xd + x_off[i], items[i].sA_col, items[i].sB_col, yd + y_off[i]};
+      if (x_src[i] == i)
+        e = cudaMemcpyAsync(xd + x_at[i], items[i].x, (size_t)T * items[i].adapter->d_in * 2, cudaMemcpyHostToDevice, stream);
+      dev[i] = essa_block_item{items[i].adapter, xd + x_at[i], items[i].sA_col, items[i].sB_col, yd + y_off[i]};
     }
     if (e != cudaSuccess) return check_cuda(ctx, e, "host call: H2D");
     st = essa_apply_block(ctx, dev, n, T, static_cast<const int32_t*>(ctx->stage_off.ptr), P,
@@ -689,12 +698,14 @@ static int32_t host_pipeline(essa_ctx* ctx, const essa_block_item* items, int32_
     for (int c = 0; c < n_chunks; ++c, ++unit) {
       const int64_t t0 = seg_host[first[c]], t1 = seg_host[first[c + 1]];
       const size_t xo = (size_t)t0 * a->d_in * 2, yo = (size_t)t0 * a->d_out * 2;
-      e = cudaMemcpyAsync(xd + x_off[i] + xo, xh + xo, (size_t)(t1 - t0) * a->d_in * 2, cudaMemcpyHostToDevice, ctx->host_h2d);
+      e = cudaSuccess;
+      if (x_src[i] == i)  // (a shared x was copied by an earlier item; copies and events on host_h2d are in order)
+        e = cudaMemcpyAsync(xd + x_at[i] + xo, xh + xo, (size_t)(t1 - t0) * a->d_in * 2, cudaMemcpyHostToDevice, ctx->host_h2d);
       if (e == cudaSuccess) e = cudaEventRecord(ctx->host_events[2 * unit], ctx->host_h2d);
       if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->host_events[2 * unit], 0);
       if (e != cudaSuccess) { drain(); return check_cuda(ctx, e, "host call: H2D"); }
       if (t1 > t0) {
-        st = essa_apply_projection(ctx, a, xd + x_off[i] + xo, t1 - t0, static_cast<const int32_t*>(ctx->stage_off.ptr) + first[c] + c,
+        st = essa_apply_projection(ctx, a, xd + x_at[i] + xo, t1 - t0, static_cast<const int32_t*>(ctx->stage_off.ptr) + first[c] + c,
                                    first[c + 1] - first[c], static_cast<const float*>(ctx->stage_sigma.ptr) + (size_t)first[c] * ld_sigma,
                                    ld_sigma, items[i].sA_col, items[i].sB_col, yd + y_off[i] + yo, stream_v);
         if (st != ESSA_OK) { drain(); return st; }

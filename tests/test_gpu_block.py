@@ -222,3 +222,26 @@ def test_layers_call_matches_block_calls_and_oracle(torch, ctx, base, dm, dkv, r
     for layer in layers:
         for it in layer:
             it[0].free()
+
+
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("3", 512, 128, 16, 100, 1),     # decode sizes: one copy in, one block launch
+                                               ("2", 512, 128, 16, 5, 1000)])  # 5000 tokens: the chunked three-stage pipeline
+def test_host_block_call_with_shared_activations(torch, ctx, base, dm, dkv, r, P, L):
+    """q, k and v reading ONE host activation buffer (as in an attention block): the host-buffer call stages it once;
+    every output still matches the oracle."""
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    n = len(cfg.projections)
+    x_qkv, x_o = case.tokens(0), case.tokens(3)
+    xh_qkv = torch.from_numpy(x_qkv).to(torch.bfloat16).pin_memory()
+    xh_o = torch.from_numpy(x_o).to(torch.bfloat16).pin_memory()
+    xs_h = [xh_qkv, xh_qkv, xh_qkv, xh_o]
+    ys_h = [torch.empty((case.T, case.adapters[i].d_out), dtype=torch.bfloat16).pin_memory() for i in range(n)]
+    off_h = torch.from_numpy(case.offsets).pin_memory()
+    sig_h = torch.from_numpy(case.sigma32).pin_memory()
+    cols = [cfg.sigma_cols(i) for i in range(n)]
+    ctx.apply_block_host([case.handles[i] for i in range(n)], xs_h, off_h, sig_h, cols, ys_h)
+    for i in range(n):
+        want = case.oracle_projection(i, x_o if i == 3 else x_qkv)
+        assert orc.relative_error(ys_h[i].float().numpy(), want) <= TOL_BF16, i
+    case.close()
