@@ -101,6 +101,12 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   ready, the wait runs out, the output is undefined and essa_get_status reports ESSA_ERR_DEVICE_TIMEOUT. */
 #define ESSA_OPT_WAIT_LIMIT_MCYCLES 3
 #define ESSA_OPT_DEBUG_STALL_RANK_ROWS 4
+/*   ESSA_OPT_DECODE_PAIRS (0 / 1, default 0): run the decode kernel's CTAs as tcgen05 CTA pairs (two W0 row tiles per
+ *   MMA of 256 rows, each CTA loading half of the token rows of x) when the token count is a multiple of 32.  The MMAs
+ *   themselves are two to four times cheaper that way, but the pair's leader waits for both CTAs' operands before every
+ *   K block and the launch measured 15 - 50 % SLOWER on B200 (config 3: 37 -> 44 us per step, config 5a: 129 -> 197 us),
+ *   so it is off unless asked for. */
+#define ESSA_OPT_DECODE_PAIRS 5
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

@@ -64,8 +64,13 @@ constexpr int kUbSlots = 2;                      // kModeInt8Tmem: the U_B slabs
 constexpr int kFinishTokens = 8;   // tokens of one finishing unit of the rank path (two threads x four tokens per rank row)
 static_assert(kFinishTokens == 8, "finish_unit loads four tokens per thread as one float4");
 constexpr int kMaxPSlices = 32;    // slots of partial down-projections per projection
-constexpr int kVatStages = 2;      // ring of V_A^T tiles (used only during a CTA's slice)
-constexpr int VAT_SLOT_BYTES = kRankPadMax * DEC_K * 2;  // 8 KB: up to 64 rank rows of 64 input features
+// Ring of V_A^T tiles (used only during a CTA's slice): 16 KB cut into slots of r_pad rows x 128 bytes, so a rank-16
+// adapter has eight tiles in flight and a rank-64 adapter two.  (A projection with few row tiles has long slices,
+// seven K blocks at the 512-channel k / v projections of the 7B shape: with two slots their V_A^T loads, one L2 round
+// trip each, ran one after the other and the whole rank path of the launch waited for them.)
+constexpr int kVatStages = 8;      // most slots (barriers are laid out for this many)
+constexpr int VAT_RING_BYTES = 2 * kRankPadMax * DEC_K * 2;  // 16 KB
+__host__ __device__ inline int vat_stages(int r_pad) { const int s = VAT_RING_BYTES / (r_pad * 128); return s > kVatStages ? kVatStages : s; }
 constexpr int DEC_AUX_BYTES = 8 * 1024;  // barriers, flags, finishing-step buffers
 constexpr uint32_t TMEM_P_COL = 256;     // the down-projection accumulator sits behind the main one
 
@@ -277,9 +282,18 @@ __device__ __forceinline__ void sum_store(uint32_t mine /*shared-space address*/
 
 __host__ __device__ constexpr uint32_t tmem_a_col(int stage) { return stage < 4 ? 128u + 32u * stage : 384u + 32u * (stage - 4); }
 
-template <int MODE>
+// PAIR: two CTAs with neighbouring cluster ranks (two W0 row tiles of the same K split) act as one 256-row tcgen05
+// CTA pair (cta_group::2).  Each streams (and, for quantised storage, converts) its own W0 tile but only its HALF of
+// the token rows of x; the leader (even rank) issues MMAs of M = 256 that read both CTAs' operands and write both
+// CTAs' accumulators.  Measured on B200: a cta_group::1 MMA of 128 rows costs ~150 cycles whatever its width, a
+// cta_group::2 MMA of 256 x N x 16 runs at the nominal rate (N / 2 cycles), so a pair spends a quarter (128 tokens)
+// to a half (256 tokens) of the tensor-core time per W0 tile, and a CTA brings in half the x bytes.
+// "full" barriers of rings the pair's MMA reads live in the leader, which posts the bytes of both CTAs; the peer's
+// copies complete on them through their cluster address; "empty" barriers exist in both CTAs (multicast commits).
+template <int MODE, bool PAIR>
 __global__ void __launch_bounds__(MODE != kModeBf16 ? kDecThreadsInt8 : kDecThreads, 1)
 essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ DBlock blk) {
+  static_assert(!(PAIR && MODE == kModeInt8Smem), "the shared-memory conversion mode has no CTA-pair variant");
   constexpr bool INT8 = MODE == kModeInt8Smem;   // codes converted through shared memory
   constexpr bool TS = MODE >= kModeInt8Tmem;     // codes converted into tensor memory (A operand from TMEM)
   constexpr bool I4 = MODE == kModeInt4Tmem;     // ... from packed INT4 codes with group-wise scales
@@ -297,14 +311,16 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int SW = p.w_stages, SX = p.x_stages;
-  const int x_bytes = p.tn * 128;
+  const int hn = PAIR ? p.tn / 2 : p.tn;  // token rows of an x tile held by this CTA
+  const int x_bytes = hn * 128;
   constexpr int W_SLOT = I4 ? RAW4_TILE_BYTES : QUANT ? RAW_TILE_BYTES : W_TILE_BYTES;
   const int SC = INT8 ? p.c_stages : (TS ? kUbSlots : 0);   // 16 KB slots behind the W0 ring
   const int SA = TS ? p.c_stages : 1;                       // kModeInt8Tmem: converted tiles in tensor memory
   // V_A^T tiles first: their MMA descriptor spans 128 rows, of which only the r_pad rows of the TMA box are data
   // (the accumulator rows beyond are never read), so the 16 KB it covers must lie inside the allocation
   uint8_t* smem_v = smem;
-  uint8_t* smem_w = smem_v + kVatStages * VAT_SLOT_BYTES;  // W0 ring as stored (bf16: the U_B slabs are its last items)
+  const int SV = vat_stages(p.r_pad), v_slot = p.r_pad * 128;
+  uint8_t* smem_w = smem_v + VAT_RING_BYTES;  // W0 ring as stored (bf16: the U_B slabs are its last items)
   uint8_t* smem_c = smem_w + SW * W_SLOT;      // INT8: ring of converted bf16 tiles (the U_B slabs are its last items)
   uint8_t* smem_x = smem_c + SC * W_TILE_BYTES;  // x ring (the u tile is its last item)
   uint8_t* aux = smem_x + SX * x_bytes;
@@ -324,9 +340,16 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const uint32_t bar_ub = bar_p + 8;  // kModeInt8Tmem: one per U_B slab
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = (int)cluster_ctarank();
+  const int crank = (int)cluster_ctarank();
+  const int half = PAIR ? (crank & 1) : 0;        // which W0 tile / which half of the tokens of the pair
+  const int split = PAIR ? (crank >> 1) : crank;  // K split
+  const bool leader = half == 0;
+  const uint32_t leader_rank = (uint32_t)(crank & ~1);
+  const uint16_t pair_mask = (uint16_t)(3u << leader_rank);
   const bool is_main = (int)blockIdx.x < blk.cta_begin[blk.n_proj];  // later CTAs of the grid only take rank-path units
-  const int m_tile = ((int)blockIdx.x - blk.cta_begin[pi]) / p.splits;
+  const int m_tile = PAIR ? (((int)blockIdx.x - blk.cta_begin[pi]) / (2 * p.splits)) * 2 + half
+                          : ((int)blockIdx.x - blk.cta_begin[pi]) / p.splits;
+  const int owner_idx = PAIR ? (m_tile >> 1) : m_tile;  // which slice of the down-projection (a pair's leader owns it)
   // this CTA's K blocks [kb0, kb1)
   const int kbase = p.main_kb / p.splits, krem = p.main_kb % p.splits;
   const int kb0 = split * kbase + min(split, krem);
@@ -339,20 +362,26 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   constexpr uint32_t TMEM_COLS = 512;  // main accumulator (up to 256 tokens) + down-projection accumulator
   // The K loop starts at this CTA's slice of the down-projection and wraps around: item i is local K block
   // (r0 + i) mod nkb, and the first c_own items also feed the second accumulator.
-  const int r0 = nkb > 0 ? (m_tile * p.p_c) % nkb : 0;
-  const int c_own = (is_main && m_tile * p.p_c < nkb) ? min(p.p_c, nkb - m_tile * p.p_c) : 0;
+  const int r0 = nkb > 0 ? (owner_idx * p.p_c) % nkb : 0;  // (the same in both CTAs of a pair)
+  const int c_own = (is_main && leader && owner_idx * p.p_c < nkb) ? min(p.p_c, nkb - owner_idx * p.p_c) : 0;
   auto kcol = [&](int i) { const int l = r0 + i; return (kb0 + (l >= nkb ? l - nkb : l)) * DEC_K; };
 
+  // a copy whose completion the pair's MMA waits for: counted on the leader's barrier
+  auto tma_pair = [&](uint32_t dst, const CUtensorMap* tm, int c_inner, int c_outer, uint32_t fb) {
+    if (PAIR) tma_load_2d_pair(dst, tm, c_inner, c_outer, map_to_cta(fb, leader_rank));
+    else tma_load_2d(dst, tm, c_inner, c_outer, fb);
+  };
   auto load_w = [&](int i) {  // item i of the W0 ring
     const int s = i % SW;
     const uint32_t fb = bar_wfull + 8 * s;
-    mbar_expect_tx(fb, (uint32_t)W_SLOT);
     const uint32_t dst = smem_u32(smem_w + s * W_SLOT);
-    if (QUANT) {  // 128 rows of 64 codes (unswizzled; kModeInt8Tmem: 64-byte swizzle)
+    if (QUANT) {  // 128 rows of 64 codes (unswizzled; tensor-memory modes: swizzled); read by this CTA's converters only
+      mbar_expect_tx(fb, (uint32_t)W_SLOT);
       tma_load_2d(dst, &tmW, I4 ? kcol(i) / 2 : kcol(i), m_tile * DEC_M, fb);
-    } else {     // one 128-row box
+    } else {     // one 128-row box, an operand of the (pair's) MMA
+      if (leader) mbar_expect_tx(fb, (uint32_t)(PAIR ? 2 * W_SLOT : W_SLOT));
       const CUtensorMap* tm = i < nkb ? &tmW : ((i - nkb) == 0 ? &tmUB0 : &tmUB1);
-      tma_load_2d(dst, tm, i < nkb ? kcol(i) : 0, m_tile * DEC_M, fb);
+      tma_pair(dst, tm, i < nkb ? kcol(i) : 0, m_tile * DEC_M, fb);
     }
   };
   auto load_ub = [&](int e) {  // INT8: U_B slab e goes straight into item nkb + e of the converted ring
@@ -363,34 +392,37 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const CUtensorMap* tm = e == 0 ? &tmUB0 : &tmUB1;
     tma_load_2d(dst, tm, 0, m_tile * DEC_M, fb);
   };
-  auto load_ub_slot = [&](int e) {  // kModeInt8Tmem: U_B slab e into its own slot
+  auto load_ub_slot = [&](int e) {  // tensor-memory modes: U_B slab e into its own slot
     const uint32_t fb = bar_ub + 8 * e;
-    mbar_expect_tx(fb, (uint32_t)W_TILE_BYTES);
-    tma_load_2d(smem_u32(smem_c + e * W_TILE_BYTES), e == 0 ? &tmUB0 : &tmUB1, 0, m_tile * DEC_M, fb);
+    if (leader) mbar_expect_tx(fb, (uint32_t)(PAIR ? 2 * W_TILE_BYTES : W_TILE_BYTES));
+    tma_pair(smem_u32(smem_c + e * W_TILE_BYTES), e == 0 ? &tmUB0 : &tmUB1, 0, m_tile * DEC_M, fb);
   };
   auto load_x = [&](int i) {  // item i of the x ring
     const int s = i % SX;
     const uint32_t fb = bar_xfull + 8 * s;
     const uint32_t dst = smem_u32(smem_x + s * x_bytes);
-    mbar_expect_tx(fb, (uint32_t)x_bytes);
+    if (leader) mbar_expect_tx(fb, (uint32_t)(PAIR ? 2 * x_bytes : x_bytes));
     const CUtensorMap* tm = i < nkb ? &tmX : &tmU;
     const int col = i < nkb ? kcol(i) : 0;
-    for (int r = 0; r < p.tn; r += p.xbox) tma_load_2d(dst + (uint32_t)(r * 128), tm, col, r, fb);
+    for (int r = 0; r < hn; r += p.xbox) tma_pair(dst + (uint32_t)(r * 128), tm, col, half * hn + r, fb);
   };
   auto load_v = [&](int i) {  // V_A^T tile of item i < c_own: r_pad rank rows x 64 input features
-    const int s = i % kVatStages;
+    const int s = i % SV;
     const uint32_t fb = bar_vfull + 8 * s;
-    mbar_expect_tx(fb, (uint32_t)(p.r_pad * 128));
-    tma_load_2d(smem_u32(smem_v + s * VAT_SLOT_BYTES), &tmV, kcol(i), 0, fb);
+    mbar_expect_tx(fb, (uint32_t)v_slot);
+    tma_load_2d(smem_u32(smem_v + s * v_slot), &tmV, kcol(i), 0, fb);
   };
 
-  const int first_w = n_w < SW ? n_w : SW;  // the ring starts empty: its first fill needs no wait
+  // the ring starts empty: its first fill needs no wait (a pair's peer whose copies count on the leader's barriers
+  // starts after the cluster barrier below, once those barriers exist)
+  const int first_w = (PAIR && !QUANT && !leader) ? 0 : (n_w < SW ? n_w : SW);
   if (threadIdx.x == 0) {
     // kModeInt8Tmem: a tile of codes is read, and its converted tile written, by four warps (one arrival each)
     for (int s = 0; s < SW; ++s) { mbar_init(bar_wfull + 8 * s, 1); mbar_init(bar_wempty + 8 * s, TS ? 4 : 1); }
     for (int s = 0; s < SX; ++s) { mbar_init(bar_xfull + 8 * s, 1); mbar_init(bar_xempty + 8 * s, 1); }
     if (TS) {
-      for (int s = 0; s < SA; ++s) { mbar_init(bar_cfull + 8 * s, 4); mbar_init(bar_cempty + 8 * s, 1); }
+      // (a pair's leader collects the converting warps of both CTAs)
+      for (int s = 0; s < SA; ++s) { mbar_init(bar_cfull + 8 * s, PAIR ? 8 : 4); mbar_init(bar_cempty + 8 * s, 1); }
       for (int e = 0; e < kUbSlots; ++e) mbar_init(bar_ub + 8 * e, 1);
     } else {
       for (int s = 0; s < SC; ++s) { mbar_init(bar_cfull + 8 * s, 1); mbar_init(bar_cempty + 8 * s, 1); }
@@ -404,16 +436,15 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     *reinterpret_cast<volatile int*>(tmem_slot + 4) = 0;  // ... and whose turn it is to claim a slot
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int i = 0; i < first_w; ++i) load_w(i);  // the frozen weights depend on nothing: stream at once
-    if (TS) for (int e = 0; e < n_ext; ++e) load_ub_slot(e);
   }
   if (warp == 1 && is_main) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
-  __syncthreads();
+  if (PAIR) cluster_sync_all(); else __syncthreads();  // PAIR: both CTAs' barriers exist before either uses the other's
   tc_fence_after();
-  const uint32_t tmem_base = is_main ? *tmem_slot : 0u;
+  const uint32_t tmem_base = is_main ? *tmem_slot : 0u;  // PAIR: the same address in both CTAs (an SM's only allocation)
   // Everything up to here (barriers, TMEM, the first tiles of the frozen W0) depends on no earlier kernel and, with
   // a programmatic dependent launch, overlaps the kernel before this one in the stream (typically the population
   // draw); x, the singular values, the scratch buffers and y are touched only after this point.  In a fused draw +
@@ -453,16 +484,29 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       while (!mbar_try_wait(bar_f + 8 * (i % S), (uint32_t)((i / S) & 1)) && clock64() - t0 < kWaitLimitCycles) {}
     }
   };
+  // a pair's peer cannot see the completion of copies that are counted on the leader's barrier: it gives them time
+  auto drain_remote = [&]() {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}
+  };
   if (warp == 0) {
     if (lane == 0) {
       int iw = first_w, iv = 0;
       bool ok = true;
+      if (TS) for (int e = 0; e < n_ext; ++e) load_ub_slot(e);
       while (ok && (iw < n_w || iv < c_own)) {
-        // the V_A^T tile of item iv goes out no later than the W0 tile of the same item
+        // The V_A^T tile of item iv goes out no later than the W0 tile of the same item, as soon as its slot is free;
+        // the thread only blocks for the slot when nothing else is left to issue or when the W0 slot it would wait
+        // for next is held by an MMA that itself needs this tile.
         if (iv < c_own && iv <= iw) {
-          if (iv >= kVatStages) ok = mbar_wait(bar_vempty + 8 * (iv % kVatStages), (uint32_t)(((iv / kVatStages) & 1) ^ 1), abort_flag, p.status);
-          if (ok) load_v(iv++);
-          continue;
+          const uint32_t vb = bar_vempty + 8 * (iv % SV), vph = (uint32_t)(((iv / SV) & 1) ^ 1);
+          bool slot_free = iv < SV || mbar_test_wait(vb, vph);
+          if (!slot_free && (iw >= n_w || iw - SW >= iv)) slot_free = ok = mbar_wait(vb, vph, abort_flag, p.status);
+          if (slot_free) {
+            load_v(iv++);
+            continue;
+          }
+          if (!ok) break;
         }
         if (iw < n_w) {
           if (iw >= SW) ok = mbar_wait(bar_wempty + 8 * (iw % SW), (uint32_t)(((iw / SW) & 1) ^ 1), abort_flag, p.status);
@@ -470,8 +514,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         }
       }
       if (!ok || *abort_flag) {
-        drain(iw, SW, bar_wfull);
-        drain(iv, kVatStages, bar_vfull);
+        if (PAIR && !QUANT && !leader) drain_remote(); else drain(iw, SW, bar_wfull);
+        drain(iv, SV, bar_vfull);
       }
     }
   } else if (warp == kXWarp) {
@@ -500,12 +544,24 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         }
         if (ok) load_x(ix++);
       }
-      if (!ok || *abort_flag) drain(ix, SX, bar_xfull);
+      if (!ok || *abort_flag) { if (PAIR && !leader) drain_remote(); else drain(ix, SX, bar_xfull); }
     }
   } else if (warp == 1 && is_main) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(DEC_M, p.tn);
+    if (lane == 0 && leader) {
+      const uint32_t idesc = make_idesc(PAIR ? 2 * DEC_M : DEC_M, p.tn);
+      auto mma = [&](uint32_t d, uint64_t da, uint64_t db, uint32_t acc) {
+        if (PAIR) umma_bf16_2cta(d, da, db, idesc, acc); else umma_bf16(d, da, db, idesc, acc);
+      };
+      auto mma_ts = [&](uint32_t d, uint32_t ta, uint64_t db, uint32_t acc) {
+        if (PAIR) umma_bf16_ts_2cta(d, ta, db, idesc, acc); else umma_bf16_ts(d, ta, db, idesc, acc);
+      };
+      auto commit = [&](uint32_t bar) {  // PAIR: to the barrier at this offset in both CTAs
+        if (PAIR) umma_commit_2cta(bar, pair_mask); else umma_commit(bar);
+      };
+      auto commit_own = [&](uint32_t bar) {  // to this CTA's barrier only
+        if (PAIR) umma_commit_2cta(bar, (uint16_t)(1u << crank)); else umma_commit(bar);
+      };
       bool ok = true;
       for (int i = 0; i < nkb; ++i) {
         const int sw = INT8 ? i % SC : TS ? i % SA : i % SW, sx = i % SX;
@@ -519,24 +575,25 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         if (TS) {  // A operand: the converted tile in tensor memory, 8 columns (16 bf16) per K step
           const uint32_t ta = tmem_base + tmem_a_col(sw);
 #pragma unroll
-          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16_ts(tmem_base, ta + 8 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < DEC_K / 16; ++k) mma_ts(tmem_base, ta + 8 * k, dx + 2 * k, (i > 0 || k > 0) ? 1u : 0u);
         } else {
 #pragma unroll
-          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base, dw + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < DEC_K / 16; ++k) mma(tmem_base, dw + 2 * k, dx + 2 * k, (i > 0 || k > 0) ? 1u : 0u);
         }
         if (i < c_own) {
           // this CTA's slice of the down-projection: V_A^T tile against the same x tile, second accumulator
-          const int sv = i % kVatStages;
-          if (!mbar_wait(bar_vfull + 8 * sv, (uint32_t)((i / kVatStages) & 1), abort_flag, p.status)) { ok = false; break; }
+          const int sv = i % SV;
+          if (!mbar_wait(bar_vfull + 8 * sv, (uint32_t)((i / SV) & 1), abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t dv = make_smem_desc(smem_u32(smem_v + sv * VAT_SLOT_BYTES));
+          const uint64_t dv = make_smem_desc(smem_u32(smem_v + sv * v_slot));
 #pragma unroll
-          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base + TMEM_P_COL, dv + 2 * k, dx + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-          umma_commit(bar_vempty + 8 * sv);
-          if (i == c_own - 1) umma_commit(bar_p);  // the slice is complete
+          // (PAIR: the peer's rows of this accumulator come from whatever its shared memory holds there; never read)
+          for (int k = 0; k < DEC_K / 16; ++k) mma(tmem_base + TMEM_P_COL, dv + 2 * k, dx + 2 * k, (i > 0 || k > 0) ? 1u : 0u);
+          commit_own(bar_vempty + 8 * sv);
+          if (i == c_own - 1) commit_own(bar_p);  // the slice is complete
         }
-        umma_commit(((INT8 || TS) ? bar_cempty : bar_wempty) + 8 * sw);
-        umma_commit(bar_xempty + 8 * sx);
+        commit(((INT8 || TS) ? bar_cempty : bar_wempty) + 8 * sw);
+        commit(bar_xempty + 8 * sx);
       }
       if (ok && n_ext > 0) {
         // rank term: u tile (x ring item nkb) against the U_B slabs (W0 ring items nkb ..)
@@ -550,13 +607,13 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
           if (!mbar_wait(ubar, TS ? 0u : (uint32_t)((INT8 ? i / SC : i / SW) & 1), abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint64_t dub = make_smem_desc(smem_u32(((INT8 || TS) ? smem_c : smem_w) + su * W_TILE_BYTES));
-          for (int k = 0; k < ksteps; ++k) umma_bf16(tmem_base, dub + 2 * k, du + 2 * k, idesc, 1u);
+          for (int k = 0; k < ksteps; ++k) mma(tmem_base, dub + 2 * k, du + 2 * k, 1u);
         }
       }
       if (ok) {
-        umma_commit(bar_d);
+        commit(bar_d);
       } else {
-        umma_commit(bar_drain);
+        commit_own(bar_drain);
         const long long t0 = clock64();
         while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < kWaitLimitCycles) {}
       }
@@ -704,7 +761,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(bar_cfull + 8 * sa);
+        if (PAIR) mbar_arrive_cluster(map_to_cta(bar_cfull + 8 * sa, leader_rank)); else mbar_arrive(bar_cfull + 8 * sa);
         mbar_arrive(bar_wempty + 8 * sr);
       }
     }
@@ -728,7 +785,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         while (!mbar_try_wait(bar_p, 0)) {}  // complete: returns at once (acquire for every lane)
         tc_fence_after();
         if (quad * 32 < p.r_pad) {
-          float* slot = p.p_part + (size_t)(split * p.p_per_split + m_tile) * kDecodeMaxTokens * kRankPadMax;
+          float* slot = p.p_part + (size_t)(split * p.p_per_split + owner_idx) * kDecodeMaxTokens * kRankPadMax;
 #pragma unroll 1
           for (int c = 0; c < p.tn / 16; ++c) {
             float v[16];
@@ -803,7 +860,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       tmem_ld16(t_lane + c * 16, v);
       const int owner = (c * 16) / per;
       const int j = c * 16 - owner * per;  // first token of the chunk within the owner's slice
-      const uint32_t dst = map_to_cta(recv_addr + (uint32_t)((((split * per + j) * DEC_M) + row) * 4), (uint32_t)owner);
+      const uint32_t dst = map_to_cta(recv_addr + (uint32_t)((((split * per + j) * DEC_M) + row) * 4),
+                                      (uint32_t)(PAIR ? 2 * owner + half : owner));
 #pragma unroll
       for (int i = 0; i < 16; ++i) st_dsmem_f32(dst + (uint32_t)(i * DEC_M * 4), v[i]);
     }
@@ -848,12 +906,13 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
 // Shared-memory rings: V_A^T tiles, the W0 ring (16 KB bf16 tiles, or 8 KB tiles of codes), the 16 KB slots behind it
 // (kModeInt8Smem: c_stages converted tiles; kModeInt8Tmem: the U_B slabs), the x ring.
 inline int dec_w_slot(int mode) { return mode == kModeBf16 ? W_TILE_BYTES : mode == kModeInt4Tmem ? RAW4_TILE_BYTES : RAW_TILE_BYTES; }
-inline int dec_ring_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
+// (x_rows: token rows of an x tile held by one CTA: all of them, or half when the CTAs work in pairs)
+inline int dec_ring_bytes(int mode, int w_stages, int c_stages, int x_stages, int x_rows) {
   const int slots16k = mode == kModeInt8Smem ? c_stages : mode >= kModeInt8Tmem ? kUbSlots : 0;
-  return kVatStages * VAT_SLOT_BYTES + w_stages * dec_w_slot(mode) + slots16k * W_TILE_BYTES + x_stages * tn * 128;
+  return VAT_RING_BYTES + w_stages * dec_w_slot(mode) + slots16k * W_TILE_BYTES + x_stages * x_rows * 128;
 }
-inline int dec_smem_bytes(int mode, int w_stages, int c_stages, int x_stages, int tn) {
-  return 1024 + dec_ring_bytes(mode, w_stages, c_stages, x_stages, tn) + DEC_AUX_BYTES;
+inline int dec_smem_bytes(int mode, int w_stages, int c_stages, int x_stages, int x_rows) {
+  return 1024 + dec_ring_bytes(mode, w_stages, c_stages, x_stages, x_rows) + DEC_AUX_BYTES;
 }
 // INT8 storage converts into tensor memory whenever the accumulators leave room for the converted tiles there.
 // INT4 storage has the tensor-memory mode only: larger calls take the prefill kernels (negative: no decode schedule).
@@ -867,14 +926,19 @@ inline int dec_mode(int w0_dtype, int tn) {
 
 // Schedule shared by the projections of one decode launch (n of them, sizes d_in[i] -> d_out[i], same storage type):
 // cluster size, ring depths.  Returns false when the launch would not fit one wave of the GPU.
-static bool plan_decode_block(int n, const int* d_in, const int* d_out, int w0_dtype, int64_t T, int sm_count, int* splits_out,
-                              int* w_stages_out, int* x_stages_out, int* m_tiles_total_out, int* c_stages_out = nullptr) {
+// *pair_out: the CTAs work as tcgen05 pairs (allow_pair, a token count that halves into multiples of 16, a mode that
+// has the pair variant, and no fewer CTAs streaming than without).
+static bool plan_decode_block(int n, const int* d_in, const int* d_out, int w0_dtype, int64_t T, int sm_count, bool allow_pair,
+                              int* splits_out, int* w_stages_out, int* x_stages_out, int* m_tiles_total_out,
+                              int* c_stages_out = nullptr, bool* pair_out = nullptr) {
   if (T <= 0 || T > kDecodeMaxTokens || n < 1 || n > kMaxBlockProj) return false;
   const int sm = sm_count > 0 ? sm_count : 148;
   const int tn = (int)((T + 15) / 16) * 16;
-  int m_total = 0, min_kb = 1 << 30;
+  int m_total = 0, m_pairs = 0, min_kb = 1 << 30;
   for (int i = 0; i < n; ++i) {
-    m_total += (d_out[i] + DEC_M - 1) / DEC_M;
+    const int m = (d_out[i] + DEC_M - 1) / DEC_M;
+    m_total += m;
+    m_pairs += (m + 1) / 2;  // an odd last tile is paired with an empty one
     if (d_in[i] / DEC_K < min_kb) min_kb = d_in[i] / DEC_K;
   }
   // cluster size: a power of two (packs into a GPC's SMs without stragglers), at most 8 (portable limit).
@@ -885,16 +949,28 @@ static bool plan_decode_block(int n, const int* d_in, const int* d_out, int w0_d
   if (n > 1 && m_total > resident(1)) return false;
   int splits = 1;
   while (splits * 2 <= 8 && m_total * splits * 2 <= resident(splits * 2) && splits * 2 <= min_kb) splits *= 2;
+  const int mode = dec_mode(w0_dtype, tn);
+  if (mode < 0) return false;
+  // pairs: a cluster is 2 x splits CTAs
+  bool pair = false;
+  if (allow_pair && mode != kModeInt8Smem && tn % 32 == 0 && tn >= 64 && 2 * m_pairs <= resident(2)) {
+    int ps = 1;
+    while (ps * 4 <= 8 && 2 * m_pairs * ps * 2 <= resident(ps * 4) && ps * 2 <= min_kb) ps *= 2;
+    if (2 * m_pairs * ps >= m_total * splits) {
+      pair = true;
+      splits = ps;
+      m_total = 2 * m_pairs;
+    }
+  }
   // Ring depths.  Per K block the tensor core needs ~560 cycles; a tile load takes ~2500 (L2) to ~4000 (HBM)
   // cycles, so both rings want several tiles in flight: equal depth first, what is left goes to W0.
   // INT8 storage: W0 tiles travel as 8 KB of codes; a ring of converted bf16 tiles (which also takes the U_B slabs,
   // loaded into it directly) sits between the converting warps and the tensor core.
-  const int mode = dec_mode(w0_dtype, tn);
-  if (mode < 0) return false;
   const int c_stages = mode == kModeInt8Smem ? kInt8ConvStages : mode >= kModeInt8Tmem ? kTmemAStages : 0;
   const int w_slot = dec_w_slot(mode);
-  const int xb = tn * 128;
-  const int budget = kDecSmemBudget - dec_smem_bytes(mode, 0, c_stages, 0, tn);
+  const int x_rows = pair ? tn / 2 : tn;  // token rows of an x tile per CTA
+  const int xb = x_rows * 128;
+  const int budget = kDecSmemBudget - dec_smem_bytes(mode, 0, c_stages, 0, 0);
   int x_stages = budget / (w_slot + xb);
   if (x_stages > kMaxXStages) x_stages = kMaxXStages;
   if (x_stages < 1) return false;
@@ -902,8 +978,9 @@ static bool plan_decode_block(int n, const int* d_in, const int* d_out, int w0_d
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
   if (w_stages < 1) return false;
   // the receive buffer of the cluster reduction overlays the rings
-  if (dec_ring_bytes(mode, w_stages, c_stages, x_stages, tn) < dec_recv_bytes(tn, splits)) return false;
+  if (dec_ring_bytes(mode, w_stages, c_stages, x_stages, x_rows) < dec_recv_bytes(tn, splits)) return false;
   if (c_stages_out) *c_stages_out = c_stages;
+  if (pair_out) *pair_out = pair;
   *splits_out = splits;
   *w_stages_out = w_stages;
   *x_stages_out = x_stages;
@@ -917,8 +994,9 @@ bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, in
   const bool int8 = w0_dtype == ESSA_W0_INT8_PERCHANNEL;
   int splits, w_stages, x_stages, m_tiles;
   const int di = d_in, dout = d_out;
-  if (!plan_decode_block(1, &di, &dout, w0_dtype, T, sm_count, &splits, &w_stages, &x_stages, &m_tiles)) return false;
-  out->block_m = DEC_M;
+  bool pair = false;
+  if (!plan_decode_block(1, &di, &dout, w0_dtype, T, sm_count, false, &splits, &w_stages, &x_stages, &m_tiles, nullptr, &pair)) return false;
+  out->block_m = pair ? 2 * DEC_M : DEC_M;  // rows of W0 per MMA: one CTA's tile, or a pair's two
   out->block_n = (int)((T + 15) / 16) * 16;
   out->block_k = DEC_K;
   out->stages = w_stages;
@@ -950,39 +1028,44 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     d_out[i] = items[i].a->d_out;
   }
   int splits, w_stages, x_stages, m_total, c_stages;
-  if (!plan_decode_block(n, d_in, d_out, w0_dtype, T, ctx->sm_count, &splits, &w_stages, &x_stages, &m_total, &c_stages)) {
+  bool pair = false;
+  if (!plan_decode_block(n, d_in, d_out, w0_dtype, T, ctx->sm_count, ctx->decode_pairs, &splits, &w_stages, &x_stages, &m_total,
+                         &c_stages, &pair)) {
     if (n > 1) return kBlockNotFused;
     return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: no decode schedule fits shared memory");
   }
   const int tn = (int)((T + 15) / 16) * 16;
   const int mode = dec_mode(w0_dtype, tn);
   if (mode < 0) return kBlockNotFused;
+  const int csize = pair ? 2 * splits : splits;  // CTAs per cluster
+  const int x_rows = pair ? tn / 2 : tn;         // token rows of an x tile per CTA
 
   // only CTAs of the first wave may be producers of u: ask the runtime how many clusters fit at once
-  static int resident_caches[64][4][9] = {};  // per device, kernel mode, cluster size
-  int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
-  const void* kernel = mode == kModeBf16      ? (const void*)essa_decode_kernel<kModeBf16>
-                       : mode == kModeInt8Smem ? (const void*)essa_decode_kernel<kModeInt8Smem>
-                       : mode == kModeInt8Tmem ? (const void*)essa_decode_kernel<kModeInt8Tmem>
-                                               : (const void*)essa_decode_kernel<kModeInt4Tmem>;
+  static int resident_caches[64][8][9] = {};  // per device, kernel instance, cluster size
+  const int inst = mode * 2 + (pair ? 1 : 0);
+  int* resident_cache = resident_caches[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][inst];
+  const void* kernel = mode == kModeBf16      ? (pair ? (const void*)essa_decode_kernel<kModeBf16, true> : (const void*)essa_decode_kernel<kModeBf16, false>)
+                       : mode == kModeInt8Smem ? (const void*)essa_decode_kernel<kModeInt8Smem, false>
+                       : mode == kModeInt8Tmem ? (pair ? (const void*)essa_decode_kernel<kModeInt8Tmem, true> : (const void*)essa_decode_kernel<kModeInt8Tmem, false>)
+                                               : (pair ? (const void*)essa_decode_kernel<kModeInt4Tmem, true> : (const void*)essa_decode_kernel<kModeInt4Tmem, false>);
   const int threads = mode != kModeBf16 ? kDecThreadsInt8 : kDecThreads;
   {
-    static bool attr_done[64][4] = {};  // the attribute is per device and kernel instance
-    bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][mode];
+    static bool attr_done[64][8] = {};  // the attribute is per device and kernel instance
+    bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0][inst];
     if (!done) {
       const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBudget);
       if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(essa_decode_kernel)");
       done = true;
     }
   }
-  if (resident_cache[splits] == 0) {
+  if (resident_cache[csize] == 0) {
     cudaLaunchConfig_t q{};
-    q.gridDim = dim3((unsigned)(148 * splits), 1, 1);
+    q.gridDim = dim3((unsigned)(148 * csize), 1, 1);
     q.blockDim = dim3((unsigned)threads, 1, 1);
     q.dynamicSmemBytes = (size_t)kDecSmemBudget;
     cudaLaunchAttribute qa[1];
     qa[0].id = cudaLaunchAttributeClusterDimension;
-    qa[0].val.clusterDim.x = (unsigned)splits;
+    qa[0].val.clusterDim.x = (unsigned)csize;
     qa[0].val.clusterDim.y = 1;
     qa[0].val.clusterDim.z = 1;
     q.attrs = qa;
@@ -992,9 +1075,9 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
       cudaGetLastError();
       n_clusters = 1;  // unknown: only the first cluster is certainly in the first wave
     }
-    resident_cache[splits] = n_clusters;
+    resident_cache[csize] = n_clusters;
   }
-  const int resident_ctas = resident_cache[splits] * splits;
+  const int resident_ctas = resident_cache[csize] * csize;
   const int main_ctas = m_total * splits;
   if (n > 1 && main_ctas > resident_ctas) return kBlockNotFused;
   // Launch a full wave: the CTAs beyond the W0-streaming ones only take finishing units of the rank path (groups
@@ -1025,11 +1108,12 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     DParams& p = blk.proj[i];
     p.T = (int)T;
     p.tn = tn;
-    p.xbox = tn;  // one box per tile (at most 256 rows)
+    p.xbox = x_rows;  // one box per tile (at most 256 rows)
     p.d_in = a->d_in;
     p.d_out = a->d_out;
     p.main_kb = a->d_in / DEC_K;
     p.m_tiles = (a->d_out + DEC_M - 1) / DEC_M;
+    if (pair) p.m_tiles = (p.m_tiles + 1) / 2 * 2;  // CTAs come in pairs; a tile past d_out loads zeros and stores nothing
     p.splits = splits;
     p.w_stages = w_stages;
     p.x_stages = x_stages;
@@ -1046,7 +1130,8 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
     {
       const int nkb_max = (p.main_kb + splits - 1) / splits;
       int owners = kMaxPSlices / splits;  // per split
-      if (owners > p.m_tiles) owners = p.m_tiles;
+      const int owner_ctas = pair ? p.m_tiles / 2 : p.m_tiles;  // per split: a pair's leader owns a slice
+      if (owners > owner_ctas) owners = owner_ctas;
       if (owners > 16) owners = 16;
       if (owners < 1) owners = 1;
       p.p_c = (nkb_max + owners - 1) / owners;
@@ -1110,7 +1195,7 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   }
   for (int i = n; i <= kMaxBlockProj; ++i) { blk.cta_begin[i] = cta; blk.unit_begin[i] = unit; }
 
-  const int smem_bytes = dec_smem_bytes(mode, w_stages, c_stages, x_stages, tn);
+  const int smem_bytes = dec_smem_bytes(mode, w_stages, c_stages, x_stages, x_rows);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid_total, 1, 1);
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
@@ -1118,17 +1203,15 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)splits;
+  attr[0].val.clusterDim.x = (unsigned)csize;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see grid_dep_wait in the kernel
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = mode == kModeBf16      ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeBf16>, maps, blk)
-                        : mode == kModeInt8Smem ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Smem>, maps, blk)
-                        : mode == kModeInt8Tmem ? cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt8Tmem>, maps, blk)
-                                                : cudaLaunchKernelEx(&cfg, essa_decode_kernel<kModeInt4Tmem>, maps, blk);
+  void* kargs[] = {(void*)&maps, (void*)&blk};
+  const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel, kargs);
   if (e != cudaSuccess) return check_cuda(ctx, e, "essa_decode_kernel launch");
   ctx->launches += 1;
   ctx->dec_set_issued[set & 1] += (uint32_t)grid_total;

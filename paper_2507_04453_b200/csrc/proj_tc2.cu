@@ -31,7 +31,7 @@ constexpr int P2_M = 128;        // token rows per CTA (256 per pair)
 constexpr int P2_NH = 128;       // W0 rows per CTA (256 channels per pair)
 constexpr int P2_N = 256;
 constexpr int P2_K = 64;
-constexpr int P2_THREADS = 192;
+constexpr int P2_THREADS = 224;  // warps 0..5 as below, warp 6 = second TMA producer (the W0 / U_B halves)
 constexpr int P2_A_BYTES = P2_M * P2_K * 2, P2_B_BYTES = P2_NH * P2_K * 2, P2_STAGE = P2_A_BYTES + P2_B_BYTES;  // 32 KB
 constexpr int P2_STAGES = 6;
 __host__ __device__ constexpr int p2_stages(int rp) { return rp > 48 ? 5 : P2_STAGES; }
@@ -127,8 +127,13 @@ essa_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer (each CTA: its halves)
+  if (warp == 0 || warp == 6) {
+    // ------------------------------------------------------------------ TMA producers (each CTA: its halves).  Warp 0
+    // brings in the activation rows (and the V_A^T rows of a fused first-column tile), warp 6 the W0 / U_B rows: a
+    // thread that has just issued a 16 KB box does not get back to the next free slot in time to keep both operand
+    // streams full (measured on the decode kernel: one issuing thread was 1.4 times slower per K block than two).
+    // Both walk the same stages and wait for the same `empty` phases; the leader's warp 0 posts the byte count.
+    const bool prod_a = warp == 0;
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -141,7 +146,7 @@ essa_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int row_a = m_tile * 2 * P2_M + (int)rank * P2_M;     // tokens of this CTA
         const int row_b = n_tile * P2_N + (int)rank * P2_NH;        // channels of this CTA
         for (int kb = 0; kb < total_kb; ++kb) {
-          if (RP > 0 && kb == p.main_kb) {
+          if (RP > 0 && kb == p.main_kb && prod_a) {
             // the u slab of this CTA's token rows: published by the first-column tile of this token tile
             const uint32_t* flag = p.u_ready + 2 * m_tile + (int)rank;
             const long long t0 = clock64();
@@ -158,15 +163,19 @@ essa_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, p.status)) { ok = false; break; }
           const bool with_v = down && kb < p.main_kb;
-          if (leader) mbar_expect_tx(bar_full + 8 * stage, 2u * (P2_STAGE + (with_v ? V_BYTES : 0)));  // the bytes of both CTAs
+          if (leader && prod_a) mbar_expect_tx(bar_full + 8 * stage, 2u * (P2_STAGE + (with_v ? V_BYTES : 0)));  // the bytes of both CTAs
           const uint32_t fb = full_leader + 8 * stage;
           const uint32_t da = smem_u32(smem_a + stage * P2_A_BYTES), db = smem_u32(smem_b + stage * P2_B_BYTES);
           if (kb < p.main_kb) {
-            tma_load_2d_pair(da, &tmA, kb * P2_K, row_a, fb);
-            tma_load_2d_pair(db, &tmB, kb * P2_K, row_b, fb);
-            if (with_v) tma_load_2d_pair(smem_u32(smem_v + stage * V_BYTES), &tmV, kb * P2_K, (int)rank * (RP / 2), fb);
-          } else {
+            if (prod_a) {
+              tma_load_2d_pair(da, &tmA, kb * P2_K, row_a, fb);
+              if (with_v) tma_load_2d_pair(smem_u32(smem_v + stage * V_BYTES), &tmV, kb * P2_K, (int)rank * (RP / 2), fb);
+            } else {
+              tma_load_2d_pair(db, &tmB, kb * P2_K, row_b, fb);
+            }
+          } else if (prod_a) {
             tma_load_2d_pair(da, &tmA2, 0, row_a, fb);
+          } else {
             tma_load_2d_pair(db, (kb - p.main_kb) == 0 ? &tmB2a : &tmB2b, 0, row_b, fb);
           }
           ++issued;

@@ -128,3 +128,19 @@ def test_quantised_storage_token_counts_in_tensor_memory_mode(torch, ctx, w0, T)
     for i in (0, 1):
         y, _ = _run(torch, ctx, case, i, _offsets(rng, cfg.P, T), T, TOL_INT8)
     case.close()
+
+
+@pytest.mark.parametrize("w0,T", [("bf16", 256), ("bf16", 96), ("int8", 128), ("int4", 64)])
+def test_cta_pair_variant(torch, w0, T):
+    """ESSA_OPT_DECODE_PAIRS: two W0 row tiles per MMA of 256 rows (cta_group::2), each CTA loading half of the token
+    rows; an odd number of row tiles (d_kv = 200 -> 2 tiles, d_model 640 -> 5) pairs the last tile with an empty one."""
+    c = binding.Context(0)
+    c.set_option(binding.ESSA_OPT_DECODE_PAIRS, 1)
+    cfg = wl.scaled_config({"int8": "5a", "int4": "6a", "bf16": "3"}[w0], d_model=640, d_kv=200, rank=24, P=5, seg_len=1)
+    case = Case(torch, c, cfg)
+    rng = np.random.default_rng(T)
+    for i in (0, 1):
+        _run(torch, c, case, i, _offsets(rng, cfg.P, T), T, TOL_BF16 if w0 == "bf16" else TOL_INT8)
+    assert c.get_status() == 0
+    case.close()
+    c.close()
