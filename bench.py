@@ -290,6 +290,9 @@ def measure_config(key, cfg, args, env):
         ctx.set_option(binding.ESSA_OPT_PAIR_TILES, args.pair_tiles)
     if args.fuse_down >= 0:
         ctx.set_option(binding.ESSA_OPT_FUSE_DOWN, args.fuse_down)
+    for item in args.set_option:
+        opt, val = item.split("=")
+        ctx.set_option(int(opt), int(val))
     adapters = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
     offsets = wl.make_segments(cfg)
     T = int(offsets[-1])
@@ -648,6 +651,8 @@ def main():
     ap.add_argument("--fuse-down", type=int, default=-1, help="override ESSA_OPT_FUSE_DOWN (0 / 1)")
     ap.add_argument("--single-calls", action="store_true",
                     help="decode configurations: one essa_apply_projection per projection instead of one essa_apply_block")
+    ap.add_argument("--set-option", action="append", default=[], metavar="ID=VALUE",
+                    help="essa_set_option(ID, VALUE) on every context (scheduling experiments), e.g. 6=0")
     ap.add_argument("--no-layers", action="store_true", help="skip the multi-layer (essa_apply_layers) measurement of decode configurations")
     ap.add_argument("--separate-calls", action="store_true",
                     help="decode configurations: essa_sample_population then essa_apply_block instead of the fused call")

@@ -107,6 +107,10 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   K block and the launch measured 15 - 50 % SLOWER on B200 (config 3: 37 -> 44 us per step, config 5a: 129 -> 197 us),
  *   so it is off unless asked for. */
 #define ESSA_OPT_DECODE_PAIRS 5
+/*   ESSA_OPT_DECODE_DOWN_CTAS (0 / 1, default 1): when a decode launch has at least four thread blocks of its wave left
+ *   over beyond the ones that stream W0, those compute the down-projection V_A^T x for the whole launch (x and V_A^T
+ *   come from L2) instead of the first row tiles carrying slices of it on their K loops.  0 restores the slices. */
+#define ESSA_OPT_DECODE_DOWN_CTAS 6
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

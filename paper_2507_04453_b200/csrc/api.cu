@@ -261,6 +261,7 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
       return ESSA_OK;
     case ESSA_OPT_DEBUG_STALL_RANK_ROWS: ctx->debug_stall_rank_rows = value != 0; return ESSA_OK;
     case ESSA_OPT_DECODE_PAIRS: ctx->decode_pairs = value != 0; return ESSA_OK;
+    case ESSA_OPT_DECODE_DOWN_CTAS: ctx->down_ctas = value != 0; return ESSA_OK;
     default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
   }
 }

@@ -36,6 +36,7 @@ struct essa_ctx {
   int wait_limit_mcycles = 3000;  // ESSA_OPT_WAIT_LIMIT_MCYCLES
   bool debug_stall_rank_rows = false;  // ESSA_OPT_DEBUG_STALL_RANK_ROWS
   bool decode_pairs = false;  // ESSA_OPT_DECODE_PAIRS
+  bool down_ctas = true;      // ESSA_OPT_DECODE_DOWN_CTAS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
   int fuse_down = 0;            // ... which also compute the down-projection (no rank-down launch): 0 never (default),
                                 // 1 in the token range where it measured faster, 2 whenever pair tiles are used

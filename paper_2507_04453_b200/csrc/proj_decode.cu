@@ -116,6 +116,15 @@ struct DBlock {
   int cta_begin[kMaxBlockProj + 1];   // multiples of the cluster size; cta_begin[n_proj] = W0-streaming CTAs
   int unit_begin[kMaxBlockProj + 1];  // rank-path units (token group x K slice) per projection
   int rank_ctas;                      // CTAs 0 .. rank_ctas-1 (all in the first wave) take units w, w + rank_ctas, ...
+  // Down-projection CTAs.  When the wave has CTAs to spare beyond the W0-streaming ones (n_down > 0: CTAs
+  // cta_begin[n_proj] .. + n_down - 1), THEY compute p = V_A^T x: CTA c of them takes K blocks
+  // [c KB / n_down, (c + 1) KB / n_down) of every projection (x and V_A^T tiles from L2, one accumulator per
+  // projection, delivered to slot c) and the W0-streaming CTAs carry no slices at all.  Otherwise (n_down = 0)
+  // the slices ride on the K loops of the first row tiles as described at the top of the file.  (Measured at the
+  // 7B decode shape: the 512-channel k / v projections have four row tiles per K split, so their CTAs carried
+  // seven-block slices, finished 4 k cycles after everybody else and delivered so late that the up-projection of
+  // every projection waited for them.)
+  int n_down;
   // Fused draw + block call: the singular-value table is being written by the population-draw kernel launched just
   // before this one; that kernel counts its finished blocks in *sigma_ready.  The launch then does not wait for the
   // draw as a whole (it streams W0 and x beside it) and only the rank path waits for the count (bounded).
@@ -157,7 +166,7 @@ __host__ __device__ inline int dec_recv_bytes(int tn, int splits) {
 // row of the core matrix, u_j = sB_k,j v_j, stored as bf16; then the group's tokens are added to the published-row
 // count.  Everything that does not depend on the slices (candidate lookup, singular values, the row of M) is
 // requested before the wait for them.  Returns false when the wait gave up.
-__device__ __forceinline__ bool finish_unit(const DParams& p, int grp, float* qbuf /*[kFinishTokens][64]*/, volatile int* flag,
+__device__ __forceinline__ bool finish_unit(const DParams& p, int n_down, int grp, float* qbuf /*[kFinishTokens][64]*/, volatile int* flag,
                                             volatile int* abort_flag, int etid) {
   constexpr int TPT = kFinishTokens / 2;  // tokens per thread
   const int j = etid & 63, h = etid >> 6;
@@ -201,22 +210,43 @@ __device__ __forceinline__ bool finish_unit(const DParams& p, int grp, float* qb
     float pj[TPT];
 #pragma unroll
     for (int g = 0; g < TPT; ++g) pj[g] = 0.f;
-    if (j < p.r) {
-      // slot sp * p_per_split + sl exists when slice sl of split sp does; eight loads in flight at a time
+    // With a padded rank of 16 or 32 only a quarter or half of the 64 rank lanes carry a coordinate: the lanes
+    // beyond help with the loads.  Lane j = G jj-lanes: group sg = j / RPp sums the slots sg, sg + G, ... of
+    // coordinate jj = j % RPp (eight 16-byte loads in flight), the groups' sums meet in shared memory and are
+    // added in group order (still one fixed order: results stay bit-identical run to run).
+    const int RPp = p.r_pad <= 16 ? 16 : p.r_pad <= 32 ? 32 : 64;
+    const int G = 64 / RPp, jj = j % RPp, sg = j / RPp;
+    float4* pbuf = reinterpret_cast<float4*>(qbuf + kFinishTokens * kRankPadMax);  // [2][G][RPp] float4, 2 KB
+    if (jj < p.r) {
+      // slot sp * p_per_split + sl exists when slice sl of split sp does
       const int kbase = p.main_kb / p.splits, krem = p.main_kb % p.splits;
-      const int n_flat = p.splits * p.p_per_split;
-      const float* base = p.p_part + (size_t)j * kDecodeMaxTokens + t0 + TPT * h;
-      for (int i0 = 0; i0 < n_flat; i0 += 8) {
+      const int n_flat = n_down > 0 ? n_down : p.splits * p.p_per_split;
+      const float* base = p.p_part + (size_t)jj * kDecodeMaxTokens + t0 + TPT * h;
+      for (int i0 = sg; i0 < n_flat; i0 += 8 * G) {
         float4 v4[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-          const int idx = i0 + u;
+          const int idx = i0 + u * G;
           const int sp = idx / p.p_per_split, sl = idx - sp * p.p_per_split;
-          const bool valid = idx < n_flat && sl * p.p_c < kbase + (sp < krem ? 1 : 0);
+          // (down-projection CTAs: slot idx exists when CTA idx got at least one K block of this projection)
+          const bool valid = idx < n_flat && (n_down > 0 ? ((long long)(idx + 1) * p.main_kb) / n_down > ((long long)idx * p.main_kb) / n_down
+                                                         : sl * p.p_c < kbase + (sp < krem ? 1 : 0));
           v4[u] = valid ? ld_cg_f32x4(base + (size_t)idx * kRankPadMax * kDecodeMaxTokens) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) { pj[0] += v4[u].x; pj[1] += v4[u].y; pj[2] += v4[u].z; pj[3] += v4[u].w; }
+      }
+    }
+    if (G > 1) {
+      pbuf[(h * G + sg) * RPp + jj] = make_float4(pj[0], pj[1], pj[2], pj[3]);
+      epi_bar_sync();
+      if (sg == 0) {
+        for (int q = 1; q < G; ++q) {
+          const float4 o = pbuf[(h * G + q) * RPp + jj];
+          pj[0] += o.x; pj[1] += o.y; pj[2] += o.z; pj[3] += o.w;
+        }
+      } else {
+        pj[0] = pj[1] = pj[2] = pj[3] = 0.f;  // lanes beyond the padded rank carry no coordinate
       }
     }
 #pragma unroll
@@ -328,7 +358,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // dead once every MMA of the cluster has completed
   float* recv = reinterpret_cast<float*>(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2 + 2 * kVatStages + 1 + kUbSlots));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * kMaxWStages + 2 * kMaxXStages + 2 * kMaxCStages + 2 + 2 * kVatStages + 1 + kUbSlots + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* qbuf = reinterpret_cast<float*>(aux + 1024);      // [kFinishTokens][64]
 
@@ -338,6 +368,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   const uint32_t bar_d = bar_cempty + 8 * kMaxCStages, bar_drain = bar_d + 8;
   const uint32_t bar_vfull = bar_drain + 8, bar_vempty = bar_vfull + 8 * kVatStages, bar_p = bar_vempty + 8 * kVatStages;
   const uint32_t bar_ub = bar_p + 8;  // kModeInt8Tmem: one per U_B slab
+  const uint32_t bar_pr = bar_ub + 8 * kUbSlots, bar_pfree = bar_pr + 16;  // down-projection CTAs: accumulator ready / read out (two each)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int crank = (int)cluster_ctarank();
@@ -363,7 +394,9 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   // The K loop starts at this CTA's slice of the down-projection and wraps around: item i is local K block
   // (r0 + i) mod nkb, and the first c_own items also feed the second accumulator.
   const int r0 = nkb > 0 ? (owner_idx * p.p_c) % nkb : 0;  // (the same in both CTAs of a pair)
-  const int c_own = (is_main && leader && owner_idx * p.p_c < nkb) ? min(p.p_c, nkb - owner_idx * p.p_c) : 0;
+  const int c_own = (blk.n_down == 0 && is_main && leader && owner_idx * p.p_c < nkb) ? min(p.p_c, nkb - owner_idx * p.p_c) : 0;
+  const int dcta = (int)blockIdx.x - blk.cta_begin[blk.n_proj];  // index among the down-projection CTAs
+  const bool is_down = !is_main && dcta < blk.n_down;
   auto kcol = [&](int i) { const int l = r0 + i; return (kb0 + (l >= nkb ? l - nkb : l)) * DEC_K; };
 
   // a copy whose completion the pair's MMA waits for: counted on the leader's barrier
@@ -431,20 +464,21 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     mbar_init(bar_drain, 1);
     for (int s = 0; s < kVatStages; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 1); }
     mbar_init(bar_p, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_pr + 8 * b, 1); mbar_init(bar_pfree + 8 * b, 1); }
     *abort_flag = 0;
     *reinterpret_cast<volatile int*>(tmem_slot + 3) = 0;  // conversion ticket
     *reinterpret_cast<volatile int*>(tmem_slot + 4) = 0;  // ... and whose turn it is to claim a slot
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int i = 0; i < first_w; ++i) load_w(i);  // the frozen weights depend on nothing: stream at once
   }
-  if (warp == 1 && is_main) {
+  if (warp == 1 && (is_main || is_down)) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   if (PAIR) cluster_sync_all(); else __syncthreads();  // PAIR: both CTAs' barriers exist before either uses the other's
   tc_fence_after();
-  const uint32_t tmem_base = is_main ? *tmem_slot : 0u;  // PAIR: the same address in both CTAs (an SM's only allocation)
+  const uint32_t tmem_base = (is_main || is_down) ? *tmem_slot : 0u;  // PAIR: the same address in both CTAs (an SM's only allocation)
   // Everything up to here (barriers, TMEM, the first tiles of the frozen W0) depends on no earlier kernel and, with
   // a programmatic dependent launch, overlaps the kernel before this one in the stream (typically the population
   // draw); x, the singular values, the scratch buffers and y are touched only after this point.  In a fused draw +
@@ -489,7 +523,90 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000LL) {}
   };
-  if (warp == 0) {
+  // ------------------------------------------------------------------ down-projection CTA (see DBlock::n_down)
+  // Its units are (projection, K block) in projection order; unit u uses slot u mod depth of the x ring (x tiles of
+  // whichever projection, tn rows each) and of a ring of eight 8 KB V_A^T slots at the start of shared memory (this
+  // CTA has no W0 ring).  Projection q (counting the ones it has K blocks of) accumulates in TMEM columns 256 (q & 1).
+  constexpr int RV = 8, RV_SLOT = 8192;
+  auto down_range = [&](int pj, int& a, int& b) {
+    const int KB = blk.proj[pj].main_kb;
+    a = (int)(((long long)dcta * KB) / blk.n_down);
+    b = (int)(((long long)(dcta + 1) * KB) / blk.n_down);
+  };
+  if (is_down && warp == 0) {
+    if (lane == 0) {
+      int u = 0;
+      bool ok = true;
+      for (int pj = 0; ok && pj < blk.n_proj; ++pj) {
+        int a, b;
+        down_range(pj, a, b);
+        for (int kb = a; ok && kb < b; ++kb, ++u) {
+          const int sv = u % RV;
+          if (u >= RV) ok = mbar_wait(bar_vempty + 8 * sv, (uint32_t)(((u / RV) & 1) ^ 1), abort_flag, p.status);
+          if (!ok) break;
+          mbar_expect_tx(bar_vfull + 8 * sv, (uint32_t)(blk.proj[pj].r_pad * 128));
+          tma_load_2d(smem_u32(smem + sv * RV_SLOT), &maps.tm[pj][5], kb * DEC_K, 0, bar_vfull + 8 * sv);
+        }
+      }
+      if (!ok || *abort_flag) drain(u, RV, bar_vfull);
+    }
+  } else if (is_down && warp == kXWarp) {
+    if (lane == 0) {
+      int u = 0;
+      bool ok = true;
+      if (blk.layer_mode == 2) {
+        ok = wait_layers_flag();
+        if (ok) fence_proxy_async_global();
+      }
+      for (int pj = 0; ok && pj < blk.n_proj; ++pj) {
+        int a, b;
+        down_range(pj, a, b);
+        for (int kb = a; ok && kb < b; ++kb, ++u) {
+          const int sx = u % SX;
+          if (u >= SX) ok = mbar_wait(bar_xempty + 8 * sx, (uint32_t)(((u / SX) & 1) ^ 1), abort_flag, p.status);
+          if (!ok) break;
+          mbar_expect_tx(bar_xfull + 8 * sx, (uint32_t)x_bytes);
+          tma_load_2d(smem_u32(smem_x + sx * x_bytes), &maps.tm[pj][1], kb * DEC_K, 0, bar_xfull + 8 * sx);
+        }
+      }
+      if (!ok || *abort_flag) drain(u, SX, bar_xfull);
+    }
+  } else if (is_down && warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(DEC_M, p.tn);
+      int u = 0, q = 0;
+      bool ok = true;
+      for (int pj = 0; ok && pj < blk.n_proj; ++pj) {
+        int a, b;
+        down_range(pj, a, b);
+        if (b <= a) continue;
+        const int acc = q & 1;
+        // the accumulator was last used two projections ago: its slot must have been read out
+        if (q >= 2 && !mbar_wait(bar_pfree + 8 * acc, (uint32_t)(((q >> 1) - 1) & 1), abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = a; kb < b; ++kb, ++u) {
+          const int sx = u % SX, sv = u % RV;
+          if (!mbar_wait(bar_xfull + 8 * sx, (uint32_t)((u / SX) & 1), abort_flag, p.status) ||
+              !mbar_wait(bar_vfull + 8 * sv, (uint32_t)((u / RV) & 1), abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t dv = make_smem_desc(smem_u32(smem + sv * RV_SLOT));
+          const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
+#pragma unroll
+          for (int k = 0; k < DEC_K / 16; ++k) umma_bf16(tmem_base + (uint32_t)(acc * 256), dv + 2 * k, dx + 2 * k, idesc, (kb > a || k > 0) ? 1u : 0u);
+          umma_commit(bar_xempty + 8 * sx);
+          umma_commit(bar_vempty + 8 * sv);
+        }
+        if (!ok) break;
+        umma_commit(bar_pr + 8 * acc);
+        ++q;
+      }
+      if (!ok) {
+        umma_commit(bar_drain);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < kWaitLimitCycles) {}
+      }
+    }
+  } else if (warp == 0) {
     if (lane == 0) {
       int iw = first_w, iv = 0;
       bool ok = true;
@@ -776,6 +893,44 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   if (epi) {
     const int etid = threadIdx.x - 64;
     volatile int* flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+    if (is_down) {
+      int q = 0;
+      bool fine = true;
+      for (int pj = 0; fine && pj < blk.n_proj; ++pj) {
+        int a, b;
+        down_range(pj, a, b);
+        if (b <= a) continue;
+        const DParams& pp = blk.proj[pj];
+        const int acc = q & 1;
+        int have = 0;
+        if (lane == 0) have = mbar_wait(bar_pr + 8 * acc, (uint32_t)((q >> 1) & 1), abort_flag, p.status) ? 1 : 0;
+        have = __shfl_sync(0xffffffffu, have, 0);
+        if (!have) { fine = false; break; }
+        while (!mbar_try_wait(bar_pr + 8 * acc, (uint32_t)((q >> 1) & 1))) {}  // complete: acquire for every lane
+        tc_fence_after();
+        if (quad * 32 < pp.r_pad) {
+          float* slot = pp.p_part + (size_t)dcta * kDecodeMaxTokens * kRankPadMax;
+#pragma unroll 1
+          for (int c = 0; c < pp.tn / 16; ++c) {
+            float v[16];
+            tmem_ld16(t_lane + (uint32_t)(acc * 256) + c * 16, v);
+            if (row < pp.r_pad) {
+              float4* dst = reinterpret_cast<float4*>(slot + (size_t)row * kDecodeMaxTokens + c * 16);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+          }
+        }
+        tc_fence_before();
+        __threadfence();
+        epi_bar_sync();
+        if (etid == 0) {
+          red_release_add_u32(pp.p_count, 1u);
+          mbar_arrive(bar_pfree + 8 * acc);
+        }
+        ++q;
+      }
+    }
     if (c_own > 0) {
       // this CTA's slice of the down-projection: accumulator rows (rank index) x columns (token) -> its slot
       int have = 0;
@@ -833,7 +988,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       for (int unit = blockIdx.x; fine && unit < blk.unit_begin[blk.n_proj]; unit += blk.rank_ctas) {
         int pj = 0;
         while (pj + 1 < blk.n_proj && unit >= blk.unit_begin[pj + 1]) ++pj;
-        fine = finish_unit(blk.proj[pj], unit - blk.unit_begin[pj], qbuf, flag, abort_flag, etid);
+        fine = finish_unit(blk.proj[pj], blk.n_down, unit - blk.unit_begin[pj], qbuf, flag, abort_flag, etid);
       }
     }
     got = is_main ? 1 : 0;
@@ -893,7 +1048,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     }
   }
   __syncthreads();
-  if (warp == 1 && is_main) {
+  if (warp == 1 && (is_main || is_down)) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
@@ -1099,6 +1254,13 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
   blk.other_wait_target = ctx->dec_set_issued[(set & 1) ^ 1];
   const int s0 = (set & 1) * kMaxBlockProj;  // first scratch slot of this launch
   blk.rank_ctas = grid_total < resident_ctas ? grid_total : resident_ctas;
+  // CTAs of the wave beyond the W0-streaming ones take over the down-projection when there are at least four of them
+  // (no CTA pairs: their x tiles are halves), at most one slot each, and their V_A^T ring fits below the x ring.
+  {
+    const int spare = grid_total - main_ctas;
+    const int below_x = VAT_RING_BYTES + w_stages * dec_w_slot(mode) + (mode == kModeInt8Smem ? c_stages : mode >= kModeInt8Tmem ? kUbSlots : 0) * W_TILE_BYTES;
+    blk.n_down = (!pair && spare >= 4 && below_x >= 8 * 8192 + W_TILE_BYTES && ctx->down_ctas) ? (spare < kMaxPSlices ? spare : kMaxPSlices) : 0;
+  }
   int cta = 0, unit = 0;
   // The counters' next values are committed to the context only once the launch has been accepted: after a failed
   // call the device never reaches them, and a later call must not wait for rows nobody publishes.
@@ -1137,6 +1299,10 @@ int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_
       p.p_c = (nkb_max + owners - 1) / owners;
       p.p_per_split = (nkb_max + p.p_c - 1) / p.p_c;
       int delivered = 0;
+      if (blk.n_down > 0) {  // one slot per down-projection CTA that gets a K block of this projection
+        for (int c = 0; c < blk.n_down; ++c)
+          delivered += ((long long)(c + 1) * p.main_kb) / blk.n_down > ((long long)c * p.main_kb) / blk.n_down ? 1 : 0;
+      } else
       for (int sp = 0; sp < splits; ++sp) {
         const int nkb_s = p.main_kb / splits + (sp < p.main_kb % splits ? 1 : 0);
         delivered += (nkb_s + p.p_c - 1) / p.p_c;

@@ -144,3 +144,19 @@ def test_cta_pair_variant(torch, w0, T):
     assert c.get_status() == 0
     case.close()
     c.close()
+
+
+@pytest.mark.parametrize("w0,T,r", [("bf16", 256, 16), ("bf16", 77, 33), ("int8", 128, 64), ("int8", 200, 24), ("int4", 100, 16)])
+def test_slices_on_the_row_tiles_when_no_down_projection_ctas(torch, w0, T, r):
+    """ESSA_OPT_DECODE_DOWN_CTAS = 0: the down-projection rides as slices on the K loops of the first row tiles (the
+    scheme a launch without spare thread blocks uses), same results."""
+    c = binding.Context(0)
+    c.set_option(binding.ESSA_OPT_DECODE_DOWN_CTAS, 0)
+    cfg = wl.scaled_config({"int8": "5a", "int4": "6a", "bf16": "3"}[w0], d_model=1024, d_kv=200, rank=r, P=6, seg_len=1)
+    case = Case(torch, c, cfg)
+    rng = np.random.default_rng(T + r)
+    for i in (0, 1):
+        _run(torch, c, case, i, _offsets(rng, cfg.P, T), T, TOL_BF16 if w0 == "bf16" else TOL_INT8)
+    assert c.get_status() == 0
+    case.close()
+    c.close()
