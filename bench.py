@@ -325,14 +325,16 @@ def measure_config(key, cfg, args, env):
     step_no = [0]
     cols = [cfg.sigma_cols(i) for i in range(len(handles))]
     decode = T <= 256  # one-launch decode schedule (essa_plan.decode)
-    block_call = decode and len(handles) > 1 and not args.single_calls
+    # the block's projections share tokens, segments and the table -> one essa_apply_block call (decode sizes: one launch;
+    # prefill sizes: the rank-down launches, then one launch for the base + up step of all projections)
+    block_call = len(handles) > 1 and not args.single_calls
 
     # Decode steps are tens of microseconds: their two calls are marshalled once (binding.PreparedSample /
     # PreparedBlock: the same C entry points, argument tuples built ahead of time) so that the host keeps ahead.
     stream_handle = stream.cuda_stream
     prep_sample = ctx.prepare_sample(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, sigma, k_begin)
     prep_blocks = [ctx.prepare_block(hs, xs, d_off, sigma, cols, ys) for hs in handle_sets] if block_call else None
-    fused_call = block_call and not args.separate_calls
+    fused_call = block_call and decode and not args.separate_calls  # (at prefill sizes the draw is a separate call)
     prep_fused = [ctx.prepare_sample_block(d_mean, cma.step, d_B, d_D, cma.seed, cfg.P, sigma, hs, xs, d_off, cols, ys, k_begin)
                   for hs in handle_sets] if fused_call else None
 
@@ -437,7 +439,7 @@ def measure_config(key, cfg, args, env):
     # ---- multi-layer call (decode configurations): L layers' blocks in ONE essa_apply_layers call, each layer with its
     # own device copy of the adapters (so every layer streams its W0 from HBM); per-layer time beside the single block's
     layers_rec = None
-    if block_call and world == 1 and not args.no_layers:
+    if block_call and decode and world == 1 and not args.no_layers:
         L = {"3": 28, "5a": 80, "6a": 80}.get(key, 8)  # decoder layers of the backbone the shapes come from
         adapters_again = [wl.make_adapter(cfg, i) for i in range(len(cfg.projections))]
         while len(handle_sets) < L:
@@ -521,7 +523,8 @@ def measure_config(key, cfg, args, env):
     nominal = block_roofline(cfg, T, NOMINAL_PEAKS["bf16_tflops"], NOMINAL_PEAKS["hbm_gbs"])
     calls = max(prof["calls"], 1)
     main_s = prof["base_up_ms"] * 1e-3 / calls  # average launch duration
-    per_call = 1 if block_call else len(handles)  # a block call is one launch for all projections
+    # timed launches of the dominant kernel per step: 1 when a block call covers all projections with one launch
+    per_call = max(1, round(prof["calls"] / steps))
     if model["bound"] == "tensor":
         per_launch = model["flops_main"] / per_call
         achieved, peak, peak_nom, unit = per_launch / main_s / 1e12, peaks[tf_key], NOMINAL_PEAKS["bf16_tflops"], "TFLOP/s"
@@ -536,7 +539,8 @@ def measure_config(key, cfg, args, env):
     if decode:
         kernel = "essa_decode_kernel (one launch for the block's projections)" if block_call else "essa_decode_kernel (whole call)"
     else:
-        kernel = "essa_tc2_kernel / essa_tc_kernel (base contraction + up-projection)"
+        kernel = ("essa_tcw_kernel (base contraction + up-projection of the block's projections in one launch)" if per_call == 1 and block_call
+                  else "essa_tcw_kernel / essa_tc2_kernel / essa_tc_kernel (base contraction + up-projection)")
     roofline = {"bound": model["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
                 "traffic": traffic, "kernel": kernel, "peak_kind": peak_kind, "peak_source": f"{peak_src} ({peak_kind})",
                 "peak_nominal": peak_nom, "frac_of_nominal": achieved / peak_nom,

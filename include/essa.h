@@ -111,6 +111,11 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   over beyond the ones that stream W0, those compute the down-projection V_A^T x for the whole launch (x and V_A^T
  *   come from L2) instead of the first row tiles carrying slices of it on their K loops.  0 restores the slices. */
 #define ESSA_OPT_DECODE_DOWN_CTAS 6
+/*   ESSA_OPT_WIDE_TILES (0 / 1 / 2, default 1): prefill base + up launches use 512-token x 256-channel CTA-pair tiles
+ *   (two accumulators per pair; the tensor cores run at their rate on that loop) where the planner's estimate puts
+ *   them ahead of the 256 x 256 pair tiles (1), wherever the pair tiles would run (2), or never (0).  Both tile
+ *   shapes add the K blocks in the same order in fp32. */
+#define ESSA_OPT_WIDE_TILES 7
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

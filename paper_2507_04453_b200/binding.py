@@ -32,6 +32,7 @@ ESSA_OPT_WAIT_LIMIT_MCYCLES = 3
 ESSA_OPT_DEBUG_STALL_RANK_ROWS = 4
 ESSA_OPT_DECODE_PAIRS = 5
 ESSA_OPT_DECODE_DOWN_CTAS = 6
+ESSA_OPT_WIDE_TILES = 7
 
 EXPORTED_SYMBOLS = (
     "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",

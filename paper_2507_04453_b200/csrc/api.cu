@@ -262,6 +262,10 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
     case ESSA_OPT_DEBUG_STALL_RANK_ROWS: ctx->debug_stall_rank_rows = value != 0; return ESSA_OK;
     case ESSA_OPT_DECODE_PAIRS: ctx->decode_pairs = value != 0; return ESSA_OK;
     case ESSA_OPT_DECODE_DOWN_CTAS: ctx->down_ctas = value != 0; return ESSA_OK;
+    case ESSA_OPT_WIDE_TILES:
+      if (value < 0 || value > 2) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_WIDE_TILES takes 0, 1 or 2");
+      ctx->wide_tiles = value;
+      return ESSA_OK;
     default: return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: unknown option");
   }
 }
@@ -274,7 +278,8 @@ int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches) {
 
 int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_t max_d_out) {
   if (!ctx || max_tokens < 0 || max_d_in < 0 || max_d_out < 0) return ESSA_ERR_INVALID_ARG;
-  int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)max_tokens * kRankPadMax * 2, false, nullptr);
+  // one rank-path vector per projection of a block (a prefill-sized block call keeps all of them at once)
+  int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)ESSA_MAX_BLOCK_ITEMS * ((size_t)max_tokens * kRankPadMax * 2 + 256), false, nullptr);
   if (st != ESSA_OK) return st;
   // split-K is only used while there are fewer tiles than SMs: at most sm_count tiles of 128 x 256 fp32
   st = ensure_scratch(ctx, ctx->splitk_ws, (size_t)ctx->sm_count * 128 * 256 * 4, true, nullptr);
@@ -496,6 +501,14 @@ static int32_t apply_block_impl(essa_ctx* ctx, const essa_block_item* items, int
       if (ev) { cudaEventRecord(ev[2], stream); ++ctx->prof_calls; }
       return st;
     }
+  }
+  {
+    BlockItem bi[ESSA_MAX_BLOCK_ITEMS];
+    for (int32_t i = 0; i < n_items; ++i)
+      bi[i] = BlockItem{items[i].adapter, static_cast<const __nv_bfloat16*>(items[i].x), items[i].sA_col, items[i].sB_col,
+                        static_cast<__nv_bfloat16*>(items[i].y)};
+    const int32_t st = launch_block_prefill(ctx, bi, n_items, T, seg, P, sigma, ld_sigma, stream);
+    if (st != kBlockNotFused) return st;
   }
   for (int32_t i = 0; i < n_items; ++i) {
     ProjArgs g{static_cast<const __nv_bfloat16*>(items[i].x), T, seg, P, sigma, ld_sigma, items[i].sA_col, items[i].sB_col,

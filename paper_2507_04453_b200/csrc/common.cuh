@@ -38,6 +38,7 @@ struct essa_ctx {
   bool decode_pairs = false;  // ESSA_OPT_DECODE_PAIRS
   bool down_ctas = true;      // ESSA_OPT_DECODE_DOWN_CTAS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
+  int wide_tiles = 1;           // ... on 512 x 256 pair tiles: 0 never, 1 where the planner's estimate favours them, 2 always
   int fuse_down = 0;            // ... which also compute the down-projection (no rank-down launch): 0 never (default),
                                 // 1 in the token range where it measured faster, 2 whenever pair tiles are used
   essa::Scratch pair_ready;     // [token tiles][2] uint32: epoch of the last call that published u for (token tile, CTA rank)
@@ -176,6 +177,16 @@ struct PairDown {
 int32_t launch_base_up_pair(essa_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2,
                             const CUtensorMap& tmB2a, const CUtensorMap& tmB2b, int T, int d_out, int main_kb, int ext_kb,
                             int ext_ksteps, __nv_bfloat16* y, const __half* scale, const PairDown* down, cudaStream_t stream);
+// proj_tc3.cu: base + up on 512-token x 256-channel pair tiles, up to kWideMaxJobs projections (same T) per launch
+constexpr int kWideMaxJobs = 4;
+struct WideJob {
+  const CUtensorMap *tmA, *tmB, *tmA2, *tmB2a, *tmB2b;  // x, W0, u, U_B slab 0 / 1: boxes of 128 rows x 64 columns
+  int d_out, main_kb, ext_kb, ext_ksteps;
+  __nv_bfloat16* y;
+  const __half* scale;
+};
+bool wide_tiles_pay(int64_t T, int d_out, int total_kb, int sm_count);
+int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int T, cudaStream_t stream);
 // proj_decode.cu
 struct BlockItem {
   const essa_adapter* a;
@@ -194,6 +205,10 @@ constexpr int32_t kBlockNotFused = 1;  // launch_block_decode: the block does no
 int32_t launch_block_decode(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
                             const float* sigma, int32_t ld_sigma, cudaStream_t stream, const uint32_t* sigma_ready = nullptr,
                             uint32_t sigma_target = 0, int set = 0, int layer_mode = 0);
+// proj_tc.cu: prefill-sized block: the projections' rank-down launches, then one wide-tile launch for all of them
+// (kBlockNotFused if the block does not suit it).
+int32_t launch_block_prefill(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
+                             const float* sigma, int32_t ld_sigma, cudaStream_t stream);
 bool plan_decode(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype, int64_t T, int32_t sm_count, essa_plan* out);
 int32_t launch_projection_decode(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& args, const essa_plan& plan,
                                  cudaStream_t stream);

@@ -198,10 +198,17 @@ essa_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_fence_after();
           const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * C::A_BYTES));
           const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * C::B_BYTES));
-          const int nk = (kb < p.main_kb) ? (BLOCK_K / UMMA_K) : p.ext_ksteps;
-          for (int k = 0; k < nk; ++k) {
-            // advancing K by 16 bf16 inside the swizzled row = +32 bytes = +2 in the (addr >> 4) field
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          // advancing K by 16 bf16 inside the swizzled row = +32 bytes = +2 in the (addr >> 4) field
+          if (kb > kb0 && kb < p.main_kb) {
+            // the hot path as straight-line code: the issuing thread's own instructions between two MMAs (a loop
+            // counter, a predicate) show up in the K block's time
+            umma_bf16(d_tmem, a_desc, b_desc, idesc, 1u);
+            umma_bf16(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+            umma_bf16(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+            umma_bf16(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+          } else {
+            const int nk = (kb < p.main_kb) ? (BLOCK_K / UMMA_K) : p.ext_ksteps;
+            for (int k = 0; k < nk; ++k) umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(bar_empty + 8 * stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -489,6 +496,39 @@ void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype
   plan_prefill(d_in, d_out, rank, w0_dtype, T, sm_count, out);
 }
 
+// Rank-down launch of a prefill call: u_t = sB_k .* (M (sA_k .* (V_A^T x_t))) for all tokens, bf16, [T][64].
+static int32_t launch_rank_down(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, int down_splits, int down_grid,
+                                const CUtensorMap& tm_x, __nv_bfloat16* u, cudaStream_t stream) {
+  KParams kp{};
+  kp.T = (int)g.T;
+  kp.n_out = a->r_pad;
+  kp.main_kb = a->d_in / BLOCK_K;
+  kp.ext_kb = 0;
+  kp.ext_ksteps = 0;
+  kp.m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
+  kp.n_tiles = 1;
+  kp.splits = down_splits;
+  kp.seg = g.seg_offsets;
+  kp.P = g.P;
+  kp.sigma = g.sigma;
+  kp.ld_sigma = g.ld_sigma;
+  kp.sA_col = g.sA_col;
+  kp.sB_col = g.sB_col;
+  kp.r = a->rank;
+  kp.M = a->M;
+  kp.u = u;
+  kp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
+  kp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
+  kp.status = ctx->d_status;
+  switch (a->r_pad) {
+    case 16: return launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream);
+    case 32: return launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream);
+    case 48: return launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream);
+    case 64: return launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, down_grid, stream);
+    default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
+  }
+}
+
 int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArgs& g, cudaStream_t stream) {
   if (g.T == 0) return ESSA_OK;
   if (g.T > 0x7fffffffLL - BLOCK_M) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: T too large");
@@ -586,35 +626,8 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   }
 
   // ---- launch 1: rank-down
-  KParams kp{};
-  kp.T = (int)g.T;
-  kp.n_out = a->r_pad;
-  kp.main_kb = a->d_in / BLOCK_K;
-  kp.ext_kb = 0;
-  kp.ext_ksteps = 0;
-  kp.m_tiles = m_tiles;
-  kp.n_tiles = 1;
-  kp.splits = pl.down_splits;
-  kp.seg = g.seg_offsets;
-  kp.P = g.P;
-  kp.sigma = g.sigma;
-  kp.ld_sigma = g.ld_sigma;
-  kp.sA_col = g.sA_col;
-  kp.sB_col = g.sB_col;
-  kp.r = a->rank;
-  kp.M = a->M;
-  kp.u = u;
-  kp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
-  kp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
-  kp.status = ctx->d_status;
   if (!fused) {
-    switch (a->r_pad) {
-      case 16: st = launch_one<16, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-      case 32: st = launch_one<32, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-      case 48: st = launch_one<48, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-      case 64: st = launch_one<64, EPI_RANK>(ctx, tm_x, a->tm_VAt, tm_x, a->tm_VAt, a->tm_VAt, kp, pl.down_grid, stream); break;
-      default: return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "apply_projection: bad padded rank");
-    }
+    st = launch_rank_down(ctx, a, g, pl.down_splits, pl.down_grid, tm_x, u, stream);
     if (st != ESSA_OK) return st;
   }
   if (ev) cudaEventRecord(ev[1], stream);
@@ -635,6 +648,24 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
   mp.ws = static_cast<float*>(ctx->splitk_ws.ptr);
   mp.cnt = static_cast<int*>(ctx->splitk_cnt.ptr);
   mp.status = ctx->d_status;
+  if (use_pairs && !fused &&
+      (ctx->wide_tiles == 2 || (ctx->wide_tiles == 1 && wide_tiles_pay(g.T, a->d_out, a->d_in / BLOCK_K + a->ext_blocks, ctx->sm_count)))) {
+    WideJob job{};
+    job.tmA = &tm_x;
+    job.tmB = (a->w0_dtype != ESSA_W0_BF16) ? &tm_wdeq : &a->tm_W0[1];
+    job.tmA2 = &tm_u;
+    job.tmB2a = &a->tm_UBp[1][0];
+    job.tmB2b = &a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0];
+    job.d_out = a->d_out;
+    job.main_kb = a->d_in / BLOCK_K;
+    job.ext_kb = a->ext_blocks;
+    job.ext_ksteps = a->r_pad / UMMA_K;
+    job.y = g.y;
+    job.scale = mp.scale;
+    st = launch_base_up_wide(ctx, &job, 1, (int)g.T, stream);
+    if (ev) cudaEventRecord(ev[2], stream);
+    return st;
+  }
   if (use_pairs) {
     const CUtensorMap& tmW128 = (a->w0_dtype != ESSA_W0_BF16) ? tm_wdeq : a->tm_W0[1];
     st = launch_base_up_pair(ctx, tm_x, tmW128, tm_u, a->tm_UBp[1][0], a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0], (int)g.T,
@@ -653,6 +684,91 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     case 128: st = launch_one<128, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, pl.grid, stream); break;
     default: st = launch_one<256, EPI_STORE>(ctx, tm_x, tmW, tm_u, tmU0, tmU1, mp, pl.grid, stream); break;
   }
+  if (ev) cudaEventRecord(ev[2], stream);
+  return st;
+}
+
+// The base + up steps of a block's projections (same tokens, segments and table) in ONE wide-tile launch after
+// their rank-down launches: the concatenated tile list fills the persistent grid's rounds far better than four
+// lists of their own (config 4: 3120 tiles on 74 pairs = 42.2 rounds, against 17.6 + 3.5 + 3.5 + 17.6 rounded up to
+// 19 + 4 + 4 + 19).  Returns kBlockNotFused when the block does not suit it (quantised storage, small shapes, options).
+int32_t launch_block_prefill(essa_ctx* ctx, const BlockItem* items, int n, int64_t T, const int32_t* seg, int32_t P,
+                             const float* sigma, int32_t ld_sigma, cudaStream_t stream) {
+  if (n < 2 || n > kWideMaxJobs || T < 512 || T > 0x7fffffffLL - 512) return kBlockNotFused;
+  if (!ctx->pair_tiles || ctx->wide_tiles == 0 || ctx->fuse_down != 0) return kBlockNotFused;
+  essa_plan pl[kWideMaxJobs];
+  const int pairs = (ctx->sm_count > 0 ? ctx->sm_count : 148) / 2;
+  long long tiles_w = 0;
+  double cost_pair = 0.0, work_w = 0.0, longest_w = 0.0;
+  for (int i = 0; i < n; ++i) {
+    const essa_adapter* a = items[i].a;
+    if (a->w0_dtype != ESSA_W0_BF16) return kBlockNotFused;  // the dequantisation scratch holds one W0 at a time
+    plan_projection(a->d_in, a->d_out, a->rank, a->w0_dtype, T, ctx->sm_count, &pl[i]);
+    if (pl[i].decode || pl[i].block_n != 256 || pl[i].splits != 1) return kBlockNotFused;
+    const int kb = a->d_in / BLOCK_K + a->ext_blocks;
+    const long long nt = (a->d_out + 255) / 256;
+    const long long t2 = ((T + 255) / 256) * nt, tw = ((T + 511) / 512) * nt;
+    cost_pair += (double)((t2 + pairs - 1) / pairs) * (kb * 880.0 + 1500.0);
+    work_w += (double)tw * (kb * 1040.0 + 6000.0);
+    longest_w = longest_w > kb * 1040.0 + 6000.0 ? longest_w : kb * 1040.0 + 6000.0;
+    tiles_w += tw;
+  }
+  // whole rounds of the persistent grid for the concatenated list (the last, partial round costs one tile)
+  const double cost_w = tiles_w <= pairs ? longest_w : work_w / pairs + longest_w * (tiles_w % pairs ? 0.5 : 0.0);
+  if (ctx->wide_tiles == 1 && cost_w >= cost_pair) return kBlockNotFused;
+
+  const int m_tiles = (int)((T + BLOCK_M - 1) / BLOCK_M);
+  const size_t u_stride = (((size_t)T * kRankPadMax * 2 + 255) / 256) * 256;
+  int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)n * u_stride, false, stream);
+  if (st != ESSA_OK) return st;
+  size_t ws_need = 0, cnt_need = 0;
+  for (int i = 0; i < n; ++i)
+    if (pl[i].down_splits > 1) {
+      const size_t w = (size_t)m_tiles * BLOCK_M * items[i].a->r_pad * 4;
+      ws_need = ws_need > w ? ws_need : w;
+      cnt_need = (size_t)m_tiles * 4;
+    }
+  if (ws_need) {
+    st = ensure_scratch(ctx, ctx->splitk_ws, ws_need, true, stream);
+    if (st != ESSA_OK) return st;
+    st = ensure_scratch(ctx, ctx->splitk_cnt, cnt_need, true, stream);
+    if (st != ESSA_OK) return st;
+  }
+  CUtensorMap tm_x[kWideMaxJobs], tm_u[kWideMaxJobs];
+  WideJob jobs[kWideMaxJobs];
+  for (int i = 0; i < n; ++i) {
+    const essa_adapter* a = items[i].a;
+    __nv_bfloat16* u = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ctx->u_buf.ptr) + (size_t)i * u_stride);
+    st = make_tensor_map_2d(ctx, &tm_x[i], 0, items[i].x, (uint64_t)T, (uint64_t)a->d_in, (uint64_t)a->d_in * 2, BLOCK_M, BLOCK_K, 128);
+    if (st != ESSA_OK) return st;
+    st = make_tensor_map_2d(ctx, &tm_u[i], 0, u, (uint64_t)T, kRankPadMax, kRankPadMax * 2, BLOCK_M, BLOCK_K, 128);
+    if (st != ESSA_OK) return st;
+    jobs[i].tmA = &tm_x[i];
+    jobs[i].tmB = &a->tm_W0[1];
+    jobs[i].tmA2 = &tm_u[i];
+    jobs[i].tmB2a = &a->tm_UBp[1][0];
+    jobs[i].tmB2b = &a->tm_UBp[1][a->ext_blocks > 1 ? 1 : 0];
+    jobs[i].d_out = a->d_out;
+    jobs[i].main_kb = a->d_in / BLOCK_K;
+    jobs[i].ext_kb = a->ext_blocks;
+    jobs[i].ext_ksteps = a->r_pad / UMMA_K;
+    jobs[i].y = items[i].y;
+    jobs[i].scale = nullptr;
+  }
+  cudaEvent_t* ev = nullptr;
+  if (ctx->prof_on) {
+    if ((size_t)(ctx->prof_calls + 1) * 3 <= ctx->prof_events.size()) ev = &ctx->prof_events[(size_t)ctx->prof_calls++ * 3];
+    else ++ctx->prof_dropped;
+  }
+  if (ev) cudaEventRecord(ev[0], stream);
+  for (int i = 0; i < n; ++i) {
+    const ProjArgs g{items[i].x, T, seg, P, sigma, ld_sigma, items[i].sA_col, items[i].sB_col, items[i].y};
+    __nv_bfloat16* u = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ctx->u_buf.ptr) + (size_t)i * u_stride);
+    st = launch_rank_down(ctx, items[i].a, g, pl[i].down_splits, pl[i].down_grid, tm_x[i], u, stream);
+    if (st != ESSA_OK) return st;
+  }
+  if (ev) cudaEventRecord(ev[1], stream);
+  st = launch_base_up_wide(ctx, jobs, n, (int)T, stream);
   if (ev) cudaEventRecord(ev[2], stream);
   return st;
 }

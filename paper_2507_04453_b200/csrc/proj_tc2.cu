@@ -218,8 +218,17 @@ essa_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           tc_fence_after();
           const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * P2_A_BYTES));
           const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * P2_B_BYTES));
-          const int nk = (kb < p.main_kb) ? (P2_K / 16) : p.ext_ksteps;
-          for (int k = 0; k < nk; ++k) umma_bf16_2cta(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          if (kb > 0 && kb < p.main_kb) {
+            // the hot path as straight-line code: the issuing thread's own instructions between two MMAs (a loop
+            // counter, a predicate) show up in the K block's time
+            umma_bf16_2cta(d_tmem, a_desc, b_desc, idesc, 1u);
+            umma_bf16_2cta(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+            umma_bf16_2cta(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+            umma_bf16_2cta(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+          } else {
+            const int nk = (kb < p.main_kb) ? (P2_K / 16) : p.ext_ksteps;
+            for (int k = 0; k < nk; ++k) umma_bf16_2cta(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
           if (down && kb < p.main_kb) {
             constexpr uint32_t idesc_p = make_idesc(2 * P2_M, RP > 0 ? RP : 16);
             const uint64_t v_desc = make_smem_desc(smem_u32(smem_v + stage * V_BYTES));

@@ -1,7 +1,8 @@
 """GPU parity of essa_apply_block (the q, k, v, o projections of a block in one call) against the CPU oracle.
 
-At decode sizes the block runs as one launch of the decode kernel; otherwise it degrades to one call per
-projection.  Either way every projection's output must match the oracle like a single call does.
+At decode sizes the block runs as one launch of the decode kernel; at prefill sizes as the projections' rank-down
+launches followed by one launch for the base + up step of all of them, where the shapes suit that, else as one call
+per projection.  Either way every projection's output must match the oracle like a single call does.
 """
 import numpy as np
 import pytest
@@ -83,14 +84,34 @@ def test_block_equals_single_calls_in_structure_and_is_deterministic(torch, ctx)
     case.close()
 
 
-@pytest.mark.parametrize("name,max_cands", [("3", 24), ("5a", 12)])
-def test_block_full_size(torch, ctx, name, max_cands):
-    """The benchmark's decode configurations through the block call, in the launch configuration bench.py times."""
+def test_prefill_block_is_one_base_up_launch(torch, ctx):
+    """A prefill-sized block whose projections all suit the wide pair tiles: four rank-down launches, then ONE launch for
+    the base + up step of all four (ragged segments, T = 4348: the last 512-token tile holds 252 rows); with the wide
+    tiles switched off the block degrades to one call (two launches) per projection.  Both match the oracle."""
+    cfg = wl.scaled_config("4", d_model=1024, d_kv=1024, rank=32, P=12, seg_len=600)
+    case = Case(torch, ctx, cfg)
+    try:
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 2)
+        launches, xs, ys = _block(torch, ctx, case)
+        assert launches == len(cfg.projections) + 1
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 0)
+        launches0, _, ys0 = _block(torch, ctx, case)
+        assert launches0 == 2 * len(cfg.projections)
+        for a, b in zip(ys, ys0):  # same K order in fp32; u may differ in its last bit (split-K rank-down launches)
+            assert orc.relative_error(a.float().cpu().numpy(), b.float().cpu().numpy().astype(np.float64)) <= 8e-3
+    finally:
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 1)
+    case.close()
+
+
+@pytest.mark.parametrize("name,max_cands,want_launches", [("3", 24, 1), ("5a", 12, 1), ("4", 4, 5)])
+def test_block_full_size(torch, ctx, name, max_cands, want_launches):
+    """The benchmark's configurations through the block call, in the launch configuration bench.py times."""
     cfg = wl.CONFIGS[name]
     case = Case(torch, ctx, cfg)
     cands = wl.stratified_candidates(cfg, case.offsets)[:max_cands]
     launches, xs, ys = _block(torch, ctx, case, cands)
-    assert launches == 1
+    assert launches == want_launches
     tol = TOL_INT8 if cfg.w0_dtype == "int8" else TOL_BF16
     for i in range(4):  # every element against the CUDA-core path
         ref = ctx.apply_projection_simt(case.handles[i], xs[i], case.d_offsets, case.d_sigma, *cfg.sigma_cols(i))

@@ -193,6 +193,38 @@ def test_scaled_configs_full_outputs(torch, ctx, name):
     case.close()
 
 
+@pytest.mark.parametrize("base,dm,dkv,r,P,L", [("2", 1024, 256, 16, 4, 700),    # T = 2800: the last 512-token tile holds 240 rows
+                                               ("4", 768, 256, 32, 24, 300),    # ragged segments, three channel tiles
+                                               ("2", 1024, 256, 33, 13, 197),   # T = 2561: one row in the last tile; padded rank 48
+                                               ("5b", 2048, 512, 64, 16, 128),  # INT8 storage: two rank slabs, scale in the epilogue
+                                               ("6b", 2048, 512, 64, 9, 130)])  # INT4 group-wise storage
+def test_wide_pair_tiles(torch, ctx, base, dm, dkv, r, P, L):
+    """Prefill base + up on 512-token x 256-channel pair tiles (ESSA_OPT_WIDE_TILES = 2) matches the oracle, and the
+    256 x 256 pair tiles (ESSA_OPT_WIDE_TILES = 0) to the last bit or so: both add the K blocks in the same order in
+    fp32; only u can differ in its last bit between two calls (the rank-down launch splits K at these token counts and
+    adds its partial sums in arrival order)."""
+    from paper_2507_04453_b200 import binding
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg, projections=[0])
+    tol = TOL_BF16 if cfg.w0_dtype == "bf16" else TOL_INT8
+    code = {"bf16": 0, "int8": 1, "int4": 2}[cfg.w0_dtype]
+    plan = binding.plan_projection(dm, dm, r, code, case.T)
+    assert plan["block_n"] == 256 and plan["splits"] == 1 and case.T >= 512  # the shape the pair tiles take
+    x = case.tokens(0)
+    want = case.oracle_projection(0, x)
+    try:
+        outs = {}
+        for wide in (2, 0):
+            ctx.set_option(binding.ESSA_OPT_WIDE_TILES, wide)
+            outs[wide] = case.gpu_projection(0, x)
+            assert np.isfinite(outs[wide]).all()
+        assert orc.relative_error(outs[2], want) <= tol
+        assert np.mean(outs[2] != outs[0]) < 0.02 and orc.relative_error(outs[2], outs[0].astype(np.float64)) <= 8e-3
+    finally:
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 1)
+    case.close()
+
+
 @pytest.mark.parametrize("base,dm,dkv,r,P,L", [("2", 1024, 256, 16, 4, 700),    # T = 2800: 11 token tiles, ragged last tile
                                                ("2", 1024, 256, 33, 8, 300),    # padded rank 48
                                                ("5b", 2048, 512, 64, 16, 128)])  # INT8 storage, rank 64, five stages
