@@ -116,6 +116,16 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   them ahead of the 256 x 256 pair tiles (1), wherever the pair tiles would run (2), or never (0).  Both tile
  *   shapes add the K blocks in the same order in fp32. */
 #define ESSA_OPT_WIDE_TILES 7
+/*   ESSA_OPT_DOWN_SPLITS (0 .. 64, default 0): split of the K range of a prefill call's rank-down launch (each token
+ *   tile's down-projection is shared by that many thread blocks, which add their fp32 partial sums in a workspace);
+ *   0 leaves the choice to the planner, which balances the persistent grid's rounds. */
+#define ESSA_OPT_DOWN_SPLITS 8
+/*   ESSA_OPT_L2_HINTS (default 1): L2 eviction priorities the wide prefill kernel attaches to its TMA copies.  Bits 0-2:
+ *   bit 0 = the W0 rows of a projection's leading channel tiles are loaded evict-last (as many tiles as fit ~21 MB: more
+ *   than that thrashes), bit 1 = x / u loads evict-first (measured harmful: the pairs that share a token tile lose it),
+ *   bit 2 = y stores evict-first.  Bits 8-15, if non-zero: the number of leading channel tiles to mark, instead of the
+ *   21 MB rule (for measurements). */
+#define ESSA_OPT_L2_HINTS 9
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

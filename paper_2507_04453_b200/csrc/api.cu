@@ -262,6 +262,14 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
     case ESSA_OPT_DEBUG_STALL_RANK_ROWS: ctx->debug_stall_rank_rows = value != 0; return ESSA_OK;
     case ESSA_OPT_DECODE_PAIRS: ctx->decode_pairs = value != 0; return ESSA_OK;
     case ESSA_OPT_DECODE_DOWN_CTAS: ctx->down_ctas = value != 0; return ESSA_OK;
+    case ESSA_OPT_DOWN_SPLITS:
+      if (value < 0 || value > 64) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_DOWN_SPLITS takes 0 .. 64");
+      ctx->down_splits = value;
+      return ESSA_OK;
+    case ESSA_OPT_L2_HINTS:
+      if (value < 0 || value > 0xffff) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_L2_HINTS takes 0 .. 65535");
+      ctx->l2_hints = value;
+      return ESSA_OK;
     case ESSA_OPT_WIDE_TILES:
       if (value < 0 || value > 2) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_WIDE_TILES takes 0, 1 or 2");
       ctx->wide_tiles = value;
@@ -282,9 +290,13 @@ int32_t essa_reserve(essa_ctx* ctx, int64_t max_tokens, int32_t max_d_in, int32_
   int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)ESSA_MAX_BLOCK_ITEMS * ((size_t)max_tokens * kRankPadMax * 2 + 256), false, nullptr);
   if (st != ESSA_OK) return st;
   // split-K is only used while there are fewer tiles than SMs: at most sm_count tiles of 128 x 256 fp32
-  st = ensure_scratch(ctx, ctx->splitk_ws, (size_t)ctx->sm_count * 128 * 256 * 4, true, nullptr);
+  // ... and by the rank-down launch, whose K range may be split at any token count: 128 x 64 fp32 per token tile
+  const size_t m_tiles = (size_t)((max_tokens + 127) / 128);
+  const size_t ws_tc = (size_t)ctx->sm_count * 128 * 256 * 4, ws_down = m_tiles * 128 * kRankPadMax * 4;
+  st = ensure_scratch(ctx, ctx->splitk_ws, ws_tc > ws_down ? ws_tc : ws_down, true, nullptr);
   if (st != ESSA_OK) return st;
-  st = ensure_scratch(ctx, ctx->splitk_cnt, (size_t)ctx->sm_count * 4 * 4, true, nullptr);
+  const size_t cnt_tc = (size_t)ctx->sm_count * 4 * 4, cnt_down = m_tiles * 4;
+  st = ensure_scratch(ctx, ctx->splitk_cnt, cnt_tc > cnt_down ? cnt_tc : cnt_down, true, nullptr);
   if (st != ESSA_OK) return st;
   st = ensure_scratch(ctx, ctx->stage_x, (size_t)max_tokens * max_d_in * 2, false, nullptr);
   if (st != ESSA_OK) return st;

@@ -474,6 +474,9 @@ static void plan_prefill(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_d
   const long long items = (long long)out->tiles * best_splits;
   out->grid = (int)(items < sm ? items : sm);
   // rank-down kernel: one tile per 128 tokens, N = r_pad; split K until the SMs are covered
+  // (with at least one tile per SM the K range stays whole: splitting it to even out the persistent grid's last round
+  // measured SLOWER at every split -- config 4, four launches: 301 us unsplit, 325 / 458 / 715 us split 2 / 4 / 8 ways --
+  // because the partial sums go through fp32 atomics in a workspace)
   int ds = 1;
   if (m_tiles > 0 && m_tiles < sm) {
     ds = sm / m_tiles;
@@ -494,6 +497,17 @@ void plan_projection(int32_t d_in, int32_t d_out, int32_t rank, int32_t w0_dtype
   *out = essa_plan{};
   if (plan_decode(d_in, d_out, rank, w0_dtype, T, sm_count, out)) return;
   plan_prefill(d_in, d_out, rank, w0_dtype, T, sm_count, out);
+}
+
+// ESSA_OPT_DOWN_SPLITS: a given K split of the rank-down launch instead of the planner's.
+static void override_down_splits(const essa_ctx* ctx, essa_plan* pl, int m_tiles, int main_kb) {
+  if (ctx->down_splits <= 0) return;
+  const int sm = ctx->sm_count > 0 ? ctx->sm_count : 148;
+  int ds = ctx->down_splits < main_kb ? ctx->down_splits : main_kb;
+  if (ds < 1) ds = 1;
+  pl->down_splits = ds;
+  const long long items = (long long)m_tiles * ds;
+  pl->down_grid = (int)(items < sm ? items : sm);
 }
 
 // Rank-down launch of a prefill call: u_t = sB_k .* (M (sA_k .* (V_A^T x_t))) for all tokens, bf16, [T][64].
@@ -546,6 +560,7 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
     return dst;
   }
   const int m_tiles = (int)((g.T + BLOCK_M - 1) / BLOCK_M);
+  override_down_splits(ctx, &pl, m_tiles, a->d_in / BLOCK_K);
 
   int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)g.T * kRankPadMax * 2, false, stream);
   if (st != ESSA_OK) return st;
@@ -718,6 +733,7 @@ int32_t launch_block_prefill(essa_ctx* ctx, const BlockItem* items, int n, int64
   if (ctx->wide_tiles == 1 && cost_w >= cost_pair) return kBlockNotFused;
 
   const int m_tiles = (int)((T + BLOCK_M - 1) / BLOCK_M);
+  for (int i = 0; i < n; ++i) override_down_splits(ctx, &pl[i], m_tiles, items[i].a->d_in / BLOCK_K);
   const size_t u_stride = (((size_t)T * kRankPadMax * 2 + 255) / 256) * 256;
   int32_t st = ensure_scratch(ctx, ctx->u_buf, (size_t)n * u_stride, false, stream);
   if (st != ESSA_OK) return st;

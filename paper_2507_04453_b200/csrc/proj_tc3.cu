@@ -48,11 +48,13 @@ struct WMaps {
 
 struct WJobDev {
   int n_out, main_kb, ext_kb, ext_ksteps, n_tiles, tile_begin;
+  int keep_tiles;  // channel tiles (from 0) whose W0 rows are loaded with the evict-last L2 policy
   const __half* scale;
 };
 
 struct WParams {
   int T, m_tiles, n_jobs, tiles;
+  int l2_hints;  // bit 0: W0 / U_B loads evict-last, bit 1: x / u loads evict-first, bit 2: y stores evict-first
   WJobDev job[kWideMaxJobs];
   int32_t* status;
 };
@@ -113,6 +115,9 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
+      // W0 is read again by every later round of the grid and should stay in L2 while x and y stream past it
+      const uint64_t pol_w = l2_policy_evict_last(), pol_x = l2_policy_evict_first();
+      const bool hint_w = (p.l2_hints & 1) != 0, hint_x = (p.l2_hints & 2) != 0;
       for (int w = pair; ok && w < p.tiles; w += n_pairs) {
         int j, m_tile, n_tile;
         tile_of(w, j, m_tile, n_tile);
@@ -128,11 +133,17 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
           if (prod_a) {
             const CUtensorMap* tm = kb < jb.main_kb ? &maps.m[j][0] : &maps.m[j][2];
             const int col = kb < jb.main_kb ? kb * 64 : 0;
-            tma_load_2d_pair(da, tm, col, row_a, fb);
-            tma_load_2d_pair(da + W_BOX, tm, col, row_a + 256, fb);
+            if (hint_x) {
+              tma_load_2d_pair_hint(da, tm, col, row_a, fb, pol_x);
+              tma_load_2d_pair_hint(da + W_BOX, tm, col, row_a + 256, fb, pol_x);
+            } else {
+              tma_load_2d_pair(da, tm, col, row_a, fb);
+              tma_load_2d_pair(da + W_BOX, tm, col, row_a + 256, fb);
+            }
           } else {
             const CUtensorMap* tm = kb < jb.main_kb ? &maps.m[j][1] : (kb == jb.main_kb ? &maps.m[j][3] : &maps.m[j][4]);
-            tma_load_2d_pair(db, tm, kb < jb.main_kb ? kb * 64 : 0, row_b, fb);
+            if (hint_w && n_tile < jb.keep_tiles) tma_load_2d_pair_hint(db, tm, kb < jb.main_kb ? kb * 64 : 0, row_b, fb, pol_w);
+            else tma_load_2d_pair(db, tm, kb < jb.main_kb ? kb * 64 : 0, row_b, fb);
           }
           ++issued;
           if (++stage == W_STAGES) { stage = 0; phase ^= 1; }
@@ -209,6 +220,7 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
     const int acc = (warp - 2) >> 2;  // which accumulator this warp drains
     const int quad = warp & 3;        // the TMEM lanes this warp may read
     const uint32_t stg = smem_u32(stg_all + (warp - 2) * W_OUT_BOX);
+    const uint64_t pol_y = l2_policy_evict_first();
     int it = 0;
     for (int w = pair; w < p.tiles; w += n_pairs, ++it) {
       int j, m_tile, n_tile;
@@ -270,7 +282,8 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < p.T && col0 < jb.n_out) {
-          tma_store_2d(&maps.m[j][5], stg, col0, row0);
+          if (p.l2_hints & 4) tma_store_2d_hint(&maps.m[j][5], stg, col0, row0, pol_y);
+          else tma_store_2d(&maps.m[j][5], stg, col0, row0);
           bulk_commit_group();
         }
       }
@@ -310,6 +323,7 @@ int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int 
   p.m_tiles = (T + W_TILE_M - 1) / W_TILE_M;
   p.n_jobs = n_jobs;
   p.status = ctx->d_status;
+  p.l2_hints = ctx->l2_hints & 7;
   long long tiles = 0;
   for (int j = 0; j < n_jobs; ++j) {
     const WideJob& s = jobs[j];
@@ -320,6 +334,13 @@ int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int 
     d.ext_ksteps = s.ext_ksteps;
     d.n_tiles = (s.d_out + W_TILE_N - 1) / W_TILE_N;
     d.tile_begin = (int)tiles;
+    // Evict-last protects about 21 MB of L2 on this part: config 4's q projection (W0 = 52 MB, re-read from HBM by
+    // every round of the grid) read 1324 MB without hints, 1170 / 1057 / 1196 / 1316 MB with the first 4 / 8 / 12 / 16
+    // channel tiles (10 / 21 / 31 / 42 MB) marked, 1320 MB with all 20.  So mark as many leading tiles as fit 21 MB.
+    const int forced = ctx->l2_hints >> 8;
+    const long long tile_bytes = 256LL * s.main_kb * 64 * 2;
+    d.keep_tiles = forced > 0 ? forced : (int)(tile_bytes > 0 ? (21LL << 20) / tile_bytes : 0);
+    if (d.keep_tiles < 1) d.keep_tiles = 1;
     d.scale = s.scale;
     tiles += (long long)p.m_tiles * d.n_tiles;
     if (tiles > 0x7fffffffLL) return fail(ctx, ESSA_ERR_UNSUPPORTED_SHAPE, "launch_base_up_wide: too many tiles");
