@@ -120,11 +120,14 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   tile's down-projection is shared by that many thread blocks, which add their fp32 partial sums in a workspace);
  *   0 leaves the choice to the planner, which balances the persistent grid's rounds. */
 #define ESSA_OPT_DOWN_SPLITS 8
-/*   ESSA_OPT_L2_HINTS (default 1): L2 eviction priorities the wide prefill kernel attaches to its TMA copies.  Bits 0-2:
+/*   ESSA_OPT_L2_HINTS (default 13): how the wide prefill kernel treats L2.  Bits 0-3:
  *   bit 0 = the W0 rows of a projection's leading channel tiles are loaded evict-last (as many tiles as fit ~21 MB: more
  *   than that thrashes), bit 1 = x / u loads evict-first (measured harmful: the pairs that share a token tile lose it),
- *   bit 2 = y stores evict-first.  Bits 8-15, if non-zero: the number of leading channel tiles to mark, instead of the
- *   21 MB rule (for measurements). */
+ *   bit 2 = y stores evict-first, bit 3 = every other tile of a CTA pair walks K backwards, so that a round of the
+ *   persistent grid starts with the K slabs the round before used last (the result's fp32 summation order then
+ *   differs between tiles; it is the same from call to call).  Config 4's q projection reads 1404 MB from HBM with 0,
+ *   990 with 8, 832 with 9, 797 with 13 (x and W0 are 415 MB).  Bits 8-15, if non-zero: the number of leading channel
+ *   tiles to mark, instead of the 21 MB rule (for measurements). */
 #define ESSA_OPT_L2_HINTS 9
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */

@@ -38,7 +38,7 @@ struct essa_ctx {
   bool decode_pairs = false;  // ESSA_OPT_DECODE_PAIRS
   bool down_ctas = true;      // ESSA_OPT_DECODE_DOWN_CTAS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
-  int l2_hints = 1;             // L2 eviction hints of the wide prefill kernel's TMA copies (essa_set_option)
+  int l2_hints = 13;            // L2 eviction hints of the wide prefill kernel's TMA copies (essa_set_option)
   int down_splits = 0;          // K split of the prefill rank-down launch: 0 = the planner's choice (essa_set_option)
   int wide_tiles = 1;           // ... on 512 x 256 pair tiles: 0 never, 1 where the planner's estimate favours them, 2 always
   int fuse_down = 0;            // ... which also compute the down-projection (no rank-down launch): 0 never (default),

@@ -54,7 +54,7 @@ struct WJobDev {
 
 struct WParams {
   int T, m_tiles, n_jobs, tiles;
-  int l2_hints;  // bit 0: W0 / U_B loads evict-last, bit 1: x / u loads evict-first, bit 2: y stores evict-first
+  int l2_hints;  // bit 0: W0 / U_B loads evict-last, bit 1: x / u loads evict-first, bit 2: y stores evict-first, bit 3: K walks back on odd tiles
   WJobDev job[kWideMaxJobs];
   int32_t* status;
 };
@@ -118,11 +118,17 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
       // W0 is read again by every later round of the grid and should stay in L2 while x and y stream past it
       const uint64_t pol_w = l2_policy_evict_last(), pol_x = l2_policy_evict_first();
       const bool hint_w = (p.l2_hints & 1) != 0, hint_x = (p.l2_hints & 2) != 0;
-      for (int w = pair; ok && w < p.tiles; w += n_pairs) {
+      int it = 0;
+      for (int w = pair; ok && w < p.tiles; w += n_pairs, ++it) {
         int j, m_tile, n_tile;
         tile_of(w, j, m_tile, n_tile);
         const WJobDev& jb = p.job[j];
         const int total_kb = jb.main_kb + jb.ext_kb;
+        // Every other tile of a pair walks K backwards.  All pairs run in step, so a round of the grid streams the
+        // same K slabs of W0 (and of the token tiles it shares with the round before) in the same order; the rounds'
+        // footprint (config 4: 91 MB) exceeds what L2 keeps, and with every round walking K forwards a slab is always
+        // gone when its turn comes again.  Walking back, a round starts with the slabs the round before used last.
+        const bool k_back = (p.l2_hints & 8) != 0 && (it & 1) != 0;
         const int row_a = m_tile * W_TILE_M + (int)rank * 128;  // + 256 for the second accumulator's box
         const int row_b = n_tile * W_TILE_N + (int)rank * 128;  // channels of this CTA
         for (int kb = 0; kb < total_kb; ++kb) {
@@ -132,7 +138,7 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
           const uint32_t da = smem_u32(smem + stage * W_STAGE), db = da + W_A_BYTES;
           if (prod_a) {
             const CUtensorMap* tm = kb < jb.main_kb ? &maps.m[j][0] : &maps.m[j][2];
-            const int col = kb < jb.main_kb ? kb * 64 : 0;
+            const int col = kb < jb.main_kb ? (k_back ? jb.main_kb - 1 - kb : kb) * 64 : 0;
             if (hint_x) {
               tma_load_2d_pair_hint(da, tm, col, row_a, fb, pol_x);
               tma_load_2d_pair_hint(da + W_BOX, tm, col, row_a + 256, fb, pol_x);
@@ -142,8 +148,9 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
             }
           } else {
             const CUtensorMap* tm = kb < jb.main_kb ? &maps.m[j][1] : (kb == jb.main_kb ? &maps.m[j][3] : &maps.m[j][4]);
-            if (hint_w && n_tile < jb.keep_tiles) tma_load_2d_pair_hint(db, tm, kb < jb.main_kb ? kb * 64 : 0, row_b, fb, pol_w);
-            else tma_load_2d_pair(db, tm, kb < jb.main_kb ? kb * 64 : 0, row_b, fb);
+            const int col = kb < jb.main_kb ? (k_back ? jb.main_kb - 1 - kb : kb) * 64 : 0;
+            if (hint_w && n_tile < jb.keep_tiles) tma_load_2d_pair_hint(db, tm, col, row_b, fb, pol_w);
+            else tma_load_2d_pair(db, tm, col, row_b, fb);
           }
           ++issued;
           if (++stage == W_STAGES) { stage = 0; phase ^= 1; }
@@ -323,7 +330,7 @@ int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int 
   p.m_tiles = (T + W_TILE_M - 1) / W_TILE_M;
   p.n_jobs = n_jobs;
   p.status = ctx->d_status;
-  p.l2_hints = ctx->l2_hints & 7;
+  p.l2_hints = ctx->l2_hints & 15;
   long long tiles = 0;
   for (int j = 0; j < n_jobs; ++j) {
     const WideJob& s = jobs[j];
