@@ -129,6 +129,12 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   990 with 8, 832 with 9, 797 with 13 (x and W0 are 415 MB).  Bits 8-15, if non-zero: the number of leading channel
  *   tiles to mark, instead of the 21 MB rule (for measurements). */
 #define ESSA_OPT_L2_HINTS 9
+/*   ESSA_OPT_DOWN_PAIRS (0 .. 5, default 5): the rank-down step of prefill-sized calls runs on CTA pairs (one launch for all
+ *   projections of a block, token rows dealt to the pairs in 64-row units) where every pair gets at least four units and
+ *   the rank is at most 32 (beyond that the single-CTA kernel measured faster);
+ *   the value is the number of threads per CTA that issue its TMA copies in turn.  0 keeps one single-CTA launch of
+ *   128-token tiles per projection. */
+#define ESSA_OPT_DOWN_PAIRS 10
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

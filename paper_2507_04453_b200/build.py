@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 BUILD_DIR = os.path.join(PKG_DIR, "_build")
 LIB_PATH = os.path.join(PKG_DIR, "libessa.so")
-SOURCES = ["api.cu", "sampler.cu", "adapter_prep.cu", "proj_simt.cu", "proj_tc.cu", "proj_tc2.cu", "proj_tc3.cu", "proj_decode.cu", "cma.cu"]
+SOURCES = ["api.cu", "sampler.cu", "adapter_prep.cu", "proj_simt.cu", "proj_tc.cu", "proj_tc2.cu", "proj_tc3.cu", "proj_down.cu", "proj_decode.cu", "cma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

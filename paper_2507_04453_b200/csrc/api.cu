@@ -266,6 +266,10 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
       if (value < 0 || value > 64) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_DOWN_SPLITS takes 0 .. 64");
       ctx->down_splits = value;
       return ESSA_OK;
+    case ESSA_OPT_DOWN_PAIRS:
+      if (value < 0 || value > 5) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_DOWN_PAIRS takes 0 .. 5");
+      ctx->down_pairs = value;
+      return ESSA_OK;
     case ESSA_OPT_L2_HINTS:
       if (value < 0 || value > 0xffff) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_L2_HINTS takes 0 .. 65535");
       ctx->l2_hints = value;

@@ -38,6 +38,7 @@ struct essa_ctx {
   bool decode_pairs = false;  // ESSA_OPT_DECODE_PAIRS
   bool down_ctas = true;      // ESSA_OPT_DECODE_DOWN_CTAS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
+  int down_pairs = 5;           // prefill rank-down step on CTA pairs: 0 = off, 1..5 = TMA-issuing threads per CTA (essa_set_option)
   int l2_hints = 13;            // L2 eviction hints of the wide prefill kernel's TMA copies (essa_set_option)
   int down_splits = 0;          // K split of the prefill rank-down launch: 0 = the planner's choice (essa_set_option)
   int wide_tiles = 1;           // ... on 512 x 256 pair tiles: 0 never, 1 where the planner's estimate favours them, 2 always
@@ -189,6 +190,16 @@ struct WideJob {
 };
 bool wide_tiles_pay(int64_t T, int d_out, int total_kb, int sm_count);
 int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int T, cudaStream_t stream);
+// proj_down.cu: the rank-down step of up to kWideMaxJobs projections (same T, same padded rank) in one CTA-pair launch
+struct DownJob {
+  const essa_adapter* a;
+  const __nv_bfloat16* x;
+  int32_t sA_col, sB_col;
+  __nv_bfloat16* u;  // [T][64]
+};
+bool down_pairs_suit(const essa_ctx* ctx, const DownJob* jobs, int n_jobs, int64_t T);
+int32_t launch_rank_down_pairs(essa_ctx* ctx, const DownJob* jobs, int n_jobs, int64_t T, const int32_t* seg, int32_t P,
+                               const float* sigma, int32_t ld_sigma, cudaStream_t stream);
 // proj_decode.cu
 struct BlockItem {
   const essa_adapter* a;

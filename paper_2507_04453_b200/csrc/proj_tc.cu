@@ -642,7 +642,11 @@ int32_t launch_projection_tc(essa_ctx* ctx, const essa_adapter* a, const ProjArg
 
   // ---- launch 1: rank-down
   if (!fused) {
-    st = launch_rank_down(ctx, a, g, pl.down_splits, pl.down_grid, tm_x, u, stream);
+    const DownJob dj{a, g.x, g.sA_col, g.sB_col, u};
+    if (down_pairs_suit(ctx, &dj, 1, g.T))
+      st = launch_rank_down_pairs(ctx, &dj, 1, g.T, g.seg_offsets, g.P, g.sigma, g.ld_sigma, stream);
+    else
+      st = launch_rank_down(ctx, a, g, pl.down_splits, pl.down_grid, tm_x, u, stream);
     if (st != ESSA_OK) return st;
   }
   if (ev) cudaEventRecord(ev[1], stream);
@@ -777,11 +781,19 @@ int32_t launch_block_prefill(essa_ctx* ctx, const BlockItem* items, int n, int64
     else ++ctx->prof_dropped;
   }
   if (ev) cudaEventRecord(ev[0], stream);
-  for (int i = 0; i < n; ++i) {
-    const ProjArgs g{items[i].x, T, seg, P, sigma, ld_sigma, items[i].sA_col, items[i].sB_col, items[i].y};
-    __nv_bfloat16* u = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ctx->u_buf.ptr) + (size_t)i * u_stride);
-    st = launch_rank_down(ctx, items[i].a, g, pl[i].down_splits, pl[i].down_grid, tm_x[i], u, stream);
+  DownJob dj[kWideMaxJobs];
+  for (int i = 0; i < n; ++i)
+    dj[i] = DownJob{items[i].a, items[i].x, items[i].sA_col, items[i].sB_col,
+                    reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(ctx->u_buf.ptr) + (size_t)i * u_stride)};
+  if (down_pairs_suit(ctx, dj, n, T)) {  // one launch for the rank-down step of all projections
+    st = launch_rank_down_pairs(ctx, dj, n, T, seg, P, sigma, ld_sigma, stream);
     if (st != ESSA_OK) return st;
+  } else {
+    for (int i = 0; i < n; ++i) {
+      const ProjArgs g{items[i].x, T, seg, P, sigma, ld_sigma, items[i].sA_col, items[i].sB_col, items[i].y};
+      st = launch_rank_down(ctx, items[i].a, g, pl[i].down_splits, pl[i].down_grid, tm_x[i], dj[i].u, stream);
+      if (st != ESSA_OK) return st;
+    }
   }
   if (ev) cudaEventRecord(ev[1], stream);
   st = launch_base_up_wide(ctx, jobs, n, (int)T, stream);

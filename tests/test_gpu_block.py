@@ -93,7 +93,7 @@ def test_prefill_block_is_one_base_up_launch(torch, ctx):
     try:
         ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 2)
         launches, xs, ys = _block(torch, ctx, case)
-        assert launches == len(cfg.projections) + 1
+        assert launches == len(cfg.projections) + 1  # (too few tokens for the CTA-pair rank-down kernel: one launch each)
         ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 0)
         launches0, _, ys0 = _block(torch, ctx, case)
         assert launches0 == 2 * len(cfg.projections)
@@ -104,7 +104,37 @@ def test_prefill_block_is_one_base_up_launch(torch, ctx):
     case.close()
 
 
-@pytest.mark.parametrize("name,max_cands,want_launches", [("3", 24, 1), ("5a", 12, 1), ("4", 4, 5)])
+@pytest.mark.parametrize("base,dm,dkv,r,P,L,pairs", [("4", 512, 512, 32, 40, 1000, True),    # ragged, T = 21 394: 335 units of 64 rows per projection
+                                                     ("2", 512, 512, 16, 30, 650, True),     # T = 19 500
+                                                     ("5c", 512, 512, 17, 150, 256, True),   # INT8 storage (one call per projection), padded rank 32, mixed lengths
+                                                     ("2", 512, 512, 33, 30, 650, False)])   # padded rank 48: stays on the single-CTA kernel
+def test_rank_down_on_cta_pairs(torch, ctx, base, dm, dkv, r, P, L, pairs):
+    """Prefill-sized block with enough tokens for the CTA-pair rank-down kernel (every pair of the grid gets at least four
+    64-row units; the last tile of a pair's range is partial): bf16 blocks run ONE rank-down launch and ONE base + up
+    launch.  The result matches the oracle and, to the last bit or so, the single-CTA rank-down launches
+    (ESSA_OPT_DOWN_PAIRS = 0), which add the same K blocks in the same order."""
+    cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
+    case = Case(torch, ctx, cfg)
+    assert (case.T + 63) // 64 >= 4 * 74
+    cands = wl.stratified_candidates(cfg, case.offsets)[:10]
+    n = len(cfg.projections)
+    bf16 = cfg.w0_dtype == "bf16"
+    try:
+        launches, xs, ys = _block(torch, ctx, case, cands)
+        # quantised storage: dequantisation pass, rank-down, base + up per projection
+        assert launches == ((2 if pairs else n + 1) if bf16 else 3 * n)
+        ctx.set_option(binding.ESSA_OPT_DOWN_PAIRS, 0)
+        launches0, _, ys0 = _block(torch, ctx, case, cands)
+        assert launches0 == (n + 1 if bf16 else 3 * n)
+        for a, b in zip(ys, ys0):
+            a, b = a.float().cpu().numpy(), b.float().cpu().numpy()
+            assert np.mean(a != b) < 0.01 and orc.relative_error(a, b.astype(np.float64)) <= 8e-3
+    finally:
+        ctx.set_option(binding.ESSA_OPT_DOWN_PAIRS, 5)
+    case.close()
+
+
+@pytest.mark.parametrize("name,max_cands,want_launches", [("3", 24, 1), ("5a", 12, 1), ("4", 4, 2)])
 def test_block_full_size(torch, ctx, name, max_cands, want_launches):
     """The benchmark's configurations through the block call, in the launch configuration bench.py times."""
     cfg = wl.CONFIGS[name]
