@@ -48,9 +48,10 @@ CSRC = os.path.join(ROOT, "paper_2507_04453_b200", "csrc")
 # with the SHA-256 (first 16 hex digits) of the kernel's source file at capture time: a kernel that has changed
 # since reports "traffic": null until it is captured again.
 NCU_TRAFFIC = {
-    "2": {"bytes": 877e6, "source": "proj_tc3.cu", "sha16": "", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
-          "note": "captured at half the population and scaled (W0 traffic fixed, x and y traffic doubled); before the L2 handling of ESSA_OPT_L2_HINTS"},
-    "4": {"bytes": 3418.7e6, "source": "proj_tc3.cu", "sha16": "c89c12947229de1f", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md"},
+    "2": {"bytes": 794e6, "source": "proj_tc3.cu", "sha16": "c89c12947229de1f", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
+          "note": "captured at half the population (426.3 MB) and scaled: W0 traffic fixed, x and y traffic doubled"},
+    "4": {"bytes": 4316.7e6, "source": "proj_tc3.cu", "sha16": "c89c12947229de1f", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
+          "note": "full size; captures of the same build range from 3.4 to 5.4 GB (how well the CTA pairs stay in step)"},
     "3": {"bytes": 67.9e6, "source": "proj_decode.cu", "sha16": "b82b27e15eee5ff2", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
     "5a": {"bytes": 170.5e6, "source": "proj_decode.cu", "sha16": "b82b27e15eee5ff2", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
 }
