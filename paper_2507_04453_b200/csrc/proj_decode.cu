@@ -786,7 +786,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       if (!got_c) break;
       if (i >= nkb) continue;
       const int sr = i % SW;
-      while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}  // complete: acquire for every lane
+      // (lane 0 has observed the phase and the shuffle orders the other lanes after it: a barrier probe by all 32 lanes
+      // costs ~200 cycles even when the phase is complete)
       const uint32_t raw = smem_u32(smem_w + sr * RAW_TILE_BYTES);
       const uint32_t out = smem_u32(smem_c + sc * W_TILE_BYTES);
 #pragma unroll 2
@@ -835,9 +836,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       }
       got_c = __shfl_sync(0xffffffffu, got_c, 0);
       if (!got_c) break;
-      // both phases are complete: these return at once (acquire for every lane)
-      if (i >= SA) while (!mbar_try_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1))) {}
-      while (!mbar_try_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1))) {}
+      // lane 0 has observed both phases and the shuffle above orders the other lanes' reads of the tile after that
+      // (probing the two barriers with all 32 lanes as well cost ~420 cycles per tile although both were complete)
       tc_fence_after();  // the MMAs that read this stage have completed (their commit released it)
       uint32_t v[32];
       if (I4) {
