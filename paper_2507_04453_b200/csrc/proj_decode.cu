@@ -827,19 +827,9 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
   if (TS && warp >= 6 && warp <= 9) {
     const int band = warp & 3;
     const int r = band * 32 + lane;
-    for (int i = 0; i < nkb; ++i) {
-      const int sa = i % SA, sr = i % SW;
-      int got_c = 1;
-      if (lane == 0) {
-        if (i >= SA) got_c = mbar_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1), abort_flag, p.status) ? 1 : 0;
-        if (got_c) got_c = mbar_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1), abort_flag, p.status) ? 1 : 0;
-      }
-      got_c = __shfl_sync(0xffffffffu, got_c, 0);
-      if (!got_c) break;
-      // lane 0 has observed both phases and the shuffle above orders the other lanes' reads of the tile after that
-      // (probing the two barriers with all 32 lanes as well cost ~420 cycles per tile although both were complete)
-      tc_fence_after();  // the MMAs that read this stage have completed (their commit released it)
-      uint32_t v[32];
+    // one row of tile i: codes from the ring slot -> 32 packed bf16 pairs
+    auto convert_row = [&](int i, uint32_t (&v)[32]) {
+      const int sr = i % SW;
       if (I4) {
         // a row of the tile is 32 bytes = two 16-byte chunks, loaded with the 32-byte swizzle (chunk c of row r at
         // position c ^ ((r >> 2) & 1): again eight different bank groups per quarter-warp); the 64 codes of the row
@@ -874,13 +864,53 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
           int8x4_to_bf16x4(w[c].w, v[8 * c + 6], v[8 * c + 7]);
         }
       }
-      tmem_st32(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(sa), v);
+    };
+    // lane 0 observes the barriers of tile i (its stage of tensor memory is free, its codes have landed)
+    auto tile_ready = [&](int i) -> bool {
+      const int sa = i % SA, sr = i % SW;
+      if (i >= SA && !mbar_wait(bar_cempty + 8 * sa, (uint32_t)(((i / SA) & 1) ^ 1), abort_flag, p.status)) return false;
+      return mbar_wait(bar_wfull + 8 * sr, (uint32_t)((i / SW) & 1), abort_flag, p.status);
+    };
+    auto publish = [&](int i) {  // by lane 0, after the tile's store has completed
+      const int sa = i % SA, sr = i % SW;
+      if (PAIR) mbar_arrive_cluster(map_to_cta(bar_cfull + 8 * sa, leader_rank)); else mbar_arrive(bar_cfull + 8 * sa);
+      mbar_arrive(bar_wempty + 8 * sr);
+    };
+    // Two tiles at a time: their loads, arithmetic and stores interleave (a warp alone on a tile spent most of its
+    // ~590 cycles waiting for its own shared-memory loads and dependent arithmetic), and the barrier round trips
+    // are shared.
+    int i = 0;
+    const bool two = SW >= 2 && SA >= 2;  // (tile i + 1 must not need the slot or the stage tile i still holds)
+    for (; two && i + 1 < nkb; i += 2) {
+      int got_c = 1;
+      if (lane == 0) got_c = (tile_ready(i) && tile_ready(i + 1)) ? 1 : 0;
+      got_c = __shfl_sync(0xffffffffu, got_c, 0);
+      if (!got_c) break;
+      // lane 0 has observed the phases and the shuffle above orders the other lanes' reads of the tiles after that
+      // (probing the barriers with all 32 lanes as well cost ~420 cycles per tile although they were complete)
+      tc_fence_after();  // the MMAs that read these stages have completed (their commit released them)
+      uint32_t va[32], vb[32];
+      convert_row(i, va);
+      convert_row(i + 1, vb);
+      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(i % SA), va);
+      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col((i + 1) % SA), vb);
+      tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        if (PAIR) mbar_arrive_cluster(map_to_cta(bar_cfull + 8 * sa, leader_rank)); else mbar_arrive(bar_cfull + 8 * sa);
-        mbar_arrive(bar_wempty + 8 * sr);
-      }
+      if (lane == 0) { publish(i); publish(i + 1); }
+    }
+    for (; i < nkb; ++i) {  // an odd last tile (or every tile, with a ring of one)
+      int got_c = 1;
+      if (lane == 0) got_c = tile_ready(i) ? 1 : 0;
+      got_c = __shfl_sync(0xffffffffu, got_c, 0);
+      if (!got_c) break;
+      tc_fence_after();
+      uint32_t va[32];
+      convert_row(i, va);
+      tmem_st32(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(i % SA), va);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) publish(i);
     }
   }
 
