@@ -680,15 +680,20 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         if (PAIR) umma_commit_2cta(bar, (uint16_t)(1u << crank)); else umma_commit(bar);
       };
       bool ok = true;
+      // The loop is bound by what this thread itself executes between two MMAs (the K block's four MMAs need ~685
+      // cycles of tensor time at 256 tokens, the block took ~1080 with operands always ready), so the ring positions,
+      // phases and descriptors advance by increments: no division by the runtime ring depths, no address arithmetic.
+      const int SWm = INT8 ? SC : TS ? SA : SW;  // depth of the ring the MMA's weight operand comes from
+      int sw = 0, sx = 0;
+      uint32_t wph = 0, xph = 0;
+      const uint32_t wf0 = (INT8 || TS) ? bar_cfull : bar_wfull;
+      const uint64_t dw0 = make_smem_desc(smem_u32(INT8 ? smem_c : smem_w)), dx0 = make_smem_desc(smem_u32(smem_x));
+      const uint64_t dw_step = (uint64_t)(W_TILE_BYTES >> 4), dx_step = (uint64_t)(x_bytes >> 4);  // descriptors hold address >> 4
+      uint64_t dw = dw0, dx = dx0;
       for (int i = 0; i < nkb; ++i) {
-        const int sw = INT8 ? i % SC : TS ? i % SA : i % SW, sx = i % SX;
-        const uint32_t wf = (INT8 || TS) ? bar_cfull + 8 * sw : bar_wfull + 8 * sw;
-        const uint32_t wph = (uint32_t)((INT8 ? i / SC : TS ? i / SA : i / SW) & 1);
-        if (!mbar_wait(bar_xfull + 8 * sx, (uint32_t)((i / SX) & 1), abort_flag, p.status) ||
-            !mbar_wait(wf, wph, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_xfull + 8 * sx, xph, abort_flag, p.status) ||
+            !mbar_wait(wf0 + 8 * sw, wph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint64_t dw = make_smem_desc(smem_u32((INT8 ? smem_c : smem_w) + sw * W_TILE_BYTES));
-        const uint64_t dx = make_smem_desc(smem_u32(smem_x + sx * x_bytes));
         if (TS) {  // A operand: the converted tile in tensor memory, 8 columns (16 bf16) per K step
           const uint32_t ta = tmem_base + tmem_a_col(sw);
 #pragma unroll
@@ -711,6 +716,8 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
         }
         commit(((INT8 || TS) ? bar_cempty : bar_wempty) + 8 * sw);
         commit(bar_xempty + 8 * sx);
+        if (++sw == SWm) { sw = 0; wph ^= 1u; dw = dw0; } else { dw += dw_step; }
+        if (++sx == SX) { sx = 0; xph ^= 1u; dx = dx0; } else { dx += dx_step; }
       }
       if (ok && n_ext > 0) {
         // rank term: u tile (x ring item nkb) against the U_B slabs (W0 ring items nkb ..)
