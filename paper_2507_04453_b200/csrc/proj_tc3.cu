@@ -36,7 +36,7 @@ constexpr int W_B_BYTES = W_BOX;
 constexpr int W_STAGE = W_A_BYTES + W_B_BYTES;  // 48 KB
 constexpr int W_STAGES = 4;
 constexpr int W_THREADS = 352;
-constexpr int W_OUT_BOX = 32 * 64 * 2;  // store staging per epilogue warp: 32 token rows x 64 channels (4 KB, 128-byte swizzle)
+constexpr int W_OUT_BOX = 2 * 32 * 32 * 2;  // store staging per epilogue warp: two boxes of 32 token rows x 32 channels (2 KB each, 64-byte swizzle)
 constexpr int W_SMEM = 1024 + W_STAGES * W_STAGE + 8 * W_OUT_BOX + 1024;
 constexpr uint32_t W_TMEM_COLS = 512;  // two 256-column accumulators
 constexpr int W_TILE_M = 512, W_TILE_N = 256;
@@ -242,57 +242,56 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * W_TILE_N);
       const int row0 = m_tile * W_TILE_M + acc * 256 + (int)rank * 128 + quad * 32;  // first token row of this warp
       const int col_base = n_tile * W_TILE_N;
-      // 64 channels at a time: TMEM -> registers (scale, round to bf16) -> this warp's staging box in shared memory in
-      // the 128-byte-swizzled layout -> one TMA store, which writes whole 128-byte lines and clips rows >= T.  (Storing
-      // straight from the row-per-thread registers made every 16-byte store instruction touch 32 different lines
-      // and took 16 k cycles per tile.)  The next chunk's TMEM load is in flight meanwhile.
+      // 32 channels at a time: TMEM -> registers (scale, round to bf16) -> one of this warp's two staging boxes in shared
+      // memory (64-byte-swizzled rows) -> one TMA store, which clips rows >= T.  (Storing straight from the
+      // row-per-thread registers made every 16-byte store instruction touch 32 different lines and took 16 k cycles per
+      // tile.)  The boxes alternate, so a chunk only waits for the store issued two chunks before it to have read its
+      // box, and the next chunk's TMEM load is in flight meanwhile.
       uint32_t ra[32], rb[32];
       tmem_ld32_issue(t_addr, ra);
-      tmem_ld32_issue(t_addr + 32, rb);
-#pragma unroll 1
-      for (int c = 0; c < W_TILE_N / 64; ++c) {
-        const int col0 = col_base + c * 64;
-        tmem_ld_wait();
-        uint32_t pk[32];
+      auto chunk = [&](int c, const uint32_t (&r)[32]) {
+        const int col0 = col_base + c * 32;
+        uint32_t pk[16];
         if (jb.scale != nullptr) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float s0 = (col0 + 2 * i < jb.n_out) ? __half2float(__ldg(jb.scale + col0 + 2 * i)) : 0.f;
             const float s1 = (col0 + 2 * i + 1 < jb.n_out) ? __half2float(__ldg(jb.scale + col0 + 2 * i + 1)) : 0.f;
-            const float t0 = (col0 + 32 + 2 * i < jb.n_out) ? __half2float(__ldg(jb.scale + col0 + 32 + 2 * i)) : 0.f;
-            const float t1 = (col0 + 32 + 2 * i + 1 < jb.n_out) ? __half2float(__ldg(jb.scale + col0 + 32 + 2 * i + 1)) : 0.f;
-            pk[i] = pack_bf16x2(__uint_as_float(ra[2 * i]) * s0, __uint_as_float(ra[2 * i + 1]) * s1);
-            pk[16 + i] = pack_bf16x2(__uint_as_float(rb[2 * i]) * t0, __uint_as_float(rb[2 * i + 1]) * t1);
+            pk[i] = pack_bf16x2(__uint_as_float(r[2 * i]) * s0, __uint_as_float(r[2 * i + 1]) * s1);
           }
         } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            pk[i] = pack_bf16x2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
-            pk[16 + i] = pack_bf16x2(__uint_as_float(rb[2 * i]), __uint_as_float(rb[2 * i + 1]));
-          }
+          for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
         }
-        if (c + 1 < W_TILE_N / 64) {
-          tmem_ld32_issue(t_addr + (c + 1) * 64, ra);
-          tmem_ld32_issue(t_addr + (c + 1) * 64 + 32, rb);
+        const uint32_t box = stg + (uint32_t)((c & 1) * (W_OUT_BOX / 2));
+        if (lane == 0) bulk_wait_group_read1();  // the store issued two chunks ago has read this box
+        __syncwarp();
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4)
+          sts_v4(box + (uint32_t)(lane * 64 + ((j4 ^ ((lane >> 1) & 3)) << 4)), make_uint4(pk[4 * j4], pk[4 * j4 + 1], pk[4 * j4 + 2], pk[4 * j4 + 3]));
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.T && col0 < jb.n_out) {
+          if (p.l2_hints & 4) tma_store_2d_hint(&maps.m[j][5], box, col0, row0, pol_y);
+          else tma_store_2d(&maps.m[j][5], box, col0, row0);
+          bulk_commit_group();
+        }
+      };
+#pragma unroll 1
+      for (int c = 0; c < W_TILE_N / 32; c += 2) {
+        tmem_ld_wait();
+        tmem_ld32_issue(t_addr + (c + 1) * 32, rb);
+        chunk(c, ra);
+        tmem_ld_wait();
+        if (c + 2 < W_TILE_N / 32) {
+          tmem_ld32_issue(t_addr + (c + 2) * 32, ra);
         } else {
           // every TMEM read of this tile is done: the issuer may start the next tile in this accumulator
-          tmem_ld_wait();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * acc);  // 8 warps of the pair release the accumulator
         }
-        if (lane == 0) bulk_wait_group_read0();  // the previous store has read the staging box
-        __syncwarp();
-#pragma unroll
-        for (int j8 = 0; j8 < 8; ++j8)
-          sts_v4(stg + (uint32_t)(lane * 128 + ((j8 ^ (lane & 7)) << 4)), make_uint4(pk[4 * j8], pk[4 * j8 + 1], pk[4 * j8 + 2], pk[4 * j8 + 3]));
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0 && row0 < p.T && col0 < jb.n_out) {
-          if (p.l2_hints & 4) tma_store_2d_hint(&maps.m[j][5], stg, col0, row0, pol_y);
-          else tma_store_2d(&maps.m[j][5], stg, col0, row0);
-          bulk_commit_group();
-        }
+        chunk(c + 1, rb);
       }
     }
     if (lane == 0) bulk_wait_group0();  // the last stores have left shared memory and are written
@@ -356,7 +355,7 @@ int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int 
     maps.m[j][2] = *s.tmA2;
     maps.m[j][3] = *s.tmB2a;
     maps.m[j][4] = *s.tmB2b;
-    const int32_t ms = make_tensor_map_2d(ctx, &maps.m[j][5], 0, s.y, (uint64_t)T, (uint64_t)s.d_out, (uint64_t)s.d_out * 2, 32, 64, 128);
+    const int32_t ms = make_tensor_map_2d(ctx, &maps.m[j][5], 0, s.y, (uint64_t)T, (uint64_t)s.d_out, (uint64_t)s.d_out * 2, 32, 32, 64);
     if (ms != ESSA_OK) return ms;
   }
   for (int j = n_jobs; j < kWideMaxJobs; ++j)
