@@ -84,6 +84,20 @@ def test_block_equals_single_calls_in_structure_and_is_deterministic(torch, ctx)
     case.close()
 
 
+def test_prefill_block_with_odd_channel_counts(torch, ctx):
+    """One base + up launch for projections of 1024 and 1000 channels (1000 = 3.9 channel tiles of 256, not a multiple of
+    the 32-channel store boxes: the last box of a row is clipped) over 2400 tokens."""
+    cfg = wl.scaled_config("2", d_model=1024, d_kv=1000, rank=16, P=6, seg_len=400)
+    case = Case(torch, ctx, cfg)
+    try:
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 2)
+        launches, _, _ = _block(torch, ctx, case)
+        assert launches == len(cfg.projections) + 1
+    finally:
+        ctx.set_option(binding.ESSA_OPT_WIDE_TILES, 1)
+    case.close()
+
+
 def test_prefill_block_is_one_base_up_launch(torch, ctx):
     """A prefill-sized block whose projections all suit the wide pair tiles: four rank-down launches, then ONE launch for
     the base + up step of all four (ragged segments, T = 4348: the last 512-token tile holds 252 rows); with the wide

@@ -197,7 +197,8 @@ def test_scaled_configs_full_outputs(torch, ctx, name):
                                                ("4", 768, 256, 32, 24, 300),    # ragged segments, three channel tiles
                                                ("2", 1024, 256, 33, 13, 197),   # T = 2561: one row in the last tile; padded rank 48
                                                ("5b", 2048, 512, 64, 16, 128),  # INT8 storage: two rank slabs, scale in the epilogue
-                                               ("6b", 2048, 512, 64, 9, 130)])  # INT4 group-wise storage
+                                               ("6b", 2048, 512, 64, 9, 130),   # INT4 group-wise storage
+                                               ("4", 640, 640, 32, 24, 300)])   # 640 channels = 2.5 channel tiles: W0 rows beyond d_out read as zeros, stores clipped
 def test_wide_pair_tiles(torch, ctx, base, dm, dkv, r, P, L):
     """Prefill base + up on 512-token x 256-channel pair tiles (ESSA_OPT_WIDE_TILES = 2) matches the oracle, and the
     256 x 256 pair tiles (ESSA_OPT_WIDE_TILES = 0) to the last bit or so: both add the K blocks in the same order in
