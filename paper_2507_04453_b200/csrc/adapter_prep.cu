@@ -44,35 +44,49 @@ __global__ void build_core_kernel(const __nv_bfloat16* __restrict__ U_A, const _
   M[idx] = acc;
 }
 
-// INT8 codes -> bf16 (exact), 16 codes per thread.  count is a multiple of 64 (d_in is).
-__global__ void widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* __restrict__ out, size_t count) {
-  const size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 16;
-  if (i >= count) return;
-  const uint4 w = *reinterpret_cast<const uint4*>(q + i);
-  uint4 o0, o1;
-  int8x4_to_bf16x4(w.x, o0.x, o0.y);
-  int8x4_to_bf16x4(w.y, o0.z, o0.w);
-  int8x4_to_bf16x4(w.z, o1.x, o1.y);
-  int8x4_to_bf16x4(w.w, o1.z, o1.w);
-  reinterpret_cast<uint4*>(out + i)[0] = o0;
-  reinterpret_cast<uint4*>(out + i)[1] = o1;
-}
-
-// INT4 group-wise codes -> bf16 weights (code * group scale, rounded once), 32 codes (16 bytes) per thread; the 32
-// codes of a thread share a group (groups are 128 wide and d_in is a multiple of 128).
-__global__ void widen_int4_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ gscale, __nv_bfloat16* __restrict__ out,
-                                  int d_in, size_t count) {
-  const size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 32;  // first weight of this thread
-  if (i >= count) return;
-  const size_t o = i / d_in, c = i % d_in;
-  const float s = __half2float(gscale[o * (d_in / 128) + c / 128]);
-  const uint4 w = *reinterpret_cast<const uint4*>(packed + i / 2);
-  const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+// INT8 codes -> bf16 (exact).  A block takes 8192 consecutive codes in four rounds; per round a thread widens eight
+// codes, so a warp's loads (256 B) and stores (512 B) are each one contiguous run.  count is a multiple of 64 (d_in is).
+constexpr int kWidenPerBlock = 8192;
+__global__ void __launch_bounds__(256) widen_int8_kernel(const int8_t* __restrict__ q, __nv_bfloat16* __restrict__ out, size_t count) {
+  const size_t base = (size_t)blockIdx.x * kWidenPerBlock + (size_t)threadIdx.x * 8;
+  uint2 w[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
+    const size_t i = base + (size_t)k * 2048;
+    w[k] = i < count ? __ldg(reinterpret_cast<const uint2*>(q + i)) : make_uint2(0u, 0u);
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const size_t i = base + (size_t)k * 2048;
+    uint4 o;
+    int8x4_to_bf16x4(w[k].x, o.x, o.y);
+    int8x4_to_bf16x4(w[k].y, o.z, o.w);
+    if (i < count) *reinterpret_cast<uint4*>(out + i) = o;
+  }
+}
+
+// INT4 group-wise codes -> bf16 weights (code * group scale, rounded once); same tiling: per round a thread widens the
+// eight codes of four packed bytes, which share a group (groups are 128 wide and d_in is a multiple of 128).
+__global__ void __launch_bounds__(256) widen_int4_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ gscale,
+                                                         __nv_bfloat16* __restrict__ out, int d_in, size_t count) {
+  const size_t base = (size_t)blockIdx.x * kWidenPerBlock + (size_t)threadIdx.x * 8;  // first weight of this thread
+  const int groups = d_in / 128;
+  uint32_t w[4];
+  float s[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const size_t i = base + (size_t)k * 2048;
+    const bool in = i < count;
+    const size_t o = i / d_in, c = i % d_in;
+    w[k] = in ? __ldg(reinterpret_cast<const uint32_t*>(packed + i / 2)) : 0u;
+    s[k] = in ? __half2float(gscale[o * groups + c / 128]) : 0.f;
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const size_t i = base + (size_t)k * 2048;
     uint32_t v[4];
-    int4x8_to_bf16x8(ws[k], s, v);
-    *reinterpret_cast<uint4*>(out + i + 8 * k) = make_uint4(v[0], v[1], v[2], v[3]);
+    int4x8_to_bf16x8(w[k], s[k], v);
+    if (i < count) *reinterpret_cast<uint4*>(out + i) = make_uint4(v[0], v[1], v[2], v[3]);
   }
 }
 
@@ -191,15 +205,14 @@ int32_t launch_widen_int4(essa_ctx* ctx, const uint8_t* packed, const __half* gs
                           cudaStream_t stream) {
   const size_t count = (size_t)d_out * d_in;
   if (count == 0) return ESSA_OK;
-  const size_t threads = count / 32;
-  widen_int4_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(packed, gscale, out, d_in, count);
+  widen_int4_kernel<<<(unsigned)((count + kWidenPerBlock - 1) / kWidenPerBlock), 256, 0, stream>>>(packed, gscale, out, d_in, count);
   ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "widen_int4 launch");
 }
 
 int32_t launch_widen_int8(essa_ctx* ctx, const int8_t* q, __nv_bfloat16* out, size_t count, cudaStream_t stream) {
-  const size_t threads = (count + 15) / 16;
-  widen_int8_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(q, out, count);
+  if (count == 0) return ESSA_OK;
+  widen_int8_kernel<<<(unsigned)((count + kWidenPerBlock - 1) / kWidenPerBlock), 256, 0, stream>>>(q, out, count);
   ctx->launches += 1;
   return check_cuda(ctx, cudaGetLastError(), "widen_int8 launch");
 }

@@ -4,16 +4,19 @@
 // The launch reads x once and is bound by HBM, so what matters is that every SM streams the same number of bytes and
 // that neither the tensor core nor the threads that issue the copies hold the stream back.  (a) Balance: the token rows
 // of all jobs form one list of 64-row units; pair p of the persistent grid owns units [p U / n_pairs, (p + 1) U / n_pairs)
-// and walks them in tiles of up to four units (256 rows: M = 256 across the pair, each CTA holding up to two units);
-// boxes beyond a pair's range are not loaded.  The 128-row tiles of the single-CTA kernel left the grid's last round a
-// quarter idle (257 tiles on 148 SMs).  (b) Tensor time: one tcgen05.mma.cta_group::2 covers 256 token rows, half the
-// MMAs per byte of x of the M = 128 kernel, whose narrow MMAs (N = r_pad) cost ~150 cycles each whatever N is.
+// and walks them in tiles of up to eight units (512 rows: two halves of M = 256 across the pair, each CTA holding up to
+// two units of either half); boxes beyond a pair's range are not loaded.  The 128-row tiles of the single-CTA kernel
+// left the grid's last round a quarter idle (257 tiles on 148 SMs).  (b) Tensor time: one tcgen05.mma.cta_group::2
+// covers 256 token rows, half the MMAs per byte of x of the M = 128 kernel, whose narrow MMAs (N = r_pad) cost ~150
+// cycles each whatever N is; and a K block's eight MMAs fill the two halves' accumulators in turn before one commit,
+// which the tensor core takes at twice the rate of four MMAs into one accumulator + commit (rank-down launch of four
+// 1536-wide projections at 81920 tokens: 102 -> 96 us; of four 3584-wide ones at 163840 tokens: 302 -> 270 us).
 // (c) Several threads issue the copies, the K blocks in turn.
 //
-// Per K block (64 wide) a CTA loads its units of x (one 128-row box, or one 64-row box at the end of its range) and its
-// half of the V_A^T tile (r_pad / 2 rows); the leader issues four MMAs of M = 256, N = r_pad into one of two
-// accumulator buffers, so the epilogue of a tile (per token row in registers: sA, the r x r core M, sB; u stored as
-// bf16) overlaps the next tile's K loop.
+// Per K block (64 wide) a CTA loads its units of x (per half one 128-row box, or one 64-row box at the end of its
+// range) and its half of the V_A^T tile (r_pad / 2 rows); the leader issues per half four MMAs of M = 256, N = r_pad
+// into that half's accumulator of one of two buffers, so the epilogue of a tile (per token row in registers: sA, the
+// r x r core M, sB; u stored as bf16) overlaps the next tile's K loop.
 //
 // Warp roles per CTA (320 threads): warps 0 and 6..9 = TMA producers, warp 1 = TMEM allocator (+ MMA issuer in the
 // leader), warps 2..5 = epilogue.  Barriers as in the other pair kernels: `full` in the leader (bytes of both CTAs),
@@ -27,10 +30,11 @@ namespace {
 
 constexpr int D_UNIT_ROWS = 64;
 constexpr int D_UNIT_BYTES = D_UNIT_ROWS * 64 * 2;  // 8 KB: 64 rows x 64 bf16
-constexpr int D_A_BYTES = 2 * D_UNIT_BYTES;         // a CTA's two units
+constexpr int D_HALF_BYTES = 2 * D_UNIT_BYTES;      // a CTA's two units of one half of the tile (one 128-row operand)
+constexpr int D_A_BYTES = 2 * D_HALF_BYTES;         // both halves
 constexpr int D_THREADS = 320;
 constexpr int D_PRODUCERS = 5;
-constexpr uint32_t D_TMEM_COLS = 128;  // two accumulator buffers of up to 64 columns
+constexpr uint32_t D_TMEM_COLS = 256;  // two buffers x two halves, accumulators of up to 64 columns
 __host__ __device__ constexpr int d_v_bytes(int rp) { return rp * 64; }  // rp / 2 rows x 128 B
 __host__ __device__ constexpr int d_stages(int rp) {
   return (227 * 1024 - 2048) / (D_A_BYTES + d_v_bytes(rp)) > 10 ? 10 : (227 * 1024 - 2048) / (D_A_BYTES + d_v_bytes(rp));
@@ -88,7 +92,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
     j = (int)(g / p.units_per_job);
     const int ju = (int)(g - (long long)j * p.units_per_job);
     long long n = u_end - g;
-    if (n > 4) n = 4;
+    if (n > 8) n = 8;
     if (n > p.units_per_job - ju) n = p.units_per_job - ju;
     n_units = (int)n;
     row0 = ju * D_UNIT_ROWS;
@@ -128,7 +132,8 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
         tile_at(g, j, row0, n_units);
         g += n_units;
         const int main_kb = p.job[j].main_kb;
-        const int mine = n_units - 2 * (int)rank;  // units of this CTA: tile units 2 rank, 2 rank + 1
+        // units of this CTA: tile units 2 rank, 2 rank + 1 (first half of the tile) and 4 + 2 rank, 5 + 2 rank (second half)
+        const int mine0 = n_units - 2 * (int)rank, mine1 = n_units - 4 - 2 * (int)rank;
         const int row_mine = row0 + 2 * (int)rank * D_UNIT_ROWS;
         for (int kb = 0; kb < main_kb; ++kb, ++seq) {
           if ((int)(seq % p.n_producers) != pi) continue;
@@ -138,8 +143,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
           if (leader) mbar_expect_tx(bar_full + 8 * stage, (uint32_t)(n_units * D_UNIT_BYTES + 2 * V_BYTES));
           const uint32_t fb = full_leader + 8 * stage;
           const uint32_t da = smem_u32(smem + stage * STAGE);
-          if (mine > 1) tma_load_2d_pair(da, &maps.x2[j], kb * 64, row_mine, fb);
-          else if (mine > 0) tma_load_2d_pair(da, &maps.x[j], kb * 64, row_mine, fb);
+          if (mine0 > 1) tma_load_2d_pair(da, &maps.x2[j], kb * 64, row_mine, fb);
+          else if (mine0 > 0) tma_load_2d_pair(da, &maps.x[j], kb * 64, row_mine, fb);
+          if (mine1 > 1) tma_load_2d_pair(da + D_HALF_BYTES, &maps.x2[j], kb * 64, row_mine + 4 * D_UNIT_ROWS, fb);
+          else if (mine1 > 0) tma_load_2d_pair(da + D_HALF_BYTES, &maps.x[j], kb * 64, row_mine + 4 * D_UNIT_ROWS, fb);
           tma_load_2d_pair(da + D_A_BYTES, &maps.v[j], kb * 64, (int)rank * (RP / 2), fb);
           ++issued;
         }
@@ -167,23 +174,27 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
         const int buf = it & 1;
         if (!mbar_wait(bar_tempty + 8 * buf, (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 64);
+        const uint32_t d0 = tmem_base + (uint32_t)(buf * 128), d1 = d0 + 64u;  // the tile's two halves
+        const bool two = n_units > 4;
         for (int kb = 0; kb < main_kb; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE);
-          // the CTA's two units are consecutive 64-row boxes: one 128-row K-major operand
-          const uint64_t a_desc = make_smem_desc(sa), v_desc = make_smem_desc(sa + D_A_BYTES);
-          if (kb > 0) {  // straight-line: the issuing thread's own instructions between two MMAs count
-            umma_bf16_2cta(d_tmem, a_desc, v_desc, idesc, 1u);
-            umma_bf16_2cta(d_tmem, a_desc + 2, v_desc + 2, idesc, 1u);
-            umma_bf16_2cta(d_tmem, a_desc + 4, v_desc + 4, idesc, 1u);
-            umma_bf16_2cta(d_tmem, a_desc + 6, v_desc + 6, idesc, 1u);
-          } else {
-            umma_bf16_2cta(d_tmem, a_desc, v_desc, idesc, 0u);
-            umma_bf16_2cta(d_tmem, a_desc + 2, v_desc + 2, idesc, 1u);
-            umma_bf16_2cta(d_tmem, a_desc + 4, v_desc + 4, idesc, 1u);
-            umma_bf16_2cta(d_tmem, a_desc + 6, v_desc + 6, idesc, 1u);
+          // a CTA's two units of a half are consecutive 64-row boxes: one 128-row K-major operand per half
+          const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + D_HALF_BYTES), v_desc = make_smem_desc(sa + D_A_BYTES);
+          const uint32_t acc = kb > 0 ? 1u : 0u;
+          // straight-line (the issuing thread's own instructions between two MMAs count); four MMAs into the first half's
+          // accumulator, then four into the second's: filling two accumulators in turn before the commit runs at the
+          // tensor cores' rate, four MMAs into one accumulator + commit do not (~840 cycles instead of 512)
+          umma_bf16_2cta(d0, a0, v_desc, idesc, acc);
+          umma_bf16_2cta(d0, a0 + 2, v_desc + 2, idesc, 1u);
+          umma_bf16_2cta(d0, a0 + 4, v_desc + 4, idesc, 1u);
+          umma_bf16_2cta(d0, a0 + 6, v_desc + 6, idesc, 1u);
+          if (two) {
+            umma_bf16_2cta(d1, a1, v_desc, idesc, acc);
+            umma_bf16_2cta(d1, a1 + 2, v_desc + 2, idesc, 1u);
+            umma_bf16_2cta(d1, a1 + 4, v_desc + 4, idesc, 1u);
+            umma_bf16_2cta(d1, a1 + 6, v_desc + 6, idesc, 1u);
           }
           umma_commit_2cta(bar_empty + 8 * stage, 3);  // the stage is free in both CTAs
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -213,51 +224,57 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
       if (!got) break;
       while (!mbar_try_wait(bar_tfull + 8 * buf, (uint32_t)((it >> 1) & 1))) {}  // complete: acquire for every lane
       tc_fence_after();
-      const uint32_t p_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 64);
-      float q[RP];
+      const int halves = n_units > 4 ? 2 : 1;
+#pragma unroll 1
+      for (int hf = 0; hf < halves; ++hf) {
+        const uint32_t p_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 128 + hf * 64);
+        float q[RP];
 #pragma unroll
-      for (int c = 0; c < RP / 16; ++c) {
-        float v[16];
-        tmem_ld16(p_addr + c * 16, v);
+        for (int c = 0; c < RP / 16; ++c) {
+          float v[16];
+          tmem_ld16(p_addr + c * 16, v);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) q[c * 16 + i] = v[i];
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);  // the buffer may take the tile after next
-      const int unit_in_tile = 2 * (int)rank + row_in_cta / D_UNIT_ROWS;
-      const int t = row0 + (int)rank * 128 + row_in_cta;
-      if (unit_in_tile < n_units && t < p.T) {
-        const int k = find_candidate(p.seg, p.P, t);
-        const float* srow = p.sigma + (size_t)k * p.ld_sigma;
-#pragma unroll
-        for (int i = 0; i < RP; ++i) q[i] = (i < jb.r) ? q[i] * __ldg(srow + jb.sA_col + i) : 0.f;
-        uint32_t packed[kRankPadMax / 2];
-#pragma unroll
-        for (int j2 = 0; j2 < RP / 2; ++j2) {
-          float uu[2];
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int jj = 2 * j2 + h;
-            float acc = 0.f;
-#pragma unroll
-            for (int i4 = 0; i4 < RP / 4; ++i4) {
-              const float4 mm = __ldg(reinterpret_cast<const float4*>(jb.M + jj * kRankPadMax) + i4);  // same address in every lane
-              acc = fmaf(mm.x, q[4 * i4], acc);
-              acc = fmaf(mm.y, q[4 * i4 + 1], acc);
-              acc = fmaf(mm.z, q[4 * i4 + 2], acc);
-              acc = fmaf(mm.w, q[4 * i4 + 3], acc);
-            }
-            uu[h] = (jj < jb.r) ? acc * __ldg(srow + jb.sB_col + jj) : 0.f;
-          }
-          packed[j2] = pack_bf16x2(uu[0], uu[1]);
+          for (int i = 0; i < 16; ++i) q[c * 16 + i] = v[i];
         }
+        if (hf == halves - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);  // the buffer may take the tile after next
+        }
+        const int unit_in_tile = 4 * hf + 2 * (int)rank + row_in_cta / D_UNIT_ROWS;
+        const int t = row0 + hf * 256 + (int)rank * 128 + row_in_cta;
+        if (unit_in_tile < n_units && t < p.T) {
+          const int k = find_candidate(p.seg, p.P, t);
+          const float* srow = p.sigma + (size_t)k * p.ld_sigma;
 #pragma unroll
-        for (int j2 = RP / 2; j2 < kRankPadMax / 2; ++j2) packed[j2] = 0u;
-        uint4* dst = reinterpret_cast<uint4*>(jb.u + (size_t)t * kRankPadMax);
+          for (int i = 0; i < RP; ++i) q[i] = (i < jb.r) ? q[i] * __ldg(srow + jb.sA_col + i) : 0.f;
+          uint32_t packed[kRankPadMax / 2];
 #pragma unroll
-        for (int gq = 0; gq < kRankPadMax / 8; ++gq)
-          dst[gq] = make_uint4(packed[4 * gq], packed[4 * gq + 1], packed[4 * gq + 2], packed[4 * gq + 3]);
+          for (int j2 = 0; j2 < RP / 2; ++j2) {
+            float uu[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int jj = 2 * j2 + h;
+              float acc = 0.f;
+#pragma unroll
+              for (int i4 = 0; i4 < RP / 4; ++i4) {
+                const float4 mm = __ldg(reinterpret_cast<const float4*>(jb.M + jj * kRankPadMax) + i4);  // same address in every lane
+                acc = fmaf(mm.x, q[4 * i4], acc);
+                acc = fmaf(mm.y, q[4 * i4 + 1], acc);
+                acc = fmaf(mm.z, q[4 * i4 + 2], acc);
+                acc = fmaf(mm.w, q[4 * i4 + 3], acc);
+              }
+              uu[h] = (jj < jb.r) ? acc * __ldg(srow + jb.sB_col + jj) : 0.f;
+            }
+            packed[j2] = pack_bf16x2(uu[0], uu[1]);
+          }
+#pragma unroll
+          for (int j2 = RP / 2; j2 < kRankPadMax / 2; ++j2) packed[j2] = 0u;
+          uint4* dst = reinterpret_cast<uint4*>(jb.u + (size_t)t * kRankPadMax);
+#pragma unroll
+          for (int gq = 0; gq < kRankPadMax / 8; ++gq)
+            dst[gq] = make_uint4(packed[4 * gq], packed[4 * gq + 1], packed[4 * gq + 2], packed[4 * gq + 3]);
+        }
       }
     }
   }
