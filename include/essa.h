@@ -135,6 +135,10 @@ int32_t essa_get_status(essa_ctx* ctx, int32_t* device_status);
  *   the value is the number of threads per CTA that issue its TMA copies in turn.  0 keeps one single-CTA launch of
  *   128-token tiles per projection. */
 #define ESSA_OPT_DOWN_PAIRS 10
+/*   ESSA_OPT_DOWN_TILE_UNITS (0 .. 8, default 0): the most 64-row units a tile of the CTA-pair rank-down kernel takes
+ *   (up to 4: one accumulator per tile; 5 .. 8: two).  0 picks 8 where every pair gets at least twelve units and 4
+ *   otherwise (for measurements). */
+#define ESSA_OPT_DOWN_TILE_UNITS 11
 int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value);
 /* Number of kernels of this library enqueued through ctx since it was created (host counter). */
 int32_t essa_get_launch_count(essa_ctx* ctx, int64_t* launches);

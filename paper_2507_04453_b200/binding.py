@@ -36,6 +36,7 @@ ESSA_OPT_WIDE_TILES = 7
 ESSA_OPT_DOWN_SPLITS = 8
 ESSA_OPT_L2_HINTS = 9
 ESSA_OPT_DOWN_PAIRS = 10
+ESSA_OPT_DOWN_TILE_UNITS = 11
 
 EXPORTED_SYMBOLS = (
     "essa_version", "essa_status_string", "essa_create", "essa_destroy", "essa_last_error", "essa_get_status",

@@ -270,6 +270,10 @@ int32_t essa_set_option(essa_ctx* ctx, int32_t option, int32_t value) {
       if (value < 0 || value > 5) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_DOWN_PAIRS takes 0 .. 5");
       ctx->down_pairs = value;
       return ESSA_OK;
+    case ESSA_OPT_DOWN_TILE_UNITS:
+      if (value < 0 || value > 8) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_DOWN_TILE_UNITS takes 0 .. 8");
+      ctx->down_tile_units = value;
+      return ESSA_OK;
     case ESSA_OPT_L2_HINTS:
       if (value < 0 || value > 0xffff) return fail(ctx, ESSA_ERR_INVALID_ARG, "set_option: ESSA_OPT_L2_HINTS takes 0 .. 65535");
       ctx->l2_hints = value;

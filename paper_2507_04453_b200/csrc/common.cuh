@@ -38,6 +38,7 @@ struct essa_ctx {
   bool decode_pairs = false;  // ESSA_OPT_DECODE_PAIRS
   bool down_ctas = true;      // ESSA_OPT_DECODE_DOWN_CTAS
   bool pair_tiles = true;       // prefill base + up on 256 x 256 CTA-pair tiles (essa_set_option)
+  int down_tile_units = 0;      // most 64-row units per tile of that kernel: 0 = automatic, 1..8 (essa_set_option)
   int down_pairs = 5;           // prefill rank-down step on CTA pairs: 0 = off, 1..5 = TMA-issuing threads per CTA (essa_set_option)
   int l2_hints = 13;            // L2 eviction hints of the wide prefill kernel's TMA copies (essa_set_option)
   int down_splits = 0;          // K split of the prefill rank-down launch: 0 = the planner's choice (essa_set_option)

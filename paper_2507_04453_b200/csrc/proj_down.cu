@@ -5,12 +5,14 @@
 // that neither the tensor core nor the threads that issue the copies hold the stream back.  (a) Balance: the token rows
 // of all jobs form one list of 64-row units; pair p of the persistent grid owns units [p U / n_pairs, (p + 1) U / n_pairs)
 // and walks them in tiles of up to eight units (512 rows: two halves of M = 256 across the pair, each CTA holding up to
-// two units of either half); boxes beyond a pair's range are not loaded.  The 128-row tiles of the single-CTA kernel
+// two units of either half) where it has at least twelve units, of up to four otherwise (one half; the ring is then
+// twice as deep); boxes beyond a pair's range are not loaded.  The 128-row tiles of the single-CTA kernel
 // left the grid's last round a quarter idle (257 tiles on 148 SMs).  (b) Tensor time: one tcgen05.mma.cta_group::2
 // covers 256 token rows, half the MMAs per byte of x of the M = 128 kernel, whose narrow MMAs (N = r_pad) cost ~150
 // cycles each whatever N is; and a K block's eight MMAs fill the two halves' accumulators in turn before one commit,
 // which the tensor core takes at twice the rate of four MMAs into one accumulator + commit (rank-down launch of four
-// 1536-wide projections at 81920 tokens: 102 -> 96 us; of four 3584-wide ones at 163840 tokens: 302 -> 270 us).
+// 3584-wide inputs at 16384 tokens: 102 -> 96 us; of four 5120-wide ones at 35462 tokens: 302 -> 270 us; with fewer
+// than twelve units per pair the 256-row tiles measured faster: 63 against 73 us at 8192 tokens).
 // (c) Several threads issue the copies, the K blocks in turn.
 //
 // Per K block (64 wide) a CTA loads its units of x (per half one 128-row box, or one 64-row box at the end of its
@@ -36,10 +38,12 @@ constexpr int D_THREADS = 320;
 constexpr int D_PRODUCERS = 5;
 constexpr uint32_t D_TMEM_COLS = 256;  // two buffers x two halves, accumulators of up to 64 columns
 __host__ __device__ constexpr int d_v_bytes(int rp) { return rp * 64; }  // rp / 2 rows x 128 B
-__host__ __device__ constexpr int d_stages(int rp) {
-  return (227 * 1024 - 2048) / (D_A_BYTES + d_v_bytes(rp)) > 10 ? 10 : (227 * 1024 - 2048) / (D_A_BYTES + d_v_bytes(rp));
+// ring depth for stages that hold one half (tiles of up to four units) or both; the shared memory is the same either way
+constexpr int D_MAX_STAGES = 12;
+__host__ __device__ constexpr int d_stages(int rp, int a_bytes) {
+  return (227 * 1024 - 2048) / (a_bytes + d_v_bytes(rp)) > D_MAX_STAGES ? D_MAX_STAGES : (227 * 1024 - 2048) / (a_bytes + d_v_bytes(rp));
 }
-__host__ __device__ constexpr int d_smem(int rp) { return 1024 + d_stages(rp) * (D_A_BYTES + d_v_bytes(rp)) + 1024; }
+constexpr int d_smem() { return 227 * 1024; }
 
 struct DnMaps {
   CUtensorMap x[kWideMaxJobs];   // boxes of 64 rows x 64 columns
@@ -54,7 +58,7 @@ struct DnJob {
 };
 
 struct DnParams {
-  int T, units_per_job, n_jobs, n_producers;
+  int T, units_per_job, n_jobs, n_producers, max_units;
   long long total_units;
   DnJob job[kWideMaxJobs];
   const int32_t* seg;
@@ -66,9 +70,10 @@ struct DnParams {
 
 template <int RP>
 __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_constant__ DnMaps maps, const DnParams p) {
-  constexpr int STAGES = d_stages(RP);
   constexpr int V_BYTES = d_v_bytes(RP);
-  constexpr int STAGE = D_A_BYTES + V_BYTES;
+  const int A_BYTES = p.max_units > 4 ? D_A_BYTES : D_HALF_BYTES;  // a stage's x part: both halves of a tile, or one
+  const int STAGES = d_stages(RP, A_BYTES);
+  const int STAGE = A_BYTES + V_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* aux = smem + STAGES * STAGE;
@@ -92,7 +97,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
     j = (int)(g / p.units_per_job);
     const int ju = (int)(g - (long long)j * p.units_per_job);
     long long n = u_end - g;
-    if (n > 8) n = 8;
+    if (n > p.max_units) n = p.max_units;
     if (n > p.units_per_job - ju) n = p.units_per_job - ju;
     n_units = (int)n;
     row0 = ju * D_UNIT_ROWS;
@@ -147,7 +152,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
           else if (mine0 > 0) tma_load_2d_pair(da, &maps.x[j], kb * 64, row_mine, fb);
           if (mine1 > 1) tma_load_2d_pair(da + D_HALF_BYTES, &maps.x2[j], kb * 64, row_mine + 4 * D_UNIT_ROWS, fb);
           else if (mine1 > 0) tma_load_2d_pair(da + D_HALF_BYTES, &maps.x[j], kb * 64, row_mine + 4 * D_UNIT_ROWS, fb);
-          tma_load_2d_pair(da + D_A_BYTES, &maps.v[j], kb * 64, (int)rank * (RP / 2), fb);
+          tma_load_2d_pair(da + A_BYTES, &maps.v[j], kb * 64, (int)rank * (RP / 2), fb);
           ++issued;
         }
       }
@@ -181,7 +186,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) essa_down_kernel(const __grid_co
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE);
           // a CTA's two units of a half are consecutive 64-row boxes: one 128-row K-major operand per half
-          const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + D_HALF_BYTES), v_desc = make_smem_desc(sa + D_A_BYTES);
+          const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + D_HALF_BYTES), v_desc = make_smem_desc(sa + A_BYTES);
           const uint32_t acc = kb > 0 ? 1u : 0u;
           // straight-line (the issuing thread's own instructions between two MMAs count); four MMAs into the first half's
           // accumulator, then four into the second's: filling two accumulators in turn before the commit runs at the
@@ -294,14 +299,14 @@ int32_t launch_down(essa_ctx* ctx, const DnMaps& maps, const DnParams& p, int pa
   static bool attr_done[64] = {};  // the attribute is per device
   bool& done = attr_done[(ctx->device >= 0 && ctx->device < 64) ? ctx->device : 0];
   if (!done) {
-    const cudaError_t ea = cudaFuncSetAttribute(essa_down_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize, d_smem(RP));
+    const cudaError_t ea = cudaFuncSetAttribute(essa_down_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize, d_smem());
     if (ea != cudaSuccess) return check_cuda(ctx, ea, "cudaFuncSetAttribute(essa_down_kernel)");
     done = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
   cfg.blockDim = dim3(D_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)d_smem(RP);
+  cfg.dynamicSmemBytes = (size_t)d_smem();
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -340,6 +345,10 @@ int32_t launch_rank_down_pairs(essa_ctx* ctx, const DownJob* jobs, int n_jobs, i
   p.n_jobs = n_jobs;
   p.n_producers = ctx->down_pairs > D_PRODUCERS ? D_PRODUCERS : ctx->down_pairs;
   p.total_units = (long long)n_jobs * p.units_per_job;
+  {
+    const int pairs_dev = (ctx->sm_count > 0 ? ctx->sm_count : 148) / 2;
+    p.max_units = ctx->down_tile_units > 0 ? ctx->down_tile_units : (p.total_units >= 12LL * pairs_dev ? 8 : 4);
+  }
   p.seg = seg;
   p.P = P;
   p.sigma = sigma;

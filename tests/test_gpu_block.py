@@ -120,16 +120,18 @@ def test_prefill_block_is_one_base_up_launch(torch, ctx):
 
 @pytest.mark.parametrize("base,dm,dkv,r,P,L,pairs", [("4", 512, 512, 32, 40, 1000, True),    # ragged, T = 21 394: 335 units of 64 rows per projection
                                                      ("2", 512, 512, 16, 30, 650, True),     # T = 19 500
+                                                     ("2", 512, 512, 16, 16, 500, True),     # T = 8 000: fewer than twelve units per pair, 256-row tiles
                                                      ("5c", 512, 512, 17, 150, 256, True),   # INT8 storage (one call per projection), padded rank 32, mixed lengths
                                                      ("2", 512, 512, 33, 30, 650, False)])   # padded rank 48: stays on the single-CTA kernel
 def test_rank_down_on_cta_pairs(torch, ctx, base, dm, dkv, r, P, L, pairs):
     """Prefill-sized block with enough tokens for the CTA-pair rank-down kernel (every pair of the grid gets at least four
     64-row units; the last tile of a pair's range is partial): bf16 blocks run ONE rank-down launch and ONE base + up
     launch.  The result matches the oracle and, to the last bit or so, the single-CTA rank-down launches
-    (ESSA_OPT_DOWN_PAIRS = 0), which add the same K blocks in the same order."""
+    (ESSA_OPT_DOWN_PAIRS = 0), which add the same K blocks in the same order; 256-row and 512-row tiles
+    (ESSA_OPT_DOWN_TILE_UNITS) give the same bits."""
     cfg = wl.scaled_config(base, d_model=dm, d_kv=dkv, rank=r, P=P, seg_len=L)
     case = Case(torch, ctx, cfg)
-    assert (case.T + 63) // 64 >= 4 * 74
+    assert len(cfg.projections) * ((case.T + 63) // 64) >= 4 * 74
     cands = wl.stratified_candidates(cfg, case.offsets)[:10]
     n = len(cfg.projections)
     bf16 = cfg.w0_dtype == "bf16"
@@ -137,6 +139,13 @@ def test_rank_down_on_cta_pairs(torch, ctx, base, dm, dkv, r, P, L, pairs):
         launches, xs, ys = _block(torch, ctx, case, cands)
         # quantised storage: dequantisation pass, rank-down, base + up per projection
         assert launches == ((2 if pairs else n + 1) if bf16 else 3 * n)
+        if pairs:
+            for units in (3, 4, 8):
+                ctx.set_option(binding.ESSA_OPT_DOWN_TILE_UNITS, units)
+                _, _, ys_u = _block(torch, ctx, case, cands)
+                for a, b in zip(ys, ys_u):
+                    assert torch.equal(a, b), units
+            ctx.set_option(binding.ESSA_OPT_DOWN_TILE_UNITS, 0)
         ctx.set_option(binding.ESSA_OPT_DOWN_PAIRS, 0)
         launches0, _, ys0 = _block(torch, ctx, case, cands)
         assert launches0 == (n + 1 if bf16 else 3 * n)
@@ -145,6 +154,7 @@ def test_rank_down_on_cta_pairs(torch, ctx, base, dm, dkv, r, P, L, pairs):
             assert np.mean(a != b) < 0.01 and orc.relative_error(a, b.astype(np.float64)) <= 8e-3
     finally:
         ctx.set_option(binding.ESSA_OPT_DOWN_PAIRS, 5)
+        ctx.set_option(binding.ESSA_OPT_DOWN_TILE_UNITS, 0)
     case.close()
 
 
