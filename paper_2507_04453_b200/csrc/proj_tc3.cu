@@ -36,7 +36,7 @@ constexpr int W_B_BYTES = W_BOX;
 constexpr int W_STAGE = W_A_BYTES + W_B_BYTES;  // 48 KB
 constexpr int W_STAGES = 4;
 constexpr int W_THREADS = 352;
-constexpr int W_OUT_BOX = 2 * 32 * 32 * 2;  // store staging per epilogue warp: two boxes of 32 token rows x 32 channels (2 KB each, 64-byte swizzle)
+constexpr int W_OUT_BOX = 32 * 64 * 2;  // store staging per epilogue warp: one box of 32 token rows x 64 channels (4 KB, 128-byte swizzle)
 constexpr int W_SMEM = 1024 + W_STAGES * W_STAGE + 8 * W_OUT_BOX + 1024;
 constexpr uint32_t W_TMEM_COLS = 512;  // two 256-column accumulators
 constexpr int W_TILE_M = 512, W_TILE_N = 256;
@@ -242,11 +242,11 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * W_TILE_N);
       const int row0 = m_tile * W_TILE_M + acc * 256 + (int)rank * 128 + quad * 32;  // first token row of this warp
       const int col_base = n_tile * W_TILE_N;
-      // 32 channels at a time: TMEM -> registers (scale, round to bf16) -> one of this warp's two staging boxes in shared
-      // memory (64-byte-swizzled rows) -> one TMA store, which clips rows >= T.  (Storing straight from the
-      // row-per-thread registers made every 16-byte store instruction touch 32 different lines and took 16 k cycles per
-      // tile.)  The boxes alternate, so a chunk only waits for the store issued two chunks before it to have read its
-      // box, and the next chunk's TMEM load is in flight meanwhile.
+      // 32 channels at a time: TMEM -> registers (scale, round to bf16) -> this warp's staging box in shared memory
+      // (128-byte-swizzled rows of 64 channels); every second chunk completes the box -> one TMA store, which clips
+      // rows >= T and channels >= n_out.  (Storing straight from the row-per-thread registers made every 16-byte store
+      // instruction touch 32 different lines and took 16 k cycles per tile.)  The next chunk's TMEM load is in flight
+      // while a chunk is packed and staged; a box is refilled once the store before has read it.
       uint32_t ra[32], rb[32];
       tmem_ld32_issue(t_addr, ra);
       auto chunk = [&](int c, const uint32_t (&r)[32]) {
@@ -263,18 +263,22 @@ __global__ void __launch_bounds__(W_THREADS, 1) essa_tcw_kernel(const __grid_con
 #pragma unroll
           for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
         }
-        const uint32_t box = stg + (uint32_t)((c & 1) * (W_OUT_BOX / 2));
-        if (lane == 0) bulk_wait_group_read1();  // the store issued two chunks ago has read this box
-        __syncwarp();
+        const int half = c & 1;
+        if (half == 0) {
+          if (lane == 0) bulk_wait_group_read0();  // the store before has read the box
+          __syncwarp();
+        }
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4)
-          sts_v4(box + (uint32_t)(lane * 64 + ((j4 ^ ((lane >> 1) & 3)) << 4)), make_uint4(pk[4 * j4], pk[4 * j4 + 1], pk[4 * j4 + 2], pk[4 * j4 + 3]));
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0 && row0 < p.T && col0 < jb.n_out) {
-          if (p.l2_hints & 4) tma_store_2d_hint(&maps.m[j][5], box, col0, row0, pol_y);
-          else tma_store_2d(&maps.m[j][5], box, col0, row0);
-          bulk_commit_group();
+          sts_v4(stg + (uint32_t)(lane * 128 + (((half * 4 + j4) ^ (lane & 7)) << 4)), make_uint4(pk[4 * j4], pk[4 * j4 + 1], pk[4 * j4 + 2], pk[4 * j4 + 3]));
+        if (half == 1) {
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && row0 < p.T && col0 - 32 < jb.n_out) {
+            if (p.l2_hints & 4) tma_store_2d_hint(&maps.m[j][5], stg, col0 - 32, row0, pol_y);
+            else tma_store_2d(&maps.m[j][5], stg, col0 - 32, row0);
+            bulk_commit_group();
+          }
         }
       };
 #pragma unroll 1
@@ -355,7 +359,7 @@ int32_t launch_base_up_wide(essa_ctx* ctx, const WideJob* jobs, int n_jobs, int 
     maps.m[j][2] = *s.tmA2;
     maps.m[j][3] = *s.tmB2a;
     maps.m[j][4] = *s.tmB2b;
-    const int32_t ms = make_tensor_map_2d(ctx, &maps.m[j][5], 0, s.y, (uint64_t)T, (uint64_t)s.d_out, (uint64_t)s.d_out * 2, 32, 32, 64);
+    const int32_t ms = make_tensor_map_2d(ctx, &maps.m[j][5], 0, s.y, (uint64_t)T, (uint64_t)s.d_out, (uint64_t)s.d_out * 2, 32, 64, 128);
     if (ms != ESSA_OK) return ms;
   }
   for (int j = n_jobs; j < kWideMaxJobs; ++j)
