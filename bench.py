@@ -48,9 +48,9 @@ CSRC = os.path.join(ROOT, "paper_2507_04453_b200", "csrc")
 # with the SHA-256 (first 16 hex digits) of the kernel's source file at capture time: a kernel that has changed
 # since reports "traffic": null until it is captured again.
 NCU_TRAFFIC = {
-    "2": {"bytes": 797e6, "source": "proj_tc3.cu", "sha16": "6d717f97da3af328", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
-          "note": "captured at half the population (427.7 MB) and scaled: W0 traffic fixed, x and y traffic doubled"},
-    "4": {"bytes": 4592e6, "source": "proj_tc3.cu", "sha16": "6d717f97da3af328", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
+    "2": {"bytes": 792e6, "source": "proj_tc3.cu", "sha16": "13fd60855285679d", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
+          "note": "captured at half the population (425.2 MB) and scaled: W0 traffic fixed, x and y traffic doubled"},
+    "4": {"bytes": 4787e6, "source": "proj_tc3.cu", "sha16": "13fd60855285679d", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
           "note": "full size; captures of the same kernel range from 3.4 to 5.4 GB (how well the CTA pairs stay in step)"},
     "3": {"bytes": 67.9e6, "source": "proj_decode.cu", "sha16": "cbe5056142bb8d7c", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
     "5a": {"bytes": 170.6e6, "source": "proj_decode.cu", "sha16": "cbe5056142bb8d7c", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
