@@ -889,12 +889,19 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     int i = 0;
     const bool two = SW >= 2 && SA >= 2;  // (tile i + 1 must not need the slot or the stage tile i still holds)
     for (; two && i + 1 < nkb; i += 2) {
+      // lanes 0..3 observe the four barriers of the two tiles side by side (free stages of tensor memory, landed codes:
+      // one lane taking them in turn spent ~100 cycles on each although they were complete); the vote orders the other
+      // lanes' reads of the tiles after that.  (Probing the barriers with all 32 lanes cost ~420 cycles per tile.)
       int got_c = 1;
-      if (lane == 0) got_c = (tile_ready(i) && tile_ready(i + 1)) ? 1 : 0;
-      got_c = __shfl_sync(0xffffffffu, got_c, 0);
+      if (lane < 4) {
+        const int ti = i + (lane & 1);
+        const bool stage_free = lane >= 2;  // lanes 2, 3: the tile's stage of tensor memory; lanes 0, 1: its codes
+        const uint32_t bar = stage_free ? bar_cempty + 8 * (ti % SA) : bar_wfull + 8 * (ti % SW);
+        const uint32_t par = stage_free ? (uint32_t)(((ti / SA) & 1) ^ 1) : (uint32_t)((ti / SW) & 1);
+        if (!stage_free || ti >= SA) got_c = mbar_wait(bar, par, abort_flag, p.status) ? 1 : 0;
+      }
+      got_c = __all_sync(0xffffffffu, got_c);
       if (!got_c) break;
-      // lane 0 has observed the phases and the shuffle above orders the other lanes' reads of the tiles after that
-      // (probing the barriers with all 32 lanes as well cost ~420 cycles per tile although they were complete)
       tc_fence_after();  // the MMAs that read these stages have completed (their commit released them)
       uint32_t va[32], vb[32];
       convert_row(i, va);
