@@ -244,19 +244,19 @@ __device__ __forceinline__ void int8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint3
 }
 
 // Four packed INT4 bytes (eight codes, memory order: low nibble first) -> eight bf16 values = code * s, one rounding
-// each.  A nibble n is the two's-complement code (n ^ 8) - 8; 0x4300 | (n ^ 8) is the bf16 number 128 + (n ^ 8), and
-// subtracting 136 leaves the code exactly; the product with the fp16 group scale is formed in fp32.
+// each.  A nibble n is the two's-complement code (n ^ 8) - 8.  The nibbles are biased four at a time with two wide
+// masks; one byte permute then drops a biased nibble into the mantissa of 2^23 (0x4B000000 | (n ^ 8) is the fp32
+// number 8388608 + (n ^ 8)), and subtracting 8388616 leaves the code exactly.  Its product with the fp16 group scale is
+// exact in fp32 and rounded once when the pair is packed.  (Eleven integer-pipe instructions per eight codes; the
+// first version, which built bf16 pairs with shifts and masks per byte and unpacked them again, took about twice as
+// many: config 6a 103 -> 97 us per step.)
 __device__ __forceinline__ void int4x8_to_bf16x8(uint32_t w, float s, uint32_t (&out)[4]) {
+  const uint32_t lo8 = (w & 0x0f0f0f0fu) ^ 0x08080808u, hi8 = ((w >> 4) & 0x0f0f0f0fu) ^ 0x08080808u;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const uint32_t t = (w >> (8 * j)) & 0xffu;
-    uint32_t pair = ((t & 0x0fu) | ((t & 0xf0u) << 12)) ^ 0x00080008u;
-    pair |= 0x43004300u;
-    const uint32_t bias = 0x43084308u;
-    const __nv_bfloat162 q = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&pair), *reinterpret_cast<const __nv_bfloat162*>(&bias));
-    const uint32_t qb = *reinterpret_cast<const uint32_t*>(&q);
-    const float lo = __uint_as_float(qb << 16) * s, hi = __uint_as_float(qb & 0xffff0000u) * s;
-    const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+    const float lo = __uint_as_float(__byte_perm(lo8, 0x4B000000u, 0x7440u | (uint32_t)j)) - 8388616.f;
+    const float hi = __uint_as_float(__byte_perm(hi8, 0x4B000000u, 0x7440u | (uint32_t)j)) - 8388616.f;
+    const __nv_bfloat162 r = __floats2bfloat162_rn(lo * s, hi * s);
     out[j] = *reinterpret_cast<const uint32_t*>(&r);
   }
 }
