@@ -835,8 +835,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     const int band = warp & 3;
     const int r = band * 32 + lane;
     // one row of tile i: codes from the ring slot -> 32 packed bf16 pairs
-    auto convert_row = [&](int i, uint32_t (&v)[32]) {
-      const int sr = i % SW;
+    auto convert_row = [&](int i, int sr /* = i mod SW */, uint32_t (&v)[32]) {
       if (I4) {
         // a row of the tile is 32 bytes = two 16-byte chunks, loaded with the 32-byte swizzle (chunk c of row r at
         // position c ^ ((r >> 2) & 1): again eight different bank groups per quarter-warp); the 64 codes of the row
@@ -888,30 +887,48 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
     // are shared.
     int i = 0;
     const bool two = SW >= 2 && SA >= 2;  // (tile i + 1 must not need the slot or the stage tile i still holds)
+    // Ring positions and phases of tiles i and i + 1 advance by increments: the divisions by the runtime ring depths
+    // they replace (sixteen per round, in every lane) cost more than the barrier observation itself.
+    int sr0 = 0, sr1 = SW > 1 ? 1 : 0, sa0 = 0, sa1 = SA > 1 ? 1 : 0;
+    uint32_t rph0 = 0, rph1 = 0, aph0 = 0, aph1 = 0;  // (i / SW) & 1, (i / SA) & 1 of the two tiles
     for (; two && i + 1 < nkb; i += 2) {
       // lanes 0..3 observe the four barriers of the two tiles side by side (free stages of tensor memory, landed codes:
       // one lane taking them in turn spent ~100 cycles on each although they were complete); the vote orders the other
       // lanes' reads of the tiles after that.  (Probing the barriers with all 32 lanes cost ~420 cycles per tile.)
       int got_c = 1;
       if (lane < 4) {
-        const int ti = i + (lane & 1);
+        const bool second = (lane & 1) != 0;
         const bool stage_free = lane >= 2;  // lanes 2, 3: the tile's stage of tensor memory; lanes 0, 1: its codes
-        const uint32_t bar = stage_free ? bar_cempty + 8 * (ti % SA) : bar_wfull + 8 * (ti % SW);
-        const uint32_t par = stage_free ? (uint32_t)(((ti / SA) & 1) ^ 1) : (uint32_t)((ti / SW) & 1);
-        if (!stage_free || ti >= SA) got_c = mbar_wait(bar, par, abort_flag, p.status) ? 1 : 0;
+        const uint32_t bar = stage_free ? bar_cempty + 8 * (second ? sa1 : sa0) : bar_wfull + 8 * (second ? sr1 : sr0);
+        const uint32_t par = stage_free ? ((second ? aph1 : aph0) ^ 1u) : (second ? rph1 : rph0);
+        if (!stage_free || i + (second ? 1 : 0) >= SA) got_c = mbar_wait(bar, par, abort_flag, p.status) ? 1 : 0;
       }
       got_c = __all_sync(0xffffffffu, got_c);
       if (!got_c) break;
       tc_fence_after();  // the MMAs that read these stages have completed (their commit released them)
       uint32_t va[32], vb[32];
-      convert_row(i, va);
-      convert_row(i + 1, vb);
-      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(i % SA), va);
-      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col((i + 1) % SA), vb);
+      convert_row(i, sr0, va);
+      convert_row(i + 1, sr1, vb);
+      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(sa0), va);
+      tmem_st32_issue(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(sa1), vb);
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { publish(i); publish(i + 1); }
+      if (lane == 0) {
+        if (PAIR) {
+          mbar_arrive_cluster(map_to_cta(bar_cfull + 8 * sa0, leader_rank));
+          mbar_arrive_cluster(map_to_cta(bar_cfull + 8 * sa1, leader_rank));
+        } else {
+          mbar_arrive(bar_cfull + 8 * sa0);
+          mbar_arrive(bar_cfull + 8 * sa1);
+        }
+        mbar_arrive(bar_wempty + 8 * sr0);
+        mbar_arrive(bar_wempty + 8 * sr1);
+      }
+      sr0 += 2; if (sr0 >= SW) { sr0 -= SW; rph0 ^= 1u; }
+      sr1 += 2; if (sr1 >= SW) { sr1 -= SW; rph1 ^= 1u; }
+      sa0 += 2; if (sa0 >= SA) { sa0 -= SA; aph0 ^= 1u; }
+      sa1 += 2; if (sa1 >= SA) { sa1 -= SA; aph1 ^= 1u; }
     }
     for (; i < nkb; ++i) {  // an odd last tile (or every tile, with a ring of one)
       int got_c = 1;
@@ -920,7 +937,7 @@ essa_decode_kernel(const __grid_constant__ DMaps maps, const __grid_constant__ D
       if (!got_c) break;
       tc_fence_after();
       uint32_t va[32];
-      convert_row(i, va);
+      convert_row(i, i % SW, va);
       tmem_st32(tmem_base + ((uint32_t)(band * 32) << 16) + tmem_a_col(i % SA), va);
       tc_fence_before();
       __syncwarp();
