@@ -52,8 +52,8 @@ NCU_TRAFFIC = {
           "note": "captured at half the population (425.2 MB) and scaled: W0 traffic fixed, x and y traffic doubled"},
     "4": {"bytes": 4787e6, "source": "proj_tc3.cu", "sha16": "13fd60855285679d", "profile": "profiles/essa_tcw_kernel_cfg2_cfg4_prefill.md",
           "note": "full size; captures of the same kernel range from 3.4 to 5.4 GB (how well the CTA pairs stay in step)"},
-    "3": {"bytes": 67.9e6, "source": "proj_decode.cu", "sha16": "7e076f5f416101ec", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
-    "5a": {"bytes": 170.5e6, "source": "proj_decode.cu", "sha16": "7e076f5f416101ec", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
+    "3": {"bytes": 67.9e6, "source": "proj_decode.cu", "sha16": "853fbc3271e38da6", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
+    "5a": {"bytes": 170.7e6, "source": "proj_decode.cu", "sha16": "853fbc3271e38da6", "profile": "profiles/essa_decode_kernel_cfg3_cfg5a.md"},
 }
 
 
